@@ -1,0 +1,217 @@
+/*
+ * xkv - compressed KV cache for streaming frame-causal attention on one GPU.
+ *
+ * C ABI of the library.  One `xkv_cache` holds the key/value cache of ONE
+ * global-attention layer under joint pruning and quantisation (Sec. 3.2-3.3 of
+ * the paper).  Per incoming frame the caller runs, in this order,
+ *
+ *     kv_append -> kv_score_evict -> kv_quant_pack -> attn_packed_causal
+ *
+ * or xkv_stream_step, which does the same for a stack of layers.
+ *
+ * Conventions
+ *   - Pointers named q, k, v, out and dev_workspace are DEVICE pointers; every
+ *     other pointer is a HOST pointer.  All device pointers must be 16-byte
+ *     aligned.  Q/K/V/out are bf16 (16-bit, truncated-fp32 format).
+ *   - A frame tensor is addressed as  base[head*head_stride + token*tok_stride + c],
+ *     c = 0..head_dim-1 contiguous, strides in ELEMENTS and multiples of 8.
+ *     [H][n][d] is (tok_stride=d, head_stride=n*d); [n][H*d] is (H*d, d).
+ *   - The first n_special tokens of a frame are its camera and register tokens,
+ *     the rest its patch tokens in raster order (Sec. 3.1).
+ *   - Calls are stream-ordered and never synchronise, allocate device memory or
+ *     read device data on the host (exceptions: xkv_debug_export,
+ *     xkv_poll_status, xkv_stream_step_host).  All cache lengths are functions
+ *     of the frame sizes seen so far and the budget, so they are tracked on the
+ *     host.
+ *   - The caller owns the workspace; the library never frees it.  Memory use of
+ *     a cache is constant for its lifetime.
+ *   - Every function returns XKV_OK (0) or a negative xkv_status.  Nothing
+ *     throws, aborts or traps.  A cache is not thread-safe; different caches may
+ *     be driven from different threads/streams.
+ */
+#ifndef XKV_H_
+#define XKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define XKV_API __attribute__((visibility("default")))
+#else
+#define XKV_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct xkv_cache xkv_cache;          /* opaque, host-side handle of one layer's cache */
+typedef void* xkv_stream;                    /* a cudaStream_t, passed as a plain pointer     */
+
+typedef enum {
+  XKV_OK            =  0,
+  XKV_E_INVALID     = -1,   /* bad argument (null, misaligned, out of range)          */
+  XKV_E_STATE       = -2,   /* call out of order for this cache                        */
+  XKV_E_NOMEM       = -3,   /* workspace too small / host allocation failed            */
+  XKV_E_UNSUPPORTED = -4,   /* parameter combination not implemented                   */
+  XKV_E_CUDA        = -5,   /* a CUDA runtime/driver call failed                       */
+  XKV_E_TIMEOUT     = -6    /* a bounded device-side wait ran out (see xkv_poll_status)*/
+} xkv_status;
+
+/* Method parameters.  Defaults of the paper: n_special = 5 (1 camera + 4
+ * register tokens, Sec. 3.1), pool_g = 16, quant_group = 64, kv_bits = 4
+ * (Sec. 4.1).  kv_bits = 16 keeps bf16 values (pruning only). */
+typedef struct {
+  int32_t n_heads;           /* H, 1..64                                                 */
+  int32_t head_dim;          /* d, only 64                                               */
+  int32_t n_special;         /* special tokens at the head of each frame, >= 0           */
+  int32_t pool_g;            /* g of GroupAvg (Eq. 2), >= 1                              */
+  int32_t quant_group;       /* G, cache positions per key group, only 64                */
+  int32_t kv_bits;           /* b: 4 or 16                                               */
+  int32_t budget;            /* L_max, the token budget (Sec. 3.2), >= 1                 */
+  int32_t max_frame_tokens;  /* largest n any frame will have, 1..65535                  */
+} xkv_params;
+
+/* Host-side counters and geometry; filled without touching the device. */
+typedef struct {
+  int32_t frames;            /* frames appended so far                                   */
+  int32_t T;                 /* tokens in the packed cache                               */
+  int32_t T_first;           /* tokens of the first frame                                */
+  int32_t rest_base;         /* physical slot where the rest segment starts (128-aligned)*/
+  int32_t T_phys;            /* physical slots in use = rest_base + (T - T_first)        */
+  int32_t capacity;          /* physical slots per head                                  */
+  int32_t cur;               /* which of the two buffer sets is current (0/1)            */
+  int32_t last_evicted;      /* tokens evicted by the last kv_score_evict                */
+  int32_t last_kept;         /* middle tokens kept by the last kv_score_evict            */
+  int32_t last_prunable;     /* size of the middle segment at the last kv_score_evict    */
+  int32_t stage;             /* 0 idle, 1 appended, 2 scored, 3 packed                   */
+  int32_t n_pending;         /* tokens of the frame in flight                            */
+  int64_t launches;          /* kernels launched for this cache so far                   */
+  uint64_t workspace_bytes;
+} xkv_info;
+
+/* Sub-buffers that xkv_debug_export can copy out (physical layout, current
+ * buffer set).  Slot p of head h: logical token j lives at p = j for
+ * j < T_first and at p = rest_base + (j - T_first) otherwise.
+ *   K_CODES / V_CODES : kv_bits = 4 : uint8 [H][capacity][d/2]; the 8 codes of channels
+ *                       8w..8w+7 form the little-endian 32-bit word
+ *                       c0 | c2<<4 | c4<<8 | c6<<12 | c1<<16 | c3<<20 | c5<<24 | c7<<28
+ *                       kv_bits = 16: bf16 [H][capacity][d]
+ *   K_PARAMS          : float2 (scale, zero) [H][capacity/64][d], group = 64 slots
+ *   V_PARAMS          : float2 (scale, zero) [H][capacity]
+ *   ORIGIN            : int32 [capacity], (frame << 16) | token, frame counted from 1
+ *   SCORES            : float [last_prunable]  importance scores S of Eq. 6 (last evicting step)
+ *   KEPT              : int32 [last_kept]      kept middle positions, ascending (last evicting step)
+ *   QVEC              : float [d]              row mean of the pooled query (last evicting step)
+ */
+typedef enum {
+  XKV_BUF_K_CODES = 0, XKV_BUF_K_PARAMS = 1, XKV_BUF_V_CODES = 2, XKV_BUF_V_PARAMS = 3,
+  XKV_BUF_ORIGIN = 4, XKV_BUF_SCORES = 5, XKV_BUF_KEPT = 6, XKV_BUF_QVEC = 7
+} xkv_buffer;
+
+/* ---- set-up ---------------------------------------------------------------- */
+
+/* Bytes of device workspace one cache needs; 0 if the parameters are invalid. */
+XKV_API size_t xkv_workspace_bytes(const xkv_params* params);
+
+/* Create a cache on `dev_workspace` (device memory, 256-byte aligned, at least
+ * xkv_workspace_bytes(params) bytes, on the current device).  Zero-fills the
+ * workspace on `stream`.  *out receives the handle. */
+XKV_API int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes,
+               xkv_stream stream, xkv_cache** out);
+
+/* Back to the empty state on the same workspace (stream-ordered zero-fill). */
+XKV_API int xkv_reset(xkv_cache* cache, xkv_stream stream);
+
+/* Free the host handle.  The workspace stays with the caller. */
+XKV_API int xkv_destroy(xkv_cache* cache);
+
+/* ---- the per-frame calls --------------------------------------------------- */
+
+/* Step 1 (Sec. 3.1, the text after Eq. 1: the new frame joins the cache).  Takes frame
+ * t's keys and values, n tokens, into the cache: values are quantised per token
+ * (Eq. 7-9) straight into their final slot; keys are staged until kv_quant_pack.
+ * k and v may be reused once the stream has passed this call.  At t = 1 this
+ * fixes T_first = n.  Errors: XKV_E_STATE unless the cache is idle;
+ * XKV_E_INVALID for n < 1, n > max_frame_tokens, bad strides or pointers. */
+XKV_API int kv_append(xkv_cache* cache, const void* k, const void* v, int32_t n,
+              int64_t tok_stride, int64_t head_stride, xkv_stream stream);
+
+/* Steps 2-3 (Sec. 3.2, Eq. 2-6).  If the cache length T after the append
+ * exceeds the budget: pooled query (special tokens kept, patch tokens averaged
+ * in groups of g, then averaged over heads), head-averaged dequantised keys of
+ * the middle segment, scores S, and the k = max(0, L_max - T_first - n) highest
+ * scores kept (ties: lower position wins), in ascending position.  Otherwise a
+ * no-op.  q is frame t's query, same n as the append.  Errors: XKV_E_STATE
+ * unless kv_append was the previous call; XKV_E_INVALID as above. */
+XKV_API int kv_score_evict(xkv_cache* cache, const void* q, int32_t n,
+                   int64_t tok_stride, int64_t head_stride, xkv_stream stream);
+
+/* Step 4 (Sec. 3.3, Eq. 7-9).  Builds the final cache = first frame, surviving
+ * middle tokens, current frame: survivors' value codes and parameters are
+ * gathered; the keys after the first frame are regrouped into runs of 64 and
+ * re-quantised per channel (a complete group whose tokens all survive in place
+ * is carried over unchanged).  Afterwards T <= max(L_max, T_first + n).
+ * Errors: XKV_E_STATE unless kv_score_evict was the previous call. */
+XKV_API int kv_quant_pack(xkv_cache* cache, xkv_stream stream);
+
+/* Step 5 (Eq. 1 with the dequantisation of Eq. 10).  out = softmax(q K~^T *
+ * softmax_scale) V~ per head over all T cached tokens (all of them belong to
+ * frames <= t, so the frame-causal mask hides nothing).  out has the strides of
+ * q.  impl: 0 = default (tensor-core kernel), 1 = the simple CUDA-core kernel
+ * kept as a cross-check.  Errors: XKV_E_STATE unless kv_quant_pack was the
+ * previous call (the cache returns to idle); XKV_E_INVALID as above. */
+XKV_API int attn_packed_causal(xkv_cache* cache, const void* q, void* out, int32_t n,
+                       int64_t tok_stride, int64_t head_stride, float softmax_scale,
+                       int32_t impl, xkv_stream stream);
+
+/* One frame through a stack of layers: for each layer in order, the four calls
+ * above with softmax_scale = 1/sqrt(head_dim).  q, k, v, out are HOST arrays of
+ * n_layers DEVICE pointers.  Stops at the first error and returns it. */
+XKV_API int xkv_stream_step(xkv_cache* const* layers, int32_t n_layers,
+                    const void* const* q, const void* const* k, const void* const* v,
+                    void* const* out, int32_t n, int64_t tok_stride, int64_t head_stride,
+                    xkv_stream stream);
+
+/* The same step for callers whose tensors live in HOST memory (pinned memory
+ * gives asynchronous copies).  q, k, v, out are HOST arrays of n_layers HOST
+ * pointers to bf16 [H][n][d] tensors; dev_staging is device scratch of at least
+ * xkv_stream_step_host_bytes(layers[0] params, n) bytes.  Copies layer by layer
+ * on `stream`, runs the layer, copies the output back, and synchronises the
+ * stream before returning. */
+XKV_API size_t xkv_stream_step_host_bytes(const xkv_params* params, int32_t n);
+XKV_API int xkv_stream_step_host(xkv_cache* const* layers, int32_t n_layers,
+                         const void* const* q, const void* const* k, const void* const* v,
+                         void* const* out, int32_t n, void* dev_staging, size_t staging_bytes,
+                         xkv_stream stream);
+
+/* ---- introspection ---------------------------------------------------------- */
+
+XKV_API int xkv_get_info(const xkv_cache* cache, xkv_info* info);
+
+/* Tests only: synchronises `stream`, then copies up to `bytes` bytes of one
+ * sub-buffer of the current buffer set to host_dst.  Returns the number of bytes
+ * copied (>= 0) or a negative xkv_status. */
+XKV_API int64_t xkv_debug_export(const xkv_cache* cache, int32_t which, void* host_dst, size_t bytes,
+                         xkv_stream stream);
+
+/* Synchronises `stream` and returns the device status word of the cache:
+ * XKV_OK, or XKV_E_TIMEOUT if a bounded wait inside a kernel ran out. */
+XKV_API int xkv_poll_status(const xkv_cache* cache, xkv_stream stream);
+
+XKV_API const char* xkv_strerror(int status);
+
+/* ---- synthetic inputs (not part of the method) -------------------------------- */
+
+/* Fills dst (device, bf16 [n_heads][n_tokens][head_dim]) with the seeded
+ * Irwin-Hall(12) variates of the input recipe: element e of the tensor is built
+ * from three 64-bit hash words of (key + 3e + i); entries of outlier_channels
+ * (HOST int32 [n_heads][n_outliers], may be null) are multiplied by `gain`. */
+XKV_API int xkv_synth_fill(void* dst, uint64_t key, int32_t n_heads, int32_t n_tokens, int32_t head_dim,
+                   const int32_t* outlier_channels, int32_t n_outliers, float gain,
+                   xkv_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* XKV_H_ */

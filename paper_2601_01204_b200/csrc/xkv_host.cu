@@ -1,0 +1,411 @@
+// Host side of libxkv: workspace layout, the per-cache call-order state machine,
+// the C ABI, and the synthetic-input generator kernel.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "xkv_internal.cuh"
+
+using namespace xkv;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+
+struct Layout {
+  int cap, row_bytes;
+  size_t off_k[2], off_kpar[2], off_v[2], off_vpar[2], off_origin[2];
+  size_t off_kstage, off_qbar, off_qvec, off_scores, off_kept, off_counters, off_status, off_attn;
+  size_t attn_bytes;
+  size_t total;
+};
+
+bool params_ok(const xkv_params* p) {
+  if (!p) return false;
+  if (p->n_heads < 1 || p->n_heads > 64) return false;
+  if (p->head_dim != kHeadDim || p->quant_group != kGroup) return false;
+  if (p->kv_bits != 4 && p->kv_bits != 16) return false;
+  if (p->n_special < 0 || p->pool_g < 1 || p->budget < 1) return false;
+  if (p->max_frame_tokens < 1 || p->max_frame_tokens > 65535) return false;
+  if (p->budget > (1 << 24)) return false;
+  return true;
+}
+
+Layout make_layout(const xkv_params* p) {
+  Layout L;
+  memset(&L, 0, sizeof(L));
+  const int max_n = p->max_frame_tokens;
+  // first segment padded to a tile; rest holds at most max(budget, max_n) tokens after a step
+  const int cap_first = round_up(max_n, kTile);
+  const int cap_rest = round_up(p->budget > max_n ? p->budget : max_n, kTile) + kTile;
+  L.cap = cap_first + cap_rest;
+  L.row_bytes = (p->kv_bits == 4) ? 32 : 128;
+  const size_t H = (size_t)p->n_heads;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += (bytes + kAlign - 1) / kAlign * kAlign; return o; };
+  L.off_status = take(256);
+  L.off_counters = take(256);
+  for (int b = 0; b < 2; ++b) {
+    L.off_k[b] = take(H * L.cap * L.row_bytes);
+    L.off_kpar[b] = take(H * (L.cap / 64) * 64 * sizeof(float2));
+    L.off_v[b] = take(H * L.cap * L.row_bytes);
+    L.off_vpar[b] = take(H * L.cap * sizeof(float2));
+    L.off_origin[b] = take((size_t)L.cap * sizeof(int32_t));
+  }
+  L.off_kstage = take(H * max_n * 64 * sizeof(__nv_bfloat16));
+  const int np_max = max_n;  // upper bound of N_pooled
+  L.off_qbar = take((size_t)np_max * 64 * sizeof(float));
+  L.off_qvec = take(64 * sizeof(float));
+  L.off_scores = take((size_t)L.cap * sizeof(float));
+  L.off_kept = take((size_t)L.cap * sizeof(int32_t));
+  L.attn_bytes = attn_tc_scratch_bytes(p);
+  L.off_attn = take(L.attn_bytes);
+  L.total = off;
+  return L;
+}
+
+bool strides_ok(int64_t ts, int64_t hs) { return ts >= kHeadDim && (ts % 8) == 0 && hs >= 0 && (hs % 8) == 0; }
+bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int zero_workspace(xkv_cache* c, cudaStream_t st) {
+  return cudaMemsetAsync(c->ws, 0, c->ws_bytes, st) == cudaSuccess ? XKV_OK : XKV_E_CUDA;
+}
+
+void reset_host_state(xkv_cache* c) {
+  c->frames = c->T = c->T_first = c->rest_base = c->cur = c->stage = 0;
+  c->n_pending = c->kk_pending = c->rold_pending = c->evict_pending = c->first_pending = 0;
+  c->last_evicted = c->last_kept = c->last_prunable = 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t xkv_workspace_bytes(const xkv_params* params) {
+  if (!params_ok(params)) return 0;
+  return make_layout(params).total;
+}
+
+int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_stream stream, xkv_cache** out) {
+  if (!out) return XKV_E_INVALID;
+  *out = nullptr;
+  if (!params) return XKV_E_INVALID;
+  if (!params_ok(params)) {
+    if (params->head_dim != kHeadDim && params->head_dim > 0) return XKV_E_UNSUPPORTED;
+    if (params->quant_group != kGroup && params->quant_group > 0) return XKV_E_UNSUPPORTED;
+    if (params->kv_bits == 2 || params->kv_bits == 8) return XKV_E_UNSUPPORTED;
+    return XKV_E_INVALID;
+  }
+  if (!dev_workspace || (reinterpret_cast<uintptr_t>(dev_workspace) % kAlign) != 0) return XKV_E_INVALID;
+  const Layout L = make_layout(params);
+  if (bytes < L.total) return XKV_E_NOMEM;
+  xkv_cache* c = new (std::nothrow) xkv_cache;
+  if (!c) return XKV_E_NOMEM;
+  memset(c, 0, sizeof(*c));
+  c->p = *params;
+  c->cap = L.cap;
+  c->row_bytes = L.row_bytes;
+  c->ws = reinterpret_cast<uint8_t*>(dev_workspace);
+  c->ws_bytes = L.total;
+  for (int b = 0; b < 2; ++b) {
+    c->buf[b].k = c->ws + L.off_k[b];
+    c->buf[b].kpar = reinterpret_cast<float2*>(c->ws + L.off_kpar[b]);
+    c->buf[b].v = c->ws + L.off_v[b];
+    c->buf[b].vpar = reinterpret_cast<float2*>(c->ws + L.off_vpar[b]);
+    c->buf[b].origin = reinterpret_cast<int32_t*>(c->ws + L.off_origin[b]);
+  }
+  c->kstage = reinterpret_cast<__nv_bfloat16*>(c->ws + L.off_kstage);
+  c->qbar = reinterpret_cast<float*>(c->ws + L.off_qbar);
+  c->qvec = reinterpret_cast<float*>(c->ws + L.off_qvec);
+  c->scores = reinterpret_cast<float*>(c->ws + L.off_scores);
+  c->kept = reinterpret_cast<int32_t*>(c->ws + L.off_kept);
+  c->counters = reinterpret_cast<unsigned int*>(c->ws + L.off_counters);
+  c->status = reinterpret_cast<int*>(c->ws + L.off_status);
+  c->attn_part = reinterpret_cast<float*>(c->ws + L.off_attn);
+  c->attn_part_bytes = L.attn_bytes;
+  reset_host_state(c);
+  const int rc = zero_workspace(c, reinterpret_cast<cudaStream_t>(stream));
+  if (rc != XKV_OK) { delete c; return rc; }
+  *out = c;
+  return XKV_OK;
+}
+
+int xkv_reset(xkv_cache* c, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  reset_host_state(c);
+  return zero_workspace(c, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int xkv_destroy(xkv_cache* c) {
+  if (!c) return XKV_E_INVALID;
+  delete c;
+  return XKV_OK;
+}
+
+int kv_append(xkv_cache* c, const void* k, const void* v, int32_t n, int64_t ts, int64_t hs, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  if (c->stage != 0) return XKV_E_STATE;
+  if (n < 1 || n > c->p.max_frame_tokens || !aligned16(k) || !aligned16(v) || !strides_ok(ts, hs))
+    return XKV_E_INVALID;
+  const bool first = (c->frames == 0);
+  int r_old = 0, kk = 0, evict = 0, dst_slot = 0;
+  if (!first) {
+    r_old = c->T - c->T_first;
+    evict = (c->T + n > c->p.budget) ? 1 : 0;               // pruning is triggered when T > L_max (Sec. 3.2)
+    kk = evict ? (c->p.budget - c->T_first - n) : r_old;    // k = max(0, L_max - T_first - T_current)
+    if (kk < 0) kk = 0;
+    dst_slot = c->rest_base + kk;
+    if (dst_slot + n > c->cap) return XKV_E_NOMEM;
+  }
+  const cudaError_t e = launch_append(c, k, v, n, ts, hs, dst_slot, first, reinterpret_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return XKV_E_CUDA;
+  c->n_pending = n;
+  c->kk_pending = kk;
+  c->rold_pending = r_old;
+  c->evict_pending = evict;
+  c->first_pending = first ? 1 : 0;
+  c->stage = 1;
+  return XKV_OK;
+}
+
+int kv_score_evict(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t hs, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  if (c->stage != 1) return XKV_E_STATE;
+  if (n != c->n_pending || !aligned16(q) || !strides_ok(ts, hs)) return XKV_E_INVALID;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  c->last_evicted = 0;
+  if (c->evict_pending) {
+    const int r_old = c->rold_pending, kk = c->kk_pending;
+    c->last_prunable = r_old;
+    c->last_kept = kk;
+    c->last_evicted = r_old - kk;
+    if (kk > 0 && kk < r_old) {
+      if (launch_pool_q(c, q, n, ts, hs, st) != cudaSuccess) return XKV_E_CUDA;
+      if (launch_score(c, r_old, st) != cudaSuccess) return XKV_E_CUDA;
+      if (launch_select(c, r_old, kk, st) != cudaSuccess) return XKV_E_CUDA;
+    }
+  }
+  c->stage = 2;
+  return XKV_OK;
+}
+
+int kv_quant_pack(xkv_cache* c, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  if (c->stage != 2) return XKV_E_STATE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int n = c->n_pending, kk = c->kk_pending;
+  const bool first = c->first_pending != 0;
+  const bool identity = !(c->evict_pending && kk > 0 && kk < c->rold_pending);
+  if (launch_pack(c, n, kk, identity, first, st) != cudaSuccess) return XKV_E_CUDA;
+  if (first) {
+    c->T_first = n;
+    c->rest_base = round_up(n, kTile);
+    c->T = n;
+  } else {
+    c->T = c->T_first + kk + n;
+    c->cur ^= 1;
+  }
+  c->frames += 1;
+  c->stage = 3;
+  return XKV_OK;
+}
+
+int attn_packed_causal(xkv_cache* c, const void* q, void* out, int32_t n, int64_t ts, int64_t hs,
+                       float softmax_scale, int32_t impl, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  if (c->stage != 3) return XKV_E_STATE;
+  if (n < 1 || n > c->p.max_frame_tokens || !aligned16(q) || !aligned16(out) || !strides_ok(ts, hs) ||
+      !(softmax_scale > 0.f) || (impl != 0 && impl != 1))
+    return XKV_E_INVALID;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  cudaError_t e;
+  if (impl == 1) {
+    e = launch_attn_simple(c, q, out, n, ts, hs, softmax_scale, st);
+  } else {
+    e = launch_attn_tc(c, q, out, n, ts, hs, softmax_scale, st);
+    if (e == cudaErrorNotSupported) return XKV_E_UNSUPPORTED;
+  }
+  if (e != cudaSuccess) return XKV_E_CUDA;
+  c->stage = 0;
+  return XKV_OK;
+}
+
+int xkv_stream_step(xkv_cache* const* layers, int32_t n_layers, const void* const* q, const void* const* k,
+                    const void* const* v, void* const* out, int32_t n, int64_t ts, int64_t hs,
+                    xkv_stream stream) {
+  if (!layers || !q || !k || !v || !out || n_layers < 1) return XKV_E_INVALID;
+  for (int l = 0; l < n_layers; ++l) {
+    xkv_cache* c = layers[l];
+    if (!c) return XKV_E_INVALID;
+    int rc = kv_append(c, k[l], v[l], n, ts, hs, stream);
+    if (rc != XKV_OK) return rc;
+    rc = kv_score_evict(c, q[l], n, ts, hs, stream);
+    if (rc != XKV_OK) return rc;
+    rc = kv_quant_pack(c, stream);
+    if (rc != XKV_OK) return rc;
+    rc = attn_packed_causal(c, q[l], out[l], n, ts, hs, 1.0f / sqrtf((float)c->p.head_dim), 0, stream);
+    if (rc != XKV_OK) return rc;
+  }
+  return XKV_OK;
+}
+
+size_t xkv_stream_step_host_bytes(const xkv_params* params, int32_t n) {
+  if (!params_ok(params) || n < 1) return 0;
+  // two slots (double buffering) of Q, K, V, out
+  const size_t t = (size_t)params->n_heads * n * kHeadDim * sizeof(__nv_bfloat16);
+  return 2 * 4 * ((t + kAlign - 1) / kAlign * kAlign);
+}
+
+int xkv_stream_step_host(xkv_cache* const* layers, int32_t n_layers, const void* const* q,
+                         const void* const* k, const void* const* v, void* const* out, int32_t n,
+                         void* dev_staging, size_t staging_bytes, xkv_stream stream) {
+  if (!layers || !q || !k || !v || !out || n_layers < 1 || !layers[0] || !dev_staging) return XKV_E_INVALID;
+  const xkv_params* p = &layers[0]->p;
+  if (n < 1 || n > p->max_frame_tokens) return XKV_E_INVALID;
+  if (staging_bytes < xkv_stream_step_host_bytes(p, n)) return XKV_E_NOMEM;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const size_t t = (size_t)p->n_heads * n * kHeadDim * sizeof(__nv_bfloat16);
+  const size_t slot = (t + kAlign - 1) / kAlign * kAlign;
+  uint8_t* base = reinterpret_cast<uint8_t*>(dev_staging);
+  const int64_t ts = kHeadDim, hs = (int64_t)n * kHeadDim;
+  for (int l = 0; l < n_layers; ++l) {
+    xkv_cache* c = layers[l];
+    if (!c || !q[l] || !k[l] || !v[l] || !out[l]) return XKV_E_INVALID;
+    uint8_t* s = base + (size_t)(l & 1) * 4 * slot;
+    void* dq = s;
+    void* dk = s + slot;
+    void* dv = s + 2 * slot;
+    void* dout = s + 3 * slot;
+    if (cudaMemcpyAsync(dk, k[l], t, cudaMemcpyHostToDevice, st) != cudaSuccess) return XKV_E_CUDA;
+    if (cudaMemcpyAsync(dv, v[l], t, cudaMemcpyHostToDevice, st) != cudaSuccess) return XKV_E_CUDA;
+    if (cudaMemcpyAsync(dq, q[l], t, cudaMemcpyHostToDevice, st) != cudaSuccess) return XKV_E_CUDA;
+    int rc = kv_append(c, dk, dv, n, ts, hs, stream);
+    if (rc != XKV_OK) return rc;
+    rc = kv_score_evict(c, dq, n, ts, hs, stream);
+    if (rc != XKV_OK) return rc;
+    rc = kv_quant_pack(c, stream);
+    if (rc != XKV_OK) return rc;
+    rc = attn_packed_causal(c, dq, dout, n, ts, hs, 1.0f / sqrtf((float)p->head_dim), 0, stream);
+    if (rc != XKV_OK) return rc;
+    if (cudaMemcpyAsync(out[l], dout, t, cudaMemcpyDeviceToHost, st) != cudaSuccess) return XKV_E_CUDA;
+  }
+  return cudaStreamSynchronize(st) == cudaSuccess ? XKV_OK : XKV_E_CUDA;
+}
+
+int xkv_get_info(const xkv_cache* c, xkv_info* info) {
+  if (!c || !info) return XKV_E_INVALID;
+  info->frames = c->frames;
+  info->T = c->T;
+  info->T_first = c->T_first;
+  info->rest_base = c->rest_base;
+  info->T_phys = c->rest_base + (c->T - c->T_first);
+  info->capacity = c->cap;
+  info->cur = c->cur;
+  info->last_evicted = c->last_evicted;
+  info->last_kept = c->last_kept;
+  info->last_prunable = c->last_prunable;
+  info->stage = c->stage;
+  info->n_pending = c->n_pending;
+  info->launches = c->launches;
+  info->workspace_bytes = c->ws_bytes;
+  return XKV_OK;
+}
+
+int64_t xkv_debug_export(const xkv_cache* c, int32_t which, void* host_dst, size_t bytes, xkv_stream stream) {
+  if (!c || !host_dst) return XKV_E_INVALID;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return XKV_E_CUDA;
+  const BufSet& b = c->buf[c->cur];
+  const size_t H = (size_t)c->p.n_heads;
+  const void* src = nullptr;
+  size_t avail = 0;
+  switch (which) {
+    case XKV_BUF_K_CODES: src = b.k; avail = H * c->cap * c->row_bytes; break;
+    case XKV_BUF_K_PARAMS: src = b.kpar; avail = H * (c->cap / 64) * 64 * sizeof(float2); break;
+    case XKV_BUF_V_CODES: src = b.v; avail = H * c->cap * c->row_bytes; break;
+    case XKV_BUF_V_PARAMS: src = b.vpar; avail = H * c->cap * sizeof(float2); break;
+    case XKV_BUF_ORIGIN: src = b.origin; avail = (size_t)c->cap * sizeof(int32_t); break;
+    case XKV_BUF_SCORES: src = c->scores; avail = (size_t)c->last_prunable * sizeof(float); break;
+    case XKV_BUF_KEPT: src = c->kept; avail = (size_t)c->last_kept * sizeof(int32_t); break;
+    case XKV_BUF_QVEC: src = c->qvec; avail = 64 * sizeof(float); break;
+    default: return XKV_E_INVALID;
+  }
+  const size_t nbytes = bytes < avail ? bytes : avail;
+  if (nbytes && cudaMemcpy(host_dst, src, nbytes, cudaMemcpyDeviceToHost) != cudaSuccess) return XKV_E_CUDA;
+  return (int64_t)nbytes;
+}
+
+int xkv_poll_status(const xkv_cache* c, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
+  int word = 0;
+  if (cudaMemcpy(&word, c->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return XKV_E_CUDA;
+  return word == 0 ? XKV_OK : XKV_E_TIMEOUT;
+}
+
+const char* xkv_strerror(int status) {
+  switch (status) {
+    case XKV_OK: return "ok";
+    case XKV_E_INVALID: return "invalid argument";
+    case XKV_E_STATE: return "call out of order for this cache";
+    case XKV_E_NOMEM: return "workspace too small or host allocation failed";
+    case XKV_E_UNSUPPORTED: return "parameter combination not supported";
+    case XKV_E_CUDA: return "CUDA call failed";
+    case XKV_E_TIMEOUT: return "bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------
+// Synthetic inputs: integer hash -> sum of twelve 16-bit fields -> bf16.
+// ---------------------------------------------------------------------------
+namespace {
+
+struct OutlierTable { int32_t ch[64 * 4]; };
+
+__device__ __forceinline__ uint64_t mix64(uint64_t x) {
+  x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
+  x ^= x >> 27; x *= 0x94D049BB133111EBull;
+  x ^= x >> 31;
+  return x;
+}
+
+__global__ void synth_kernel(__nv_bfloat16* dst, uint64_t key, long long count, int n_tokens, int head_dim,
+                             OutlierTable tab, int n_out, float gain) {
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= count) return;
+  int u = 0;
+#pragma unroll
+  for (int i = 0; i < 3; ++i) {
+    const uint64_t w = mix64(key + 3ull * (uint64_t)e + (uint64_t)i);
+    u += (int)(w & 0xFFFF) + (int)((w >> 16) & 0xFFFF) + (int)((w >> 32) & 0xFFFF) + (int)(w >> 48);
+  }
+  float x = __fmul_rn((float)(u - 6 * 65535), 1.52587890625e-05f);
+  const int c = (int)(e % head_dim);
+  const int h = (int)(e / ((long long)n_tokens * head_dim));
+  for (int j = 0; j < n_out; ++j)
+    if (tab.ch[h * 4 + j] == c) x = __fmul_rn(x, gain);
+  dst[e] = __float2bfloat16_rn(x);
+}
+
+}  // namespace
+
+extern "C" int xkv_synth_fill(void* dst, uint64_t key, int32_t n_heads, int32_t n_tokens, int32_t head_dim,
+                              const int32_t* outlier_channels, int32_t n_outliers, float gain,
+                              xkv_stream stream) {
+  if (!dst || n_heads < 1 || n_heads > 64 || n_tokens < 1 || head_dim < 1 || n_outliers < 0 || n_outliers > 4)
+    return XKV_E_INVALID;
+  if (n_outliers > 0 && !outlier_channels) return XKV_E_INVALID;
+  OutlierTable tab;
+  for (int i = 0; i < 64 * 4; ++i) tab.ch[i] = -1;
+  for (int h = 0; h < n_heads; ++h)
+    for (int j = 0; j < n_outliers; ++j) tab.ch[h * 4 + j] = outlier_channels[h * n_outliers + j];
+  const long long count = (long long)n_heads * n_tokens * head_dim;
+  synth_kernel<<<(int)((count + 255) / 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      reinterpret_cast<__nv_bfloat16*>(dst), key, count, n_tokens, head_dim, tab, n_outliers, gain);
+  return cudaGetLastError() == cudaSuccess ? XKV_OK : XKV_E_CUDA;
+}

@@ -1,0 +1,74 @@
+// Internal declarations shared by the translation units of libxkv.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "xkv.h"
+
+namespace xkv {
+
+constexpr int kHeadDim = 64;          // d
+constexpr int kGroup = 64;            // G: cache slots per key group (Sec. 4.1)
+constexpr int kTile = 128;            // key slots per attention tile; segment alignment
+constexpr int kWordsPerRow = 8;       // 32-bit words of one packed 4-bit row (64 codes)
+
+// One of the two buffer sets of a cache (physical layout, see xkv.h).
+struct BufSet {
+  uint8_t* k;        // [H][cap][row_bytes]
+  float2* kpar;      // [H][cap/64][64]   (scale, zero)
+  uint8_t* v;        // [H][cap][row_bytes]
+  float2* vpar;      // [H][cap]          (scale, zero)
+  int32_t* origin;   // [cap]
+};
+
+}  // namespace xkv
+
+// Host-side state of one layer's cache.
+struct xkv_cache {
+  xkv_params p;
+  // geometry
+  int cap;            // physical slots per head (multiple of 128)
+  int row_bytes;      // 32 (4-bit) or 128 (bf16)
+  size_t ws_bytes;
+  uint8_t* ws;
+  xkv::BufSet buf[2];
+  __nv_bfloat16* kstage;   // [H][max_n][64] staged keys of the frame in flight (4-bit mode)
+  float* qbar;             // [Np_max][64]
+  float* qvec;             // [64]
+  float* scores;           // [cap]
+  int32_t* kept;           // [cap]
+  unsigned int* counters;  // [8] device counters (self-resetting)
+  int* status;             // device status word
+  float* attn_part;        // split-KV partials of the attention kernel
+  size_t attn_part_bytes;
+  // stream state (host)
+  int frames, T, T_first, rest_base, cur, stage;
+  int n_pending, kk_pending, rold_pending, evict_pending, first_pending;
+  int last_evicted, last_kept, last_prunable;
+  long long launches;
+};
+
+namespace xkv {
+
+inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// ---- launchers implemented in the kernel translation units -------------------
+// All return cudaError_t of the launch (cudaGetLastError) and count launches.
+
+cudaError_t launch_append(xkv_cache* c, const void* k, const void* v, int n, int64_t ts, int64_t hs,
+                          int dst_slot, bool first, cudaStream_t st);
+cudaError_t launch_pool_q(xkv_cache* c, const void* q, int n, int64_t ts, int64_t hs, cudaStream_t st);
+cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st);
+cudaError_t launch_select(xkv_cache* c, int r_old, int k, cudaStream_t st);
+cudaError_t launch_pack(xkv_cache* c, int n, int kk, bool identity, bool first, cudaStream_t st);
+cudaError_t launch_attn_simple(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
+                               float scale, cudaStream_t st);
+// Returns cudaErrorNotSupported when the tensor-core kernel cannot take the call.
+cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
+                           float scale, cudaStream_t st);
+size_t attn_tc_scratch_bytes(const xkv_params* p);
+
+}  // namespace xkv

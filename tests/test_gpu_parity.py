@@ -1,0 +1,126 @@
+"""GPU parity: the CUDA library against the CPU oracle on the same seeded frames.
+
+Integer results (kept indices, 4-bit codes, origins) and the fp32 quantities
+that decide them (query vector, scores, scales, zero-points) must match bit for
+bit; attention outputs within max-abs 1e-2 * max|ref| and relative L2 5e-3.
+"""
+import numpy as np
+import pytest
+
+from paper_2601_01204_b200 import synth
+from xkv_testlib import run_stream, to_device_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def xkv():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_2601_01204_b200.xkv as m
+    return m
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_tiny_stream_4bit(xkv, impl):
+    """Config 1: 1 layer, 16 x 64, 261 tokens/frame, 8 frames, budget 1024, 4-bit."""
+    p = xkv.Params(budget=1024, max_frame_tokens=261, kv_bits=4)
+    cache, ora, worst = run_stream(xkv, p, 261, 8, seed=1, impl=impl)
+    info = cache.xkv_get_info()
+    assert info.T == 1024 and info.frames == 8 and info.last_evicted == 261
+    print("tiny 4-bit impl", impl, "worst (max-abs, rel-L2)", worst)
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_tiny_stream_16bit(xkv, impl):
+    p = xkv.Params(budget=1024, max_frame_tokens=261, kv_bits=16)
+    cache, ora, worst = run_stream(xkv, p, 261, 8, seed=2, impl=impl)
+    assert cache.xkv_get_info().T == 1024
+    print("tiny 16-bit impl", impl, "worst", worst)
+
+
+@pytest.mark.parametrize("bits", [4, 16])
+def test_token_major_layout(xkv, bits):
+    """[n][H*d] storage (tok_stride = H*d, head_stride = d)."""
+    p = xkv.Params(budget=600, max_frame_tokens=200, kv_bits=bits)
+    run_stream(xkv, p, 197, 5, seed=3, token_major=True)
+
+
+def test_budget_below_first_plus_current(xkv):
+    """k = max(0, L_max - T_first - n) = 0: the cache is first + current frame."""
+    p = xkv.Params(budget=300, max_frame_tokens=261, kv_bits=4)
+    cache, ora, _ = run_stream(xkv, p, 261, 4, seed=4)
+    assert cache.xkv_get_info().T == 522
+
+
+def test_ragged_frame_sizes_and_small_heads(xkv):
+    """Frame sizes that leave partial pooling groups and partial key groups; H = 3."""
+    p = xkv.Params(n_heads=3, budget=500, max_frame_tokens=150, kv_bits=4, pool_g=7, n_special=2)
+    run_stream(xkv, p, [129, 64, 150, 5, 77, 150, 33, 128], 8, seed=5)
+
+
+def test_single_token_frames_and_exact_budget(xkv):
+    p = xkv.Params(n_heads=2, budget=256, max_frame_tokens=128, kv_bits=4, n_special=1, pool_g=16)
+    run_stream(xkv, p, [128, 128, 1, 128, 64], 5, seed=6)
+
+
+def test_score_ties_are_broken_by_position(xkv):
+    """All-zero queries give all-equal scores (+0): the lowest positions must survive."""
+    import torch
+    p = xkv.Params(n_heads=2, budget=200, max_frame_tokens=64, kv_bits=4)
+    cache = xkv.Cache(p)
+    H, n, d = 2, 64, 64
+    for t in range(5):
+        _, kb, vb = synth.gen_frame(7, 0, t, H, n, d)
+        q = torch.zeros(H, n, d, dtype=torch.bfloat16, device="cuda")
+        cache.step(q, to_device_bf16(kb), to_device_bf16(vb))
+        info = cache.xkv_get_info()
+        if info.last_evicted:
+            kept = cache.xkv_debug_export(xkv.BUF_KEPT, info.last_kept * 4).view(np.int32)
+            assert np.array_equal(kept, np.arange(info.last_kept))
+    assert cache.xkv_get_info().T == 200
+
+
+def test_state_machine_and_argument_errors(xkv):
+    import torch
+    p = xkv.Params(budget=512, max_frame_tokens=100)
+    cache = xkv.Cache(p)
+    q = torch.zeros(16, 100, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(xkv.XkvError) as e:
+        cache.kv_quant_pack()
+    assert e.value.status == xkv.XKV_E_STATE
+    with pytest.raises(xkv.XkvError) as e:
+        cache.attn_packed_causal(q)
+    assert e.value.status == xkv.XKV_E_STATE
+    big = torch.zeros(16, 101, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(xkv.XkvError) as e:
+        cache.kv_append(big, big)
+    assert e.value.status == xkv.XKV_E_INVALID
+    cache.kv_append(q, q)
+    with pytest.raises(xkv.XkvError) as e:
+        cache.kv_append(q, q)
+    assert e.value.status == xkv.XKV_E_STATE
+    with pytest.raises(xkv.XkvError) as e:
+        cache.kv_score_evict(q[:, :50])
+    assert e.value.status == xkv.XKV_E_INVALID
+    cache.kv_score_evict(q)
+    cache.kv_quant_pack()
+    cache.attn_packed_causal(q)
+    assert cache.xkv_get_info().stage == 0
+    cache.xkv_reset()
+    assert cache.xkv_get_info().T == 0
+    # too-small workspace is refused before anything is launched
+    import ctypes as C
+    h = C.c_void_p()
+    rc = xkv.lib.xkv_create(C.byref(p.c()), cache.workspace.data_ptr(), 1024, 0, C.byref(h))
+    assert rc == xkv.XKV_E_NOMEM
+
+
+def test_synth_kernel_matches_numpy_generator(xkv):
+    import torch
+    H, n, d = 16, 261, 64
+    for tensor in (synth.TENSOR_Q, synth.TENSOR_K, synth.TENSOR_V):
+        dst = torch.empty(H, n, d, dtype=torch.bfloat16, device="cuda")
+        xkv.xkv_synth_fill(dst, 9, 2, 5, tensor)
+        got = dst.view(torch.int16).cpu().numpy().view(np.uint16)
+        assert np.array_equal(got, synth.gen_tensor_bits(9, 2, 5, tensor, H, n, d))

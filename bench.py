@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Stream frames/s of the 24-layer compressed-KV attention path on B200.
+
+One step = one frame (1374 tokens) through all 24 layers: append, score, evict,
+quantise/pack, attention over the packed cache, via xkv_stream_step.  Prints one
+JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl xkv|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+# Workload: the full stack (24 layers, 16 x 64, 1374 tokens/frame, budget 16384, 4-bit).
+WORKLOAD = dict(name="full_stack_24L_1374tok_budget16384_int4", layers=24, n_heads=16, head_dim=64,
+                n_tokens=1374, budget=16384, kv_bits=4, n_special=5, pool_g=16, quant_group=64, seed=3)
+METRIC = "stream frames/s (24-layer compressed-KV attention)"
+UNIT = "frames/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture
+# summarised under profiles/ (None until a capture of the current kernel exists).
+ATTN_DRAM_TRAFFIC_BYTES = None
+
+
+def _peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], tflops_burst=d["bf16_tflops"], tflops_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([f.strip() for f in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+
+    def summary(self) -> dict:
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def _oracle_layer_steps(w: dict, n_timed: int, n_warm: int):
+    """Streams ONE layer through the oracle to steady state, then times whole layer-steps."""
+    from oracle import xkv_oracle as xo
+    from paper_2601_01204_b200 import synth
+    p = xo.OracleParams(n_heads=w["n_heads"], head_dim=w["head_dim"], n_special=w["n_special"], pool_g=w["pool_g"],
+                        quant_group=w["quant_group"], kv_bits=w["kv_bits"], budget=w["budget"])
+    layer = xo.OracleLayer(p)
+    n = w["n_tokens"]
+    fill = -(-w["budget"] // n)                      # frames until the cache is full and evicting
+    times = []
+    for t in range(fill + n_warm + n_timed):
+        q, k, v = (synth.bf16_bits_to_f32(a) for a in synth.gen_frame(w["seed"], 0, t, w["n_heads"], n, w["head_dim"]))
+        t0 = time.perf_counter()
+        layer.append(k, v)
+        layer.score_evict(q)
+        layer.quant_pack()
+        if t >= fill:                                  # attention is skipped while filling (untimed)
+            layer.attend(q)
+        dt = time.perf_counter() - t0
+        if t >= fill + n_warm:
+            times.append(dt)
+    return times
+
+
+def _cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(w: dict, n_timed: int = 3, n_warm: int = 1) -> dict:
+    times = _oracle_layer_steps(w, n_timed, n_warm)
+    per_layer = float(np.mean(times))
+    return dict(value=1.0 / (per_layer * w["layers"]), unit=UNIT, cores=_cpu_threads(), kind="oracle",
+                sample=f"{n_timed} steady-state layer-steps of one layer (cache full at {w['budget']} tokens) timed in "
+                       f"full, x{w['layers']} layers extrapolated; {per_layer:.2f} s per layer-step")
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = WORKLOAD
+    # one "step" is a bounded sample of the frame: one of the 24 (identical-shape) layer-steps
+    steps, warm = max(1, min(args.steps, 12)), max(0, min(args.warmup, 2))
+    t_all = time.perf_counter()
+    times = _oracle_layer_steps(w, steps, warm)
+    per_layer = float(np.mean(times))
+    value = 1.0 / (per_layer * w["layers"])
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=per_layer * w["layers"] * 1e3, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f32/f64", data="synthetic",
+                config=dict(workload=w["name"], layers=w["layers"], tokens_per_frame=w["n_tokens"],
+                            budget=w["budget"], kv_bits=w["kv_bits"],
+                            sampled_steps=steps, note="each timed step is one oracle layer-step (1/24 of a frame) "
+                            "in steady state; frame time = 24 x mean"),
+                cpu_baseline=dict(value=value, unit=UNIT, kind="oracle", cores=_cpu_threads(),
+                                  sample=f"{steps} layer-steps, {time.perf_counter() - t_all:.0f} s total"),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- GPU arm
+def run_xkv(args) -> None:
+    import torch
+    import torch.distributed as dist
+    from paper_2601_01204_b200 import build, synth
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    import paper_2601_01204_b200.xkv as xkv
+
+    w = WORKLOAD
+    L, H, d, n = w["layers"], w["n_heads"], w["head_dim"], w["n_tokens"]
+    p = xkv.Params(n_heads=H, head_dim=d, n_special=w["n_special"], pool_g=w["pool_g"], quant_group=w["quant_group"],
+                   kv_bits=w["kv_bits"], budget=w["budget"], max_frame_tokens=n)
+    caches = [xkv.Cache(p, device=f"cuda:{local}") for _ in range(L)]
+    K, W = args.steps, args.warmup
+    fill = -(-w["budget"] // n)                     # 12 frames until every layer's cache is full
+    pool = min(fill + W + K, 40)                    # distinct resident frames, cycled afterwards
+    seed = w["seed"] + 1000 * rank                  # replicas stream different data
+    frames = []
+    for f in range(pool):
+        q = torch.empty(L, H, n, d, dtype=torch.bfloat16, device="cuda")
+        k = torch.empty_like(q)
+        v = torch.empty_like(q)
+        for l in range(L):
+            xkv.xkv_synth_fill(q[l], seed + l, l, f, synth.TENSOR_Q)
+            xkv.xkv_synth_fill(k[l], seed + l, l, f, synth.TENSOR_K)
+            xkv.xkv_synth_fill(v[l], seed + l, l, f, synth.TENSOR_V)
+        frames.append(tuple([x[l] for l in range(L)] for x in (q, k, v)))
+    out = torch.empty(L, H, n, d, dtype=torch.bfloat16, device="cuda")
+    outs = [out[l] for l in range(L)]
+
+    def step(t: int) -> None:
+        q, k, v = frames[t % pool]
+        xkv.xkv_stream_step(caches, q, k, v, outs)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    t = 0
+    for _ in range(fill + W):                       # untimed: fill to steady state, then W warm-up steps
+        step(t); t += 1
+    launches0 = sum(c.xkv_get_info().launches for c in caches)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(local) as clocks:
+        ev0.record()
+        for _ in range(K):
+            step(t); t += 1
+        ev1.record()
+        barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    launches = sum(c.xkv_get_info().launches for c in caches) - launches0
+    if world > 1:
+        tt = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    assert all(c.xkv_get_info().T == w["budget"] for c in caches)
+    assert all(c.xkv_poll_status() == 0 for c in caches)
+
+    # per-kernel device time over the same K steps, events on the launching stream
+    for c in caches:
+        c.xkv_profile_enable(True)
+    for _ in range(K):
+        step(t); t += 1
+    prof = {}
+    for c in caches:
+        for name, (ms, cnt) in c.xkv_profile_read().items():
+            a = prof.setdefault(name, [0.0, 0])
+            a[0] += ms; a[1] += cnt
+        c.xkv_profile_enable(False)
+
+    # end to end: host tensors in pinned memory, copies inside the timed region
+    Ke = max(1, min(K, 10))
+    host = []
+    for f in range(2):
+        q, k, v = frames[(t + f) % pool]
+        host.append(tuple([x[l].cpu().pin_memory() for l in range(L)] for x in (q, k, v)))
+    host_out = torch.empty(L, H, n, d, dtype=torch.bfloat16).pin_memory()
+    host_outs = [host_out[l] for l in range(L)]
+    staging = torch.empty(xkv.xkv_stream_step_host_bytes(p, n), dtype=torch.uint8, device="cuda")
+
+    def step_host(i: int) -> None:
+        q, k, v = host[i % 2]
+        xkv.xkv_stream_step_host(caches, q, k, v, host_outs, staging)
+
+    for i in range(3):
+        step_host(i)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(Ke):
+        step_host(i)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        tt = torch.tensor([e2e_s], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_s = float(tt.item())
+    frame_bytes = L * H * n * d * 2
+
+    if rank == 0:
+        peaks = _peaks()
+        ms_step = ms_total / K
+        attn_ms, attn_cnt = prof.get("attn", (0.0, 0))
+        flops = 4.0 * n * w["budget"] * d * H                     # useful FLOPs of one attention launch
+        attn_avg_s = (attn_ms / max(attn_cnt, 1)) * 1e-3
+        achieved = flops / attn_avg_s / 1e12 if attn_avg_s > 0 else 0.0
+        prof_total = sum(v[0] for v in prof.values())
+        line = dict(metric=METRIC, value=world * K / (ms_total * 1e-3), unit=UNIT, n_gpus=world, steps=K, warmup=W,
+                    ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f16",
+                    data="synthetic",
+                    config=dict(workload=w["name"], layers=L, heads=H, head_dim=d, tokens_per_frame=n,
+                                budget=w["budget"], kv_bits=w["kv_bits"], prefill_frames=fill, resident_frames=pool,
+                                l2="inputs exceed L2 (about 1.2 GB touched per step)", replicas=world),
+                    clocks=clocks.summary(),
+                    e2e=dict(value=world * Ke / e2e_s, unit=UNIT, h2d_bytes_per_step=3 * frame_bytes,
+                             d2h_bytes_per_step=frame_bytes, steps=Ke),
+                    gpu_launches=int(launches),
+                    roofline=dict(bound="tensor", kernel="attn_packed_causal", achieved=achieved,
+                                  peak=peaks["tflops_sustained"], unit="TFLOP/s",
+                                  frac=achieved / peaks["tflops_sustained"], peak_source=peaks["source"] + " (sustained)",
+                                  frac_of_burst=achieved / peaks["tflops_burst"], flops_per_launch=flops,
+                                  avg_launch_ms=attn_avg_s * 1e3, traffic=ATTN_DRAM_TRAFFIC_BYTES),
+                    kernels={k_: dict(ms_per_step=v_[0] / K, launches_per_step=v_[1] / K,
+                                      share=v_[0] / prof_total if prof_total else 0.0) for k_, v_ in prof.items()
+                             if v_[1]})
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(w)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="xkv", choices=["xkv", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_xkv(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -201,6 +201,22 @@ XKV_API int xkv_poll_status(const xkv_cache* cache, xkv_stream stream);
 
 XKV_API const char* xkv_strerror(int status);
 
+/* Optional per-kernel timing for benchmarks.  While enabled, every kernel the
+ * library launches for this cache is bracketed by a pair of CUDA events on the
+ * launching stream (a small overhead; leave it off in production).
+ * xkv_profile_read synchronises `stream`, adds the elapsed time of all launches
+ * recorded since the last read to the per-category totals, copies the totals to
+ * *out and clears them. */
+enum { XKV_PROF_APPEND = 0, XKV_PROF_POOL = 1, XKV_PROF_SCORE = 2, XKV_PROF_SELECT = 3,
+       XKV_PROF_REGROUP = 4, XKV_PROF_GATHER = 5, XKV_PROF_ATTN = 6, XKV_PROF_COMBINE = 7,
+       XKV_PROF_CATEGORIES = 8 };
+typedef struct {
+  double  ms[XKV_PROF_CATEGORIES];        /* summed device time per category, milliseconds */
+  int64_t launches[XKV_PROF_CATEGORIES];  /* launches per category                         */
+} xkv_profile;
+XKV_API int xkv_profile_enable(xkv_cache* cache, int enable);
+XKV_API int xkv_profile_read(xkv_cache* cache, xkv_profile* out, xkv_stream stream);
+
 /* ---- synthetic inputs (not part of the method) -------------------------------- */
 
 /* Fills dst (device, bf16 [n_heads][n_tokens][head_dim]) with the seeded

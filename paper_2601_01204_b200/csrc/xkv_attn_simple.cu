@@ -145,13 +145,13 @@ cudaError_t launch_attn_simple(xkv_cache* c, const void* q, void* out, int n, in
   const float scale_log2 = scale * 1.4426950408889634f;
   auto qq = reinterpret_cast<const __nv_bfloat16*>(q);
   auto oo = reinterpret_cast<__nv_bfloat16*>(out);
+  LaunchScope ls(c, XKV_PROF_ATTN, st);
   if (c->p.kv_bits == 16)
     attn_simple_kernel<16><<<grid, 128, 0, st>>>(qq, oo, n, ts, hs, c->buf[c->cur], c->cap, c->T_first,
                                                  c->rest_base, t_phys, scale_log2);
   else
     attn_simple_kernel<4><<<grid, 128, 0, st>>>(qq, oo, n, ts, hs, c->buf[c->cur], c->cap, c->T_first,
                                                 c->rest_base, t_phys, scale_log2);
-  c->launches++;
   return cudaGetLastError();
 }
 

@@ -126,8 +126,10 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
   c->attn_part = reinterpret_cast<float*>(c->ws + L.off_attn);
   c->attn_part_bytes = L.attn_bytes;
   reset_host_state(c);
+  c->prof = new (std::nothrow) Profiler;
+  if (!c->prof) { delete c; return XKV_E_NOMEM; }
   const int rc = zero_workspace(c, reinterpret_cast<cudaStream_t>(stream));
-  if (rc != XKV_OK) { delete c; return rc; }
+  if (rc != XKV_OK) { delete c->prof; delete c; return rc; }
   *out = c;
   return XKV_OK;
 }
@@ -140,6 +142,11 @@ int xkv_reset(xkv_cache* c, xkv_stream stream) {
 
 int xkv_destroy(xkv_cache* c) {
   if (!c) return XKV_E_INVALID;
+  if (c->prof) {
+    for (auto& e : c->prof->pending) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+    for (auto& e : c->prof->pool) cudaEventDestroy(e);
+    delete c->prof;
+  }
   delete c;
   return XKV_OK;
 }
@@ -343,6 +350,35 @@ int xkv_poll_status(const xkv_cache* c, xkv_stream stream) {
   int word = 0;
   if (cudaMemcpy(&word, c->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return XKV_E_CUDA;
   return word == 0 ? XKV_OK : XKV_E_TIMEOUT;
+}
+
+int xkv_profile_enable(xkv_cache* c, int enable) {
+  if (!c || !c->prof) return XKV_E_INVALID;
+  c->prof->on = enable != 0;
+  return XKV_OK;
+}
+
+int xkv_profile_read(xkv_cache* c, xkv_profile* out, xkv_stream stream) {
+  if (!c || !c->prof || !out) return XKV_E_INVALID;
+  if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
+  Profiler* p = c->prof;
+  for (auto& e : p->pending) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(e.b) != cudaSuccess || cudaEventElapsedTime(&ms, e.a, e.b) != cudaSuccess)
+      return XKV_E_CUDA;
+    p->ms[e.cat] += ms;
+    p->launches[e.cat] += 1;
+    p->pool.push_back(e.a);
+    p->pool.push_back(e.b);
+  }
+  p->pending.clear();
+  for (int i = 0; i < XKV_PROF_CATEGORIES; ++i) {
+    out->ms[i] = p->ms[i];
+    out->launches[i] = p->launches[i];
+    p->ms[i] = 0;
+    p->launches[i] = 0;
+  }
+  return XKV_OK;
 }
 
 const char* xkv_strerror(int status) {

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "xkv.h"
 
 namespace xkv {
@@ -22,6 +24,16 @@ struct BufSet {
   uint8_t* v;        // [H][cap][row_bytes]
   float2* vpar;      // [H][cap]          (scale, zero)
   int32_t* origin;   // [cap]
+};
+
+// Optional per-launch timing (xkv_profile_enable): one event pair per kernel launch.
+struct ProfEvent { int cat; cudaEvent_t a, b; };
+struct Profiler {
+  bool on = false;
+  std::vector<ProfEvent> pending;
+  std::vector<cudaEvent_t> pool;
+  double ms[XKV_PROF_CATEGORIES] = {0};
+  long long launches[XKV_PROF_CATEGORIES] = {0};
 };
 
 }  // namespace xkv
@@ -49,11 +61,31 @@ struct xkv_cache {
   int n_pending, kk_pending, rold_pending, evict_pending, first_pending;
   int last_evicted, last_kept, last_prunable;
   long long launches;
+  xkv::Profiler* prof;
 };
 
 namespace xkv {
 
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// Brackets one kernel launch with events when profiling is on; counts the launch.
+struct LaunchScope {
+  xkv_cache* c; int cat; cudaStream_t st; cudaEvent_t a = nullptr, b = nullptr;
+  LaunchScope(xkv_cache* c_, int cat_, cudaStream_t st_) : c(c_), cat(cat_), st(st_) {
+    c->launches++;
+    Profiler* p = c->prof;
+    if (p && p->on) {
+      auto get = [&]() { cudaEvent_t e = nullptr;
+        if (!p->pool.empty()) { e = p->pool.back(); p->pool.pop_back(); } else cudaEventCreate(&e);
+        return e; };
+      a = get(); b = get();
+      cudaEventRecord(a, st);
+    }
+  }
+  ~LaunchScope() {
+    if (a) { cudaEventRecord(b, st); c->prof->pending.push_back({cat, a, b}); }
+  }
+};
 
 // ---- launchers implemented in the kernel translation units -------------------
 // All return cudaError_t of the launch (cudaGetLastError) and count launches.

@@ -127,6 +127,7 @@ cudaError_t launch_append(xkv_cache* c, const void* k, const void* v, int n, int
   const BufSet d1 = c->buf[c->cur];
   auto kk = reinterpret_cast<const __nv_bfloat16*>(k);
   auto vv = reinterpret_cast<const __nv_bfloat16*>(v);
+  LaunchScope ls(c, XKV_PROF_APPEND, st);
   if (c->p.kv_bits == 16)
     append_kernel<16><<<blocks, 256, 0, st>>>(kk, vv, n, ts, hs, c->p.n_heads, c->cap,
                                               c->p.max_frame_tokens, dst_slot, c->frames + 1, d0, d1,
@@ -135,7 +136,6 @@ cudaError_t launch_append(xkv_cache* c, const void* k, const void* v, int n, int
     append_kernel<4><<<blocks, 256, 0, st>>>(kk, vv, n, ts, hs, c->p.n_heads, c->cap,
                                              c->p.max_frame_tokens, dst_slot, c->frames + 1, d0, d1,
                                              first, c->kstage);
-  c->launches++;
   return cudaGetLastError();
 }
 
@@ -195,10 +195,10 @@ cudaError_t launch_pool_q(xkv_cache* c, const void* q, int n, int64_t ts, int64_
   const int nsp = min(c->p.n_special, n);
   const int np = nsp + (n - nsp + c->p.pool_g - 1) / c->p.pool_g;
   const dim3 block(64, H < 16 ? H : 16);
+  LaunchScope ls(c, XKV_PROF_POOL, st);
   pool_q_kernel<<<np, block, (size_t)H * 64 * sizeof(float), st>>>(
       reinterpret_cast<const __nv_bfloat16*>(q), n, ts, hs, H, nsp, c->p.pool_g, np, c->qbar, c->qvec,
       c->counters);
-  c->launches++;
   return cudaGetLastError();
 }
 
@@ -261,13 +261,13 @@ score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* 
 cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st) {
   const int blocks = (r_old + 63) / 64;
   const size_t smem = (size_t)c->p.n_heads * 64 * sizeof(float2);
+  LaunchScope ls(c, XKV_PROF_SCORE, st);
   if (c->p.kv_bits == 16)
     score_kernel<16><<<blocks, 512, smem, st>>>(c->buf[c->cur], c->p.n_heads, c->cap, c->rest_base, r_old,
                                                 c->qvec, c->scores);
   else
     score_kernel<4><<<blocks, 512, smem, st>>>(c->buf[c->cur], c->p.n_heads, c->cap, c->rest_base, r_old,
                                                c->qvec, c->scores);
-  c->launches++;
   return cudaGetLastError();
 }
 
@@ -386,8 +386,8 @@ select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restri
 }
 
 cudaError_t launch_select(xkv_cache* c, int r_old, int k, cudaStream_t st) {
+  LaunchScope ls(c, XKV_PROF_SELECT, st);
   select_kernel<<<1, kSelThreads, 0, st>>>(c->scores, r_old, k, c->kept);
-  c->launches++;
   return cudaGetLastError();
 }
 
@@ -513,13 +513,17 @@ cudaError_t launch_pack(xkv_cache* c, int n, int kk, bool identity, bool first, 
     const int base = first ? 0 : c->rest_base;
     const int r_new = kk + n;
     const dim3 grid((r_new + 63) / 64, H);
-    regroup_k_kernel<<<grid, 512, 0, st>>>(src, dst, src, first, c->cap, c->p.max_frame_tokens, base, kk, r_new,
-                                           kept, c->kstage);
-    c->launches++;
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e;
+    {
+      LaunchScope ls(c, XKV_PROF_REGROUP, st);
+      regroup_k_kernel<<<grid, 512, 0, st>>>(src, dst, src, first, c->cap, c->p.max_frame_tokens, base, kk,
+                                             r_new, kept, c->kstage);
+      e = cudaGetLastError();
+    }
     if (e != cudaSuccess) return e;
   }
   if (kk > 0) {
+    LaunchScope ls(c, XKV_PROF_GATHER, st);
     if (c->p.kv_bits == 4) {
       const long long threads = (long long)H * kk * 2;
       gather_kernel<4><<<(int)((threads + 255) / 256), 256, 0, st>>>(src, dst, H, c->cap, c->rest_base, kk, kept);
@@ -527,7 +531,6 @@ cudaError_t launch_pack(xkv_cache* c, int n, int kk, bool identity, bool first, 
       const long long threads = (long long)H * kk * 8;
       gather_kernel<16><<<(int)((threads + 255) / 256), 256, 0, st>>>(src, dst, H, c->cap, c->rest_base, kk, kept);
     }
-    c->launches++;
   }
   return cudaGetLastError();
 }

@@ -30,8 +30,9 @@ EXPORTED = [
     "xkv_workspace_bytes", "xkv_create", "xkv_reset", "xkv_destroy", "kv_append", "kv_score_evict",
     "kv_quant_pack", "attn_packed_causal", "xkv_stream_step", "xkv_stream_step_host_bytes",
     "xkv_stream_step_host", "xkv_get_info", "xkv_debug_export", "xkv_poll_status", "xkv_strerror",
-    "xkv_synth_fill",
+    "xkv_synth_fill", "xkv_profile_enable", "xkv_profile_read",
 ]
+PROF_NAMES = ["append", "pool_q", "score", "select", "regroup_k", "gather", "attn", "attn_combine"]
 
 
 class xkv_params(C.Structure):
@@ -45,7 +46,15 @@ class xkv_info(C.Structure):
                [("launches", C.c_int64), ("workspace_bytes", C.c_uint64)]
 
 
+class xkv_profile(C.Structure):
+    _fields_ = [("ms", C.c_double * 8), ("launches", C.c_int64 * 8)]
+
+
 _vp, _i32, _i64, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+lib.xkv_profile_enable.restype = C.c_int
+lib.xkv_profile_enable.argtypes = [_vp, C.c_int]
+lib.xkv_profile_read.restype = C.c_int
+lib.xkv_profile_read.argtypes = [_vp, C.POINTER(xkv_profile), _vp]
 lib.xkv_workspace_bytes.restype = _sz
 lib.xkv_workspace_bytes.argtypes = [C.POINTER(xkv_params)]
 lib.xkv_create.restype = C.c_int
@@ -189,6 +198,14 @@ class Cache:
         info = xkv_info()
         _check(lib.xkv_get_info(self.handle, C.byref(info)), "xkv_get_info")
         return info
+
+    def xkv_profile_enable(self, on: bool) -> None:
+        _check(lib.xkv_profile_enable(self.handle, 1 if on else 0), "xkv_profile_enable")
+
+    def xkv_profile_read(self) -> dict:
+        pr = xkv_profile()
+        _check(lib.xkv_profile_read(self.handle, C.byref(pr), _stream()), "xkv_profile_read")
+        return {name: (pr.ms[i], pr.launches[i]) for i, name in enumerate(PROF_NAMES)}
 
     def xkv_poll_status(self) -> int:
         return int(lib.xkv_poll_status(self.handle, _stream()))

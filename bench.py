@@ -172,7 +172,10 @@ def run_xkv(args) -> None:
         dist.barrier()
     import paper_2601_01204_b200.xkv as xkv
 
-    w = WORKLOAD
+    w = dict(WORKLOAD)
+    if args.layers > 0:
+        w["layers"] = args.layers
+        w["name"] += f"_reduced_to_{args.layers}_layers"
     L, H, d, n = w["layers"], w["n_heads"], w["head_dim"], w["n_tokens"]
     p = xkv.Params(n_heads=H, head_dim=d, n_special=w["n_special"], pool_g=w["pool_g"], quant_group=w["quant_group"],
                    kv_bits=w["kv_bits"], budget=w["budget"], max_frame_tokens=n)
@@ -306,6 +309,8 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="xkv", choices=["xkv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling aid: run a reduced stack of the same workload (default: all 24 layers)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

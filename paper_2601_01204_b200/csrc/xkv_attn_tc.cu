@@ -91,6 +91,34 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// packed fp32 pairs (two floats in one 64-bit register)
+__device__ __forceinline__ uint64_t pack_f2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ float f2_lo(uint64_t v) { return __uint_as_float((uint32_t)v); }
+__device__ __forceinline__ float f2_hi(uint64_t v) { return __uint_as_float((uint32_t)(v >> 32)); }
+__device__ __forceinline__ uint64_t fma_f2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add_f2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul_f2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -185,29 +213,29 @@ __device__ __forceinline__ uint32_t h2_sub(uint32_t a, uint32_t b) {
   asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
   return r;
 }
-__device__ __forceinline__ uint32_t h2_fma(uint32_t a, uint32_t b, uint32_t c) {
+
+__device__ __forceinline__ uint32_t h2_mul(uint32_t a, uint32_t b) {
   uint32_t r;
-  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
   return r;
 }
 
-// Eight 4-bit codes of one packed word -> four fp16 pairs  s*q + c  (c = -z*s).
-// (w & 0x000F000F) | 0x6400 is the fp16 number 1024 + q; (w & 0x00F000F0) | 0x5400 is 64 + q.
-__device__ __forceinline__ uint4 dequant_word_h(uint32_t w, const uint32_t (&s2)[4], const uint32_t (&c2)[4]) {
+// Eight 4-bit codes of one packed word -> four fp16 pairs s * (q - z)  (Eq. 10).
+// (w & 0x000F000F) | 0x6400 is the fp16 number 1024 + q and (w & 0x00F000F0) | 0x5400 is 64 + q,
+// so one subtraction of (1024 + z) resp. (64 + z) gives q - z exactly (z is an integer), and one
+// multiplication by the fp16 scale follows.  zlo/zhi hold those two constants per channel pair:
+// pairs 0 and 2 of a word use the 1024 offset, pairs 1 and 3 the 64 offset.
+__device__ __forceinline__ uint4 dequant_word_h(uint32_t w, const uint32_t (&s2)[4], const uint32_t (&zo)[4]) {
   const uint32_t t = w >> 8;
-  uint32_t a0 = (w & 0x000F000Fu) | 0x64006400u;
-  uint32_t a1 = (w & 0x00F000F0u) | 0x54005400u;
-  uint32_t a2 = (t & 0x000F000Fu) | 0x64006400u;
-  uint32_t a3 = (t & 0x00F000F0u) | 0x54005400u;
-  a0 = h2_sub(a0, 0x64006400u);
-  a1 = h2_sub(a1, 0x54005400u);
-  a2 = h2_sub(a2, 0x64006400u);
-  a3 = h2_sub(a3, 0x54005400u);
+  const uint32_t a0 = (w & 0x000F000Fu) | 0x64006400u;
+  const uint32_t a1 = (w & 0x00F000F0u) | 0x54005400u;
+  const uint32_t a2 = (t & 0x000F000Fu) | 0x64006400u;
+  const uint32_t a3 = (t & 0x00F000F0u) | 0x54005400u;
   uint4 r;
-  r.x = h2_fma(a0, s2[0], c2[0]);
-  r.y = h2_fma(a1, s2[1], c2[1]);
-  r.z = h2_fma(a2, s2[2], c2[2]);
-  r.w = h2_fma(a3, s2[3], c2[3]);
+  r.x = h2_mul(h2_sub(a0, zo[0]), s2[0]);
+  r.y = h2_mul(h2_sub(a1, zo[1]), s2[1]);
+  r.z = h2_mul(h2_sub(a2, zo[2]), s2[2]);
+  r.w = h2_mul(h2_sub(a3, zo[3]), s2[3]);
   return r;
 }
 
@@ -287,7 +315,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_tc_kernel(const Args a) {
     // =========================== softmax warps ===============================
     const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
     float m_ref = -INFINITY;   // reference maximum (scaled, log2 units) used for the exponentials
-    float l = 0.f;
+    uint64_t l2 = 0ull;        // two partial row sums (packed fp32 pair)
     const int pad_tile = (a.t_first & 127) ? (a.t_first >> 7) : -1;
     for (int jj = 0; jj < nt; ++jj) {
       const int tile = tile_lo + jj;
@@ -300,15 +328,26 @@ __global__ void __launch_bounds__(kThreads, 2) attn_tc_kernel(const Args a) {
       tc_fence_after();
       // pass 1: row maximum
       float mx = -INFINITY;
+      if (lim >= 128) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t r[32];
-        XKV_TMEM_LD32(lane_addr + kColS + c0, r);
-        tc_wait_ld();
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t r[32];
+          XKV_TMEM_LD32(lane_addr + kColS + c0, r);
+          tc_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float x = (c0 + i < lim) ? __uint_as_float(r[i]) : -INFINITY;
-          mx = fmaxf(mx, x);
+          for (int i = 0; i < 32; i += 2) mx = max3(mx, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+        }
+      } else {
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t r[32];
+          XKV_TMEM_LD32(lane_addr + kColS + c0, r);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float x = (c0 + i < lim) ? __uint_as_float(r[i]) : -INFINITY;
+            mx = fmaxf(mx, x);
+          }
         }
       }
       mx *= a.scale_log2;
@@ -318,7 +357,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_tc_kernel(const Args a) {
       if (grow) {
         alpha = exp2f(m_ref - mx);      // 0 on the first tile (m_ref = -inf)
         m_ref = mx;
-        l *= alpha;
+        l2 = mul_f2(l2, pack_f2(alpha, alpha));
       }
       if (jj > 0) {
         // P(jj-1) has been consumed and O is quiescent once PV(jj-1) completed
@@ -339,28 +378,42 @@ __global__ void __launch_bounds__(kThreads, 2) attn_tc_kernel(const Args a) {
         }
       }
       // pass 2: exponentials, row sum, P -> TMEM (16-bit pairs)
+      const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2);
+      const uint64_t nm2 = pack_f2(-m_ref, -m_ref);
+      if (lim >= 128) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t r[32];
-        XKV_TMEM_LD32(lane_addr + kColS + c0, r);
-        tc_wait_ld();
-        uint32_t pk[16];
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t r[32];
+          XKV_TMEM_LD32(lane_addr + kColS + c0, r);
+          tc_wait_ld();
+          uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * i]), a.scale_log2, -m_ref));
-          float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), a.scale_log2, -m_ref));
-          if (c0 + 2 * i >= lim) p0 = 0.f;
-          if (c0 + 2 * i + 1 >= lim) p1 = 0.f;
-          pk[i] = kBf16 ? pack_bf2(p0, p1) : pack_h2(p0, p1);
-          // the row sum uses the rounded values that the MMA will see
-          if (kBf16) {
-            l += __uint_as_float(pk[i] << 16) + __uint_as_float(pk[i] & 0xFFFF0000u);
-          } else {
-            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&pk[i]));
-            l += f.x + f.y;
+          for (int i = 0; i < 16; ++i) {
+            const uint64_t x2 = fma_f2(pack_f2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, nm2);
+            const float p0 = fast_exp2(f2_lo(x2)), p1 = fast_exp2(f2_hi(x2));
+            l2 = add_f2(l2, pack_f2(p0, p1));
+            pk[i] = kBf16 ? pack_bf2(p0, p1) : pack_h2(p0, p1);
           }
+          XKV_TMEM_ST16(lane_addr + kColP + (c0 >> 1), pk);
         }
-        XKV_TMEM_ST16(lane_addr + kColP + (c0 >> 1), pk);
+      } else {
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t r[32];
+          XKV_TMEM_LD32(lane_addr + kColS + c0, r);
+          tc_wait_ld();
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * i]), a.scale_log2, -m_ref));
+            float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), a.scale_log2, -m_ref));
+            if (c0 + 2 * i >= lim) p0 = 0.f;
+            if (c0 + 2 * i + 1 >= lim) p1 = 0.f;
+            l2 = add_f2(l2, pack_f2(p0, p1));
+            pk[i] = kBf16 ? pack_bf2(p0, p1) : pack_h2(p0, p1);
+          }
+          XKV_TMEM_ST16(lane_addr + kColP + (c0 >> 1), pk);
+        }
       }
       tc_wait_st();
       tc_fence_before();
@@ -372,6 +425,7 @@ __global__ void __launch_bounds__(kThreads, 2) attn_tc_kernel(const Args a) {
     __syncwarp();
     tc_fence_after();
     const int row = q0 + tid;
+    const float l = f2_lo(l2) + f2_hi(l2);
     if (a.n_splits == 1) {
       const float inv_l = 1.f / l;
 #pragma unroll 1
@@ -430,16 +484,17 @@ __global__ void __launch_bounds__(kThreads, 2) attn_tc_kernel(const Args a) {
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
           const float2* par = a.kpar + ((size_t)h * (a.cap >> 6) + (tile * 2 + g)) * 64 + 8 * w;
-          uint32_t s2[4], c2[4];
+          uint32_t s2[4], zo[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const float2 p_a = __ldg(par + 2 * i), p_b = __ldg(par + 2 * i + 1);
+            const float off = (i & 1) ? 64.f : 1024.f;
             s2[i] = pack_h2(p_a.x, p_b.x);
-            c2[i] = pack_h2(-p_a.y * p_a.x, -p_b.y * p_b.x);
+            zo[i] = pack_h2(off + p_a.y, off + p_b.y);
           }
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const uint4 o = dequant_word_h(wd[4 * g + i], s2, c2);
+            const uint4 o = dequant_word_h(wd[4 * g + i], s2, zo);
             *reinterpret_cast<uint4*>(sgen + kOffK + b * 16384 + row_off + (4 * g + i) * 2048) = o;
           }
         }
@@ -465,9 +520,10 @@ __global__ void __launch_bounds__(kThreads, 2) attn_tc_kernel(const Args a) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const uint32_t s1 = pack_h2(vp[i].x, vp[i].x);
-          const uint32_t c1 = pack_h2(-vp[i].y * vp[i].x, -vp[i].y * vp[i].x);
-          const uint32_t s2[4] = {s1, s1, s1, s1}, c2[4] = {c1, c1, c1, c1};
-          const uint4 o = dequant_word_h(wd[i], s2, c2);
+          const uint32_t z_lo = pack_h2(1024.f + vp[i].y, 1024.f + vp[i].y);
+          const uint32_t z_hi = pack_h2(64.f + vp[i].y, 64.f + vp[i].y);
+          const uint32_t s2[4] = {s1, s1, s1, s1}, zo[4] = {z_lo, z_hi, z_lo, z_hi};
+          const uint4 o = dequant_word_h(wd[i], s2, zo);
           *reinterpret_cast<uint4*>(sgen + kOffV + b * 16384 + row_off + i * 2048) = o;
         }
       } else {

@@ -403,6 +403,7 @@ regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int cap, int max
                  int r_new, const int32_t* __restrict__ kept, const __nv_bfloat16* __restrict__ kstage) {
   __shared__ float s_mn[16][64];
   __shared__ float s_mx[16][64];
+  __shared__ float2 s_iz[64];
   const int tid = threadIdx.x;
   const int w = tid & 7;
   const int tok = tid >> 3;
@@ -457,19 +458,23 @@ regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int cap, int max
     for (int j = 0; j < 8; ++j) { s_mn[warp][8 * w + j] = mn[j]; s_mx[warp][8 * w + j] = mx[j]; }
   }
   __syncthreads();
+  // one thread per channel finishes the reduction and derives the group's parameters
+  if (tid < 64) {
+    float a = s_mn[0][tid], b = s_mx[0][tid];
+#pragma unroll
+    for (int r = 1; r < 16; ++r) { a = fminf(a, s_mn[r][tid]); b = fmaxf(b, s_mx[r][tid]); }
+    float sc, inv, z;
+    quant_params(a, b, sc, inv, z);
+    s_iz[tid] = make_float2(inv, z);
+    dst.kpar[dgrp + tid] = make_float2(sc, z);
+    if (two) dst2.kpar[dgrp + tid] = make_float2(sc, z);
+  }
+  __syncthreads();
   uint32_t c[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    float a = s_mn[0][8 * w + j], b = s_mx[0][8 * w + j];
-#pragma unroll
-    for (int r = 1; r < 16; ++r) { a = fminf(a, s_mn[r][8 * w + j]); b = fmaxf(b, s_mx[r][8 * w + j]); }
-    float s, inv, z;
-    quant_params(a, b, s, inv, z);
-    c[j] = valid ? quant_code(x[j], inv, z) : 0u;
-    if (tok == 0) {
-      dst.kpar[dgrp + 8 * w + j] = make_float2(s, z);
-      if (two) dst2.kpar[dgrp + 8 * w + j] = make_float2(s, z);
-    }
+    const float2 iz = s_iz[8 * w + j];
+    c[j] = valid ? quant_code(x[j], iz.x, iz.y) : 0u;
   }
   if (valid) {
     const uint32_t word = pack8(c);

@@ -27,8 +27,9 @@ def test_exports_match_header(xkv, repo_root):
 def test_workspace_bytes_and_param_validation(xkv):
     p = xkv.Params(budget=16384, max_frame_tokens=1374)
     nbytes = xkv.xkv_workspace_bytes(p)
-    # two buffer sets of 4-bit K and V codes plus parameters: tens of MiB, far below bf16 storage
-    assert 30 * 2 ** 20 < nbytes < 64 * 2 ** 20
+    # two buffer sets of 4-bit K and V codes plus parameters (about 46 MiB) and the split-KV
+    # partials of the attention kernel (about 34 MiB)
+    assert 30 * 2 ** 20 < nbytes < 96 * 2 ** 20
     assert xkv.xkv_workspace_bytes(xkv.Params(head_dim=128)) == 0
     assert xkv.xkv_workspace_bytes(xkv.Params(kv_bits=3)) == 0
     assert xkv.xkv_workspace_bytes(xkv.Params(budget=0)) == 0

@@ -55,7 +55,8 @@ typedef enum {
   XKV_E_NOMEM       = -3,   /* workspace too small / host allocation failed            */
   XKV_E_UNSUPPORTED = -4,   /* parameter combination not implemented                   */
   XKV_E_CUDA        = -5,   /* a CUDA runtime/driver call failed                       */
-  XKV_E_TIMEOUT     = -6    /* a bounded device-side wait ran out (see xkv_poll_status)*/
+  XKV_E_TIMEOUT     = -6,   /* a bounded device-side wait ran out (see xkv_poll_status)*/
+  XKV_E_LIMIT       = -7    /* the call needs more than a fixed built-in limit allows   */
 } xkv_status;
 
 /* Method parameters.  Defaults of the paper: n_special = 5 (1 camera + 4
@@ -164,6 +165,45 @@ XKV_API int kv_quant_pack(xkv_cache* cache, xkv_stream stream);
 XKV_API int attn_packed_causal(xkv_cache* cache, const void* q, void* out, int32_t n,
                        int64_t tok_stride, int64_t head_stride, float softmax_scale,
                        int32_t impl, xkv_stream stream);
+
+/* attn_packed_causal for callers that must not allocate device memory.
+ * (The paper has no counterpart: this is a deployment variant of Step 5 with the
+ * same arithmetic and the same kernel.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a host
+ * application that forbids allocation after start-up, a plug-in whose host owns
+ * the allocator, a process that shares its GPU with a job whose memory pool must
+ * not be disturbed - and that therefore cannot grow a buffer for the attention
+ * kernel's scratch.  The tensor-core kernel splits the keys of one head over
+ * several thread blocks and needs global memory for the partial results (64
+ * accumulators plus running max and sum per split, head and query).
+ * attn_packed_causal keeps them in the cache workspace; this variant keeps them
+ * in a fixed array of XKV_STATIC_SCRATCH_BYTES that is part of the library image
+ * and leaves that region of the workspace untouched.  Every GPU on which the
+ * library is used holds the array from first use until the process exits.  The
+ * call allocates nothing, neither on the device nor through any allocating
+ * routine.
+ *
+ * Rules of use
+ *   - Same arguments, state requirements and result as attn_packed_causal with
+ *     impl = 0; q and out are still the caller's.
+ *   - A launch whose partials need more than XKV_STATIC_SCRATCH_BYTES is refused
+ *     with XKV_E_LIMIT before anything is enqueued; the cache stays in the packed
+ *     state, so attn_packed_causal can still take the frame.  The need is
+ *     splits * n_heads * n * 264 bytes, splits <= 6 chosen from the grid size;
+ *     a single split (short caches) needs none.
+ *   - The first call on a device looks up the array's device address (once per
+ *     device, with that device current).  Make that first call outside any
+ *     stream capture.
+ *   - All callers in the process share the one array per GPU, and it keeps
+ *     whatever the last call left there.  Nothing in it has to start at zero:
+ *     every partial that is read was written by the same call.  Two calls whose
+ *     kernels can overlap on one GPU (different streams or threads) race on it:
+ *     serialise them. */
+#define XKV_STATIC_SCRATCH_BYTES (32u << 20)
+XKV_API int attn_packed_causal_static(xkv_cache* cache, const void* q, void* out, int32_t n,
+                              int64_t tok_stride, int64_t head_stride, float softmax_scale,
+                              xkv_stream stream);
 
 /* One frame through a stack of layers: for each layer in order, the four calls
  * above with softmax_scale = 1/sqrt(head_dim).  q, k, v, out are HOST arrays of

@@ -19,12 +19,15 @@
 // Every mbarrier wait is bounded: when the bound is hit the thread records
 // XKV_E_TIMEOUT in the cache's status word and carries on, so the kernel always
 // terminates and frees its tensor memory.
+#include <mutex>
+
 #include "xkv_internal.cuh"
 
 namespace xkv {
 
 namespace {
 
+constexpr int kMaxDevices = 64;
 constexpr int kThreads = 288;
 constexpr int kQRows = 128;
 constexpr int kMaxSplits = 6;
@@ -633,8 +636,12 @@ static int choose_splits(int items, int n_tiles, int slots) {
   return best;
 }
 
-cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs, float scale,
-                           cudaStream_t st) {
+// `part` holds the split-KV partials: accumulators float [rows_cap][64], then (max, sum) float2
+// [rows_cap].  rows_cap = 0 means "as many rows as this launch needs" and `part_bytes` is then the
+// room available: when it does not suffice nothing is launched and cudaErrorMemoryAllocation returns.
+static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
+                                     float scale, float* part, size_t rows_cap, size_t part_bytes,
+                                     cudaStream_t st) {
   static int sm_count = 0;
   static bool attr_set = false;
   if (!attr_set) {
@@ -664,9 +671,13 @@ cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_
   const int H = c->p.n_heads;
   a.n_splits = choose_splits(q_tiles * H, a.n_tiles, sm_count * 2);
   a.tiles_per_split = (a.n_tiles + a.n_splits - 1) / a.n_splits;
-  const size_t rows = (size_t)kMaxSplits * H * c->p.max_frame_tokens;
-  a.part_o = c->attn_part;
-  a.part_ml = reinterpret_cast<float2*>(c->attn_part + rows * 64);
+  size_t rows = rows_cap;
+  if (rows == 0) {
+    rows = (size_t)a.n_splits * H * n;
+    if (a.n_splits > 1 && rows * (64 * sizeof(float) + sizeof(float2)) > part_bytes) return cudaErrorMemoryAllocation;
+  }
+  a.part_o = part;
+  a.part_ml = reinterpret_cast<float2*>(part + rows * 64);
   a.status = c->status;
   const dim3 grid(q_tiles, H, a.n_splits);
   {
@@ -682,6 +693,45 @@ cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_
     attn_combine_kernel<<<(int)((threads + 255) / 256), 256, 0, st>>>(a.part_o, a.part_ml, a.n_splits, H, n, a.out, ts, hs);
   }
   return cudaGetLastError();
+}
+
+cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs, float scale,
+                           cudaStream_t st) {
+  return launch_attn_tc_on(c, q, out, n, ts, hs, scale, c->attn_part,
+                           (size_t)kMaxSplits * c->p.n_heads * c->p.max_frame_tokens, c->attn_part_bytes, st);
+}
+
+// ---------------------------------------------------------------------------
+// attn_packed_causal_static: the same attention with its split-KV partials in a
+// fixed array that is part of the loaded library image instead of the caller's
+// workspace.  See xkv.h for who needs this and for the rules of use.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_partials[XKV_STATIC_SCRATCH_BYTES];
+
+// In host code `g_static_partials` only names the symbol; the device address has to be asked
+// for, once per device, while that device is current.
+static std::mutex g_static_mutex;
+static void* g_static_addr[kMaxDevices] = {nullptr};
+
+cudaError_t launch_attn_tc_static(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
+                                  float scale, cudaStream_t st) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  void* addr = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_addr[dev]) {
+      void* p = nullptr;
+      e = cudaGetSymbolAddress(&p, g_static_partials);
+      if (e != cudaSuccess) return e;
+      g_static_addr[dev] = p;
+    }
+    addr = g_static_addr[dev];
+  }
+  return launch_attn_tc_on(c, q, out, n, ts, hs, scale, reinterpret_cast<float*>(addr), 0,
+                           (size_t)XKV_STATIC_SCRATCH_BYTES, st);
 }
 
 }  // namespace xkv

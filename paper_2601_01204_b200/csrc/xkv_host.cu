@@ -239,6 +239,21 @@ int attn_packed_causal(xkv_cache* c, const void* q, void* out, int32_t n, int64_
   return XKV_OK;
 }
 
+int attn_packed_causal_static(xkv_cache* c, const void* q, void* out, int32_t n, int64_t ts, int64_t hs,
+                              float softmax_scale, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  if (c->stage != 3) return XKV_E_STATE;
+  if (n < 1 || n > c->p.max_frame_tokens || !aligned16(q) || !aligned16(out) || !strides_ok(ts, hs) ||
+      !(softmax_scale > 0.f))
+    return XKV_E_INVALID;
+  const cudaError_t e = launch_attn_tc_static(c, q, out, n, ts, hs, softmax_scale, reinterpret_cast<cudaStream_t>(stream));
+  if (e == cudaErrorMemoryAllocation) return XKV_E_LIMIT;
+  if (e == cudaErrorNotSupported) return XKV_E_UNSUPPORTED;
+  if (e != cudaSuccess) return XKV_E_CUDA;
+  c->stage = 0;
+  return XKV_OK;
+}
+
 int xkv_stream_step(xkv_cache* const* layers, int32_t n_layers, const void* const* q, const void* const* k,
                     const void* const* v, void* const* out, int32_t n, int64_t ts, int64_t hs,
                     xkv_stream stream) {
@@ -390,6 +405,7 @@ const char* xkv_strerror(int status) {
     case XKV_E_UNSUPPORTED: return "parameter combination not supported";
     case XKV_E_CUDA: return "CUDA call failed";
     case XKV_E_TIMEOUT: return "bounded device-side wait ran out";
+    case XKV_E_LIMIT: return "request exceeds a fixed built-in limit (static scratch size)";
     default: return "unknown status";
   }
 }

@@ -101,6 +101,10 @@ cudaError_t launch_attn_simple(xkv_cache* c, const void* q, void* out, int n, in
 // Returns cudaErrorNotSupported when the tensor-core kernel cannot take the call.
 cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
                            float scale, cudaStream_t st);
+// Same kernel, split-KV partials in the library's fixed device array; cudaErrorMemoryAllocation
+// when the launch would need more than XKV_STATIC_SCRATCH_BYTES.
+cudaError_t launch_attn_tc_static(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
+                                  float scale, cudaStream_t st);
 size_t attn_tc_scratch_bytes(const xkv_params* p);
 
 }  // namespace xkv

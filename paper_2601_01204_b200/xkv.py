@@ -24,13 +24,15 @@ if not os.path.exists(LIB_PATH):
 lib = C.CDLL(LIB_PATH)
 
 XKV_OK, XKV_E_INVALID, XKV_E_STATE, XKV_E_NOMEM, XKV_E_UNSUPPORTED, XKV_E_CUDA, XKV_E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
+XKV_E_LIMIT = -7
+STATIC_SCRATCH_BYTES = 32 << 20
 BUF_K_CODES, BUF_K_PARAMS, BUF_V_CODES, BUF_V_PARAMS, BUF_ORIGIN, BUF_SCORES, BUF_KEPT, BUF_QVEC = range(8)
 
 EXPORTED = [
     "xkv_workspace_bytes", "xkv_create", "xkv_reset", "xkv_destroy", "kv_append", "kv_score_evict",
     "kv_quant_pack", "attn_packed_causal", "xkv_stream_step", "xkv_stream_step_host_bytes",
     "xkv_stream_step_host", "xkv_get_info", "xkv_debug_export", "xkv_poll_status", "xkv_strerror",
-    "xkv_synth_fill", "xkv_profile_enable", "xkv_profile_read",
+    "xkv_synth_fill", "xkv_profile_enable", "xkv_profile_read", "attn_packed_causal_static",
 ]
 PROF_NAMES = ["append", "pool_q", "score", "select", "regroup_k", "gather", "attn", "attn_combine"]
 
@@ -71,6 +73,8 @@ lib.kv_quant_pack.restype = C.c_int
 lib.kv_quant_pack.argtypes = [_vp, _vp]
 lib.attn_packed_causal.restype = C.c_int
 lib.attn_packed_causal.argtypes = [_vp, _vp, _vp, _i32, _i64, _i64, C.c_float, _i32, _vp]
+lib.attn_packed_causal_static.restype = C.c_int
+lib.attn_packed_causal_static.argtypes = [_vp, _vp, _vp, _i32, _i64, _i64, C.c_float, _vp]
 lib.xkv_stream_step.restype = C.c_int
 lib.xkv_stream_step.argtypes = [C.POINTER(_vp), _i32, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp),
                                 C.POINTER(_vp), _i32, _i64, _i64, _vp]
@@ -186,6 +190,21 @@ class Cache:
             scale = 1.0 / float(np.sqrt(self.p.head_dim))
         _check(lib.attn_packed_causal(self.handle, q.data_ptr(), out.data_ptr(), q.shape[1], ts, hs,
                                       C.c_float(scale), impl, _stream()), "attn_packed_causal")
+        return out
+
+    def attn_packed_causal_static(self, q, out=None, scale: float | None = None):
+        """attn_packed_causal with the split-KV partials in the library's fixed device array
+        (for callers that may not allocate; XKV_E_LIMIT when the launch needs more than
+        STATIC_SCRATCH_BYTES)."""
+        import torch
+        if out is None:
+            out = torch.empty_like(q)
+        ts, hs = _strides(q)
+        assert _strides(out) == (ts, hs)
+        if scale is None:
+            scale = 1.0 / float(np.sqrt(self.p.head_dim))
+        _check(lib.attn_packed_causal_static(self.handle, q.data_ptr(), out.data_ptr(), q.shape[1], ts, hs,
+                                             C.c_float(scale), _stream()), "attn_packed_causal_static")
         return out
 
     def step(self, q, k, v, out=None, impl: int = 0):

@@ -126,6 +126,12 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
   c->attn_part = reinterpret_cast<float*>(c->ws + L.off_attn);
   c->attn_part_bytes = L.attn_bytes;
   reset_host_state(c);
+  {
+    // test hook: the maintenance kernels have conversion-free fast forms of Eq. 7 and Eq. 10 with a
+    // plain fallback; XKV_FORCE_PLAIN=1 makes every kernel of this cache take the fallback
+    const char* fp = getenv("XKV_FORCE_PLAIN");
+    c->force_plain = (fp && fp[0] == '1') ? 1 : 0;
+  }
   c->prof = new (std::nothrow) Profiler;
   if (!c->prof) { delete c; return XKV_E_NOMEM; }
   const int rc = zero_workspace(c, reinterpret_cast<cudaStream_t>(stream));

@@ -61,6 +61,7 @@ struct xkv_cache {
   int n_pending, kk_pending, rold_pending, evict_pending, first_pending;
   int last_evicted, last_kept, last_prunable;
   long long launches;
+  int force_plain;         // 1: kernels take the plain (conversion-based) arithmetic forms everywhere
   xkv::Profiler* prof;
 };
 

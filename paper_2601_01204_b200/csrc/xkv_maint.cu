@@ -140,17 +140,70 @@ cudaError_t launch_append(xkv_cache* c, const void* k, const void* v, int n, int
 }
 
 // ---------------------------------------------------------------------------
+// Conversion-free forms of Eq. 10 and Eq. 7.  They produce the same fp32 results
+// as dequant8 / quant_code whenever their preconditions hold (callers check them
+// and take the plain forms otherwise), but use no int<->float conversion or
+// round instruction, which issue at a quarter of the fp32 rate.
+//
+// A 4-bit code q sitting at bit 4i of a word, OR-ed into the mantissa of
+// 2^(23-4i), is the float 2^(23-4i) + q.  Subtracting 2^(23-4i) + z (exact for
+// integer |z| < 2^22) gives q - z exactly, like float(q) - z.
+// ---------------------------------------------------------------------------
+constexpr float kZLimit = 4194304.f;     // 2^22
+constexpr float kRoundMagic = 12582912.f;  // 1.5 * 2^23: y + magic has rint(y) in its mantissa for |y| < 2^22
+
+__device__ __forceinline__ uint32_t magic_bits(int j) { return 0x4B000000u - (uint32_t)(j >> 1) * 0x02000000u; }
+__device__ __forceinline__ float magic_val(int j) { return __uint_as_float(magic_bits(j)); }
+
+// par[j] = (s, magic_val(j) + z) for the 8 channels of the word.
+__device__ __forceinline__ void dequant8_magic(uint32_t word, const float2 (&par)[8], float (&x)[8]) {
+  const uint32_t hi = word >> 16;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t src = (j & 1) ? hi : word;
+    const uint32_t bits = (src & (0xFu << (4 * (j >> 1)))) | magic_bits(j);
+    x[j] = __fmul_rn(par[j].x, __fsub_rn(__uint_as_float(bits), par[j].y));
+  }
+}
+
+// clamp(rint(x * inv) + z, 0, 15) for |x * inv| < 2^21 and integer |z| < 2^22; zadj = int(z) - bits(magic).
+__device__ __forceinline__ uint32_t quant_code_magic(float x, float inv, int zadj) {
+  const float t = __fadd_rn(__fmul_rn(x, inv), kRoundMagic);
+  const int q = (int)__float_as_uint(t) + zadj;
+  int r;
+  asm("min.relu.s32 %0, %1, 15;" : "=r"(r) : "r"(q));   // max(min(q, 15), 0)
+  return (uint32_t)r;
+}
+
+// The plain forms as real calls on scalars, so that the rarely taken fallback costs a branch and
+// not predicated copies of its instructions in the hot path, and arrays stay in registers.
+__device__ __noinline__ float dequant_one_call(uint32_t q, float s, float z) {
+  return __fmul_rn(s, __fsub_rn((float)q, z));
+}
+__device__ __noinline__ uint32_t quant_code_call(float x, float inv, float z) { return quant_code(x, inv, z); }
+
+__device__ __forceinline__ void dequant8_plain(uint32_t word, const float2* par, float (&x)[8]) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) x[j] = dequant_one_call((word >> nib_shift(j)) & 0xFu, par[j].x, par[j].y);
+}
+
+// ---------------------------------------------------------------------------
 // Pooled query, Eq. 2-3, then the row mean that Eq. 5-6 reduce to.
 // One CTA per pooled row i; thread (c, hs) builds pooled[h][i][c] for heads
 // h = hs, hs+16, ... (sequential sum over the group's tokens, divided by the
 // group size); threads with hs == 0 add the heads in order and scale by 1/H.
 // The last CTA to finish adds the rows in order and divides by N_pooled.
+// Loads are issued in batches ahead of the (ordered) additions.
 // ---------------------------------------------------------------------------
+constexpr int kPoolRows = 128;   // pooled rows staged in shared memory at a time by the last CTA
+
 __global__ void __launch_bounds__(1024)
 pool_q_kernel(const __nv_bfloat16* __restrict__ q, int n, int64_t ts, int64_t hs, int H, int n_special,
               int g, int n_pooled, float* __restrict__ qbar, float* __restrict__ qvec,
               unsigned int* __restrict__ counter) {
   extern __shared__ float s_pooled[];  // [H][64]
+  __shared__ float s_rows[kPoolRows * 64];
+  __shared__ float s_acc[64];
   __shared__ bool s_last;
   const int i = blockIdx.x;
   const int c = threadIdx.x;   // 0..63
@@ -160,8 +213,15 @@ pool_q_kernel(const __nv_bfloat16* __restrict__ q, int n, int64_t ts, int64_t hs
   else { a = n_special + (i - n_special) * g; b = min(a + g, n); }
   for (int h = hslot; h < H; h += blockDim.y) {
     const __nv_bfloat16* base = q + (int64_t)h * hs + c;
-    float acc = __bfloat162float(base[(int64_t)a * ts]);
-    for (int t = a + 1; t < b; ++t) acc = __fadd_rn(acc, __bfloat162float(base[(int64_t)t * ts]));
+    float acc = 0.f;
+    for (int t0 = a; t0 < b; t0 += 16) {
+      float x[16];
+#pragma unroll
+      for (int u = 0; u < 16; ++u) x[u] = (t0 + u < b) ? __bfloat162float(base[(int64_t)(t0 + u) * ts]) : 0.f;
+#pragma unroll
+      for (int u = 0; u < 16; ++u)
+        if (t0 + u < b) acc = (t0 + u == a) ? x[u] : __fadd_rn(acc, x[u]);
+    }
     if (i >= n_special) acc = __fdiv_rn(acc, (float)(b - a));
     s_pooled[h * 64 + c] = acc;
   }
@@ -181,11 +241,20 @@ pool_q_kernel(const __nv_bfloat16* __restrict__ q, int n, int64_t ts, int64_t hs
   __syncthreads();
   if (s_last) {
     __threadfence();
-    if (hslot == 0) {
-      float acc = __ldcg(&qbar[c]);
-      for (int r = 1; r < n_pooled; ++r) acc = __fadd_rn(acc, __ldcg(&qbar[r * 64 + c]));
-      qvec[c] = __fdiv_rn(acc, (float)n_pooled);
+    // all threads fetch the rows (one round trip), then one thread per channel adds them in order
+    const int tid = threadIdx.y * 64 + threadIdx.x, nthr = blockDim.y * 64;
+    for (int r0 = 0; r0 < n_pooled; r0 += kPoolRows) {
+      const int rows = min(kPoolRows, n_pooled - r0);
+      __syncthreads();
+      for (int e = tid; e < rows * 64; e += nthr) s_rows[e] = __ldcg(&qbar[r0 * 64 + e]);
+      __syncthreads();
+      if (hslot == 0) {
+        float acc = (r0 == 0) ? s_rows[c] : s_acc[c];
+        for (int r = (r0 == 0) ? 1 : 0; r < rows; ++r) acc = __fadd_rn(acc, s_rows[r * 64 + c]);
+        s_acc[c] = acc;
+      }
     }
+    if (hslot == 0) qvec[c] = __fdiv_rn(s_acc[c], (float)n_pooled);
     if (threadIdx.x == 0 && threadIdx.y == 0) *counter = 0u;  // re-arm for the next launch
   }
 }
@@ -209,12 +278,16 @@ cudaError_t launch_pool_q(xkv_cache* c, const void* q, int n, int64_t ts, int64_
 // word of every head in order (Eq. 10), accumulate the head sum sequentially,
 // scale by 1/H (Eq. 4), multiply by the query vector, and add the 64 products
 // with a balanced tree: three levels inside the lane, three by xor-shuffle.
+// The words of four heads are fetched ahead of their (ordered) use.
 // ---------------------------------------------------------------------------
 template <int BITS>
 __global__ void __launch_bounds__(512)
 score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* __restrict__ qvec,
-             float* __restrict__ scores) {
-  extern __shared__ float2 s_par[];  // [H][64]
+             float* __restrict__ scores, int force_plain) {
+  // Parameters of the CTA's key group.  Fast path: float4 [H][4][8] = (s, magic + z) of channels
+  // 8w + 2v and 8w + 2v + 1 at [h][v][w], so that the eight lanes of a quarter-warp read
+  // consecutive 16-byte chunks.  Plain path: float2 (s, z) [H][64].
+  extern __shared__ __align__(16) float2 s_par[];
   __shared__ float s_w[64];
   const int tid = threadIdx.x;
   const int w = tid & 7;
@@ -222,27 +295,87 @@ score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* 
   const int i = blockIdx.x * 64 + tok;          // rest-local index
   const int slot = rest_base + i;
   const int grp = (rest_base >> 6) + blockIdx.x;
+  bool plain = false;
   if (BITS == 4) {
-    for (int e = tid; e < H * 64; e += 512)
-      s_par[e] = cur.kpar[((size_t)(e >> 6) * (cap >> 6) + grp) * 64 + (e & 63)];
+    int big = force_plain;
+    float2 mine[4];                              // H <= 64: at most 8 elements per thread, 4 at a time
+    for (int e0 = 0; e0 < H * 64; e0 += 2048) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int e = e0 + u * 512 + tid;
+        mine[u] = make_float2(0.f, 0.f);
+        if (e < H * 64) mine[u] = cur.kpar[((size_t)(e >> 6) * (cap >> 6) + grp) * 64 + (e & 63)];
+        big |= !(fabsf(mine[u].y) < kZLimit);
+      }
+      // the layout depends on the path, which the whole CTA has to agree on: H * 64 <= 2048 makes
+      // this loop run once for H <= 32; for more heads the parameters are re-read below
+      if (e0 == 0 && H * 64 <= 2048) break;
+    }
+    plain = __syncthreads_or(big) != 0;
+    for (int e0 = 0; e0 < H * 64; e0 += 2048) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int e = e0 + u * 512 + tid;
+        if (e < H * 64) {
+          float2 sz = mine[u];
+          if (H * 64 > 2048) sz = cur.kpar[((size_t)(e >> 6) * (cap >> 6) + grp) * 64 + (e & 63)];
+          if (plain) {
+            s_par[e] = sz;
+          } else {
+            const int h = e >> 6, ch = e & 63;
+            sz.y = __fadd_rn(magic_val(ch & 7), sz.y);
+            // [h][v = (ch & 7) >> 1][w = ch >> 3], two float2 per float4
+            s_par[((h * 4 + ((ch & 7) >> 1)) * 8 + (ch >> 3)) * 2 + (ch & 1)] = sz;
+          }
+        }
+      }
+    }
   }
   if (tid < 64) s_w[tid] = qvec[tid];
   __syncthreads();
   const bool valid = i < r_old;
   float acc[8];
-  for (int h = 0; h < H; ++h) {
-    float x[8];
-    if (BITS == 4) {
-      const uint32_t word =
-          valid ? *reinterpret_cast<const uint32_t*>(cur.k + ((size_t)h * cap + slot) * 32 + 4 * w) : 0u;
-      dequant8(word, s_par + h * 64 + 8 * w, x);
-    } else {
-      uint4 u = make_uint4(0, 0, 0, 0);
-      if (valid) u = *reinterpret_cast<const uint4*>(cur.k + ((size_t)h * cap + slot) * 128 + 16 * w);
-      bf16x8_to_float(u, x);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+  for (int h0 = 0; h0 < H; h0 += 4) {
+    uint32_t word[4];
+    uint4 wide[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int h = h0 + u;
+      word[u] = 0u;
+      wide[u] = make_uint4(0, 0, 0, 0);
+      if (valid && h < H) {
+        if (BITS == 4) word[u] = *reinterpret_cast<const uint32_t*>(cur.k + ((size_t)h * cap + slot) * 32 + 4 * w);
+        else wide[u] = *reinterpret_cast<const uint4*>(cur.k + ((size_t)h * cap + slot) * 128 + 16 * w);
+      }
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = (h == 0) ? x[j] : __fadd_rn(acc[j], x[j]);
+    for (int u = 0; u < 4; ++u) {
+      const int h = h0 + u;
+      if (h < H) {
+        float x[8];
+        if (BITS == 4) {
+          if (plain) {
+            dequant8_plain(word[u], s_par + h * 64 + 8 * w, x);
+          } else {
+            float2 par[8];
+            const float4* pp = reinterpret_cast<const float4*>(s_par) + h * 32 + w;
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              const float4 t = pp[v * 8];
+              par[2 * v] = make_float2(t.x, t.y);
+              par[2 * v + 1] = make_float2(t.z, t.w);
+            }
+            dequant8_magic(word[u], par, x);
+          }
+        } else {
+          bf16x8_to_float(wide[u], x);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = (h == 0) ? x[j] : __fadd_rn(acc[j], x[j]);
+      }
+    }
   }
   const float inv_h = __fdiv_rn(1.f, (float)H);
   float p[8];
@@ -264,19 +397,21 @@ cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st) {
   LaunchScope ls(c, XKV_PROF_SCORE, st);
   if (c->p.kv_bits == 16)
     score_kernel<16><<<blocks, 512, smem, st>>>(c->buf[c->cur], c->p.n_heads, c->cap, c->rest_base, r_old,
-                                                c->qvec, c->scores);
+                                                c->qvec, c->scores, c->force_plain);
   else
     score_kernel<4><<<blocks, 512, smem, st>>>(c->buf[c->cur], c->p.n_heads, c->cap, c->rest_base, r_old,
-                                               c->qvec, c->scores);
+                                               c->qvec, c->scores, c->force_plain);
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------
-// Top-k of the scores (Sec. 3.2) by radix select on the order key
-// (fp32 bit pattern mapped to an unsigned whose order is the float total order),
-// then a stable compaction: keep every key above the threshold and the first
-// (k - #above) keys equal to it.  One CTA; the input is at most a few hundred KB
-// and L2-resident.
+// Top-k of the scores (Sec. 3.2).  One CTA.  The order keys (fp32 bit pattern
+// mapped to an unsigned whose order is the float total order) are held in shared
+// memory when they fit.  The k-th largest key tau is found digit by digit (12, 10
+// and 10 bits): a pass histograms the digit of the keys that match the digits
+// found so far, a suffix scan locates the bin that holds the k-th largest.  Then
+// a stable compaction keeps every key above tau and the first (k - #above) keys
+// equal to it.  Each thread owns a run of consecutive positions.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t order_key(float f) {
   const uint32_t u = __float_as_uint(f);
@@ -284,6 +419,8 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 }
 
 constexpr int kSelThreads = 1024;
+constexpr int kSelSmemKeys = 48 * 1024;   // keys held in shared memory (192 KB)
+constexpr int kSelBins = 4096;
 
 __device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned int* s_warp,
                                                         unsigned int& total) {
@@ -314,61 +451,73 @@ __device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned
   return res;
 }
 
+template <bool IN_SMEM>
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restrict__ kept) {
-  __shared__ unsigned int s_hist[256];
-  __shared__ unsigned int s_scan[256];
+  extern __shared__ uint32_t s_keys[];
+  __shared__ unsigned int s_hist[kSelBins];
   __shared__ unsigned int s_warp[33];
   __shared__ unsigned int s_prefix, s_need;
   const int tid = threadIdx.x;
   const int lane = tid & 31;
+  if (IN_SMEM)
+    for (int j = tid; j < tp; j += kSelThreads) s_keys[j] = order_key(scores[j]);
   if (tid == 0) { s_prefix = 0u; s_need = (unsigned int)k; }
-  unsigned int mask = 0u;
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    if (tid < 256) s_hist[tid] = 0u;
+  auto key_at = [&](int j) -> uint32_t { return IN_SMEM ? s_keys[j] : order_key(scores[j]); };
+
+  uint32_t mask = 0u;                  // bits of the key decided so far
+  int shift = 32;
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    const int bits = (pass == 0) ? 12 : 10;
+    const int nbins = 1 << bits;
+    shift -= bits;
+    for (int b = tid; b < nbins; b += kSelThreads) s_hist[b] = 0u;
     __syncthreads();
-    const unsigned int prefix = s_prefix;
+    const uint32_t prefix = s_prefix;
     for (int base = 0; base < tp; base += kSelThreads) {
       const int j = base + tid;
       const bool in = j < tp;
-      const uint32_t key = in ? order_key(scores[j]) : 0u;
+      const uint32_t key = in ? key_at(j) : 0u;
       const bool cand = in && ((key & mask) == prefix);
-      const unsigned int digit = cand ? ((key >> shift) & 255u) : 256u;
-      // warp-aggregated histogram update: one atomic per distinct digit per warp
-      const unsigned int peers = __match_any_sync(0xffffffffu, digit);
-      if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[digit], (unsigned int)__popc(peers));
-    }
-    __syncthreads();
-    // s_scan[b] = number of candidates with digit > b (suffix sum), 256 threads, 8 doubling steps
-    if (tid < 256) s_scan[tid] = (tid < 255) ? s_hist[tid + 1] : 0u;
-    __syncthreads();
-    for (int o = 1; o < 256; o <<= 1) {
-      unsigned int add = 0u;
-      if (tid < 256 && tid + o < 256) add = s_scan[tid + o];
-      __syncthreads();
-      if (tid < 256) s_scan[tid] += add;
-      __syncthreads();
-    }
-    if (tid < 256) {
-      const unsigned int above = s_scan[tid];
-      const unsigned int need = s_need;
-      if (above < need && need <= above + s_hist[tid]) {
-        s_prefix = prefix | ((unsigned int)tid << shift);
-        s_need = need - above;
+      const uint32_t digit = (key >> shift) & (uint32_t)(nbins - 1);
+      // a warp whose candidates all share one digit (e.g. all scores equal) adds once
+      const unsigned int cands = __ballot_sync(0xffffffffu, cand);
+      if (cands) {
+        const int leader = __ffs(cands) - 1;
+        const uint32_t d0 = __shfl_sync(0xffffffffu, digit, leader);
+        const bool same = __all_sync(0xffffffffu, !cand || digit == d0);
+        if (same) { if (lane == leader) atomicAdd(&s_hist[d0], (unsigned int)__popc(cands)); }
+        else if (cand) atomicAdd(&s_hist[digit], 1u);
       }
     }
-    mask |= 0xFFu << shift;
+    __syncthreads();
+    // suffix scan: thread t owns `per` bins counted from the top
+    const int per = nbins / kSelThreads;                   // 4 or 1
+    unsigned int h[4] = {0u, 0u, 0u, 0u};
+    unsigned int own = 0u;
+    for (int u = 0; u < per; ++u) { h[u] = s_hist[nbins - 1 - (tid * per + u)]; own += h[u]; }
+    unsigned int total;
+    unsigned int above = block_excl_scan(own, s_warp, total);   // keys with a larger digit than this thread's bins
+    const unsigned int need = s_need;
+    for (int u = 0; u < per; ++u) {
+      if (above < need && need <= above + h[u]) {
+        s_prefix = prefix | ((uint32_t)(nbins - 1 - (tid * per + u)) << shift);
+        s_need = need - above;
+      }
+      above += h[u];
+    }
+    mask |= (uint32_t)(nbins - 1) << shift;
     __syncthreads();
   }
   const uint32_t tau = s_prefix;
   const unsigned int need_eq = s_need;
-  // stable compaction; each thread owns a run of consecutive positions
-  const int ipt = (tp + kSelThreads - 1) / kSelThreads;
+  // stable compaction; an odd run length keeps the runs of a warp on different shared-memory banks
+  const int ipt = ((tp + kSelThreads - 1) / kSelThreads) | 1;
   const int j0 = min(tid * ipt, tp), j1 = min(j0 + ipt, tp);
   unsigned int cnt_eq = 0u, cnt_gt = 0u;
   for (int j = j0; j < j1; ++j) {
-    const uint32_t key = order_key(scores[j]);
+    const uint32_t key = key_at(j);
     cnt_eq += (key == tau);
     cnt_gt += (key > tau);
   }
@@ -378,7 +527,7 @@ select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restri
   if (eq_before < need_eq) take_eq = min(cnt_eq, need_eq - eq_before);
   unsigned int out = block_excl_scan(cnt_gt + take_eq, s_warp, total);
   for (int j = j0; j < j1; ++j) {
-    const uint32_t key = order_key(scores[j]);
+    const uint32_t key = key_at(j);
     bool keep = key > tau;
     if (key == tau && take_eq > 0u) { keep = true; --take_eq; }
     if (keep) kept[out++] = j;
@@ -386,63 +535,151 @@ select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restri
 }
 
 cudaError_t launch_select(xkv_cache* c, int r_old, int k, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    const cudaError_t e = cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               kSelSmemKeys * (int)sizeof(uint32_t));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
   LaunchScope ls(c, XKV_PROF_SELECT, st);
-  select_kernel<<<1, kSelThreads, 0, st>>>(c->scores, r_old, k, c->kept);
+  if (r_old <= kSelSmemKeys)
+    select_kernel<true><<<1, kSelThreads, (size_t)r_old * sizeof(uint32_t), st>>>(c->scores, r_old, k, c->kept);
+  else
+    select_kernel<false><<<1, kSelThreads, 0, st>>>(c->scores, r_old, k, c->kept);
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------
-// kv_quant_pack, keys (4-bit).  One CTA per (new 64-slot group, head); thread =
-// (token, 8-channel word).  Survivors are dequantised with the parameters of
-// the group they came from (Eq. 10), new keys come from the bf16 staging buffer;
-// per-channel min/max over the group's tokens; new parameters and codes
-// (Eq. 7-8).  A complete group whose 64 tokens all survive in place is copied.
+// kv_quant_pack, 4-bit.  One CTA per (new 64-slot key group, four heads); 128
+// threads per head, thread = (8-channel word, four tokens 16 apart).
+// Keys: survivors are dequantised with the parameters of the group they came
+// from (Eq. 10), new keys come from the bf16 staging buffer; per-channel min/max
+// over the group's tokens; new parameters and codes (Eq. 7-8).  A complete group
+// whose 64 tokens all survive in place is copied.
+// Values: the survivors' code rows and parameters, and the origins, move to
+// their new slots in the other buffer set (they were quantised on arrival).
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(512)
-regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int cap, int max_n, int base_slot, int kk,
-                 int r_new, const int32_t* __restrict__ kept, const __nv_bfloat16* __restrict__ kstage) {
-  __shared__ float s_mn[16][64];
-  __shared__ float s_mx[16][64];
-  __shared__ float2 s_iz[64];
+constexpr int kRgHeads = 4;
+
+__global__ void __launch_bounds__(128 * kRgHeads, 2)
+regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int H, int cap, int max_n, int base_slot, int kk,
+                 int r_new, const int32_t* __restrict__ kept, const __nv_bfloat16* __restrict__ kstage,
+                 int force_plain) {
+  __shared__ int s_old[64];                      // source position (rest-local) of each token, -1 = new key
+  __shared__ float s_mn[kRgHeads][4][64];
+  __shared__ float s_mx[kRgHeads][4][64];
+  __shared__ float2 s_iz[kRgHeads][64];
   const int tid = threadIdx.x;
-  const int w = tid & 7;
-  const int tok = tid >> 3;
-  const int warp = tid >> 5;
   const int gamma = blockIdx.x;
-  const int h = blockIdx.y;
-  const int i = gamma * 64 + tok;
-  const bool valid = i < r_new;
-  const size_t dslot = (size_t)h * cap + base_slot + i;
-  const size_t dgrp = ((size_t)h * (cap >> 6) + (base_slot >> 6) + gamma) * 64;
+  const int hl = tid >> 7;                       // head within the CTA
+  const int h = blockIdx.y * kRgHeads + hl;
+  const int t = tid & 127;
+  const int w = t & 7;
+  const int tq = t >> 3;                         // tokens tq + 16 u
+  const int wih = t >> 5;                        // warp within the head
+  const bool head_ok = h < H;
+  if (tid < 64) {
+    const int i = gamma * 64 + tid;
+    s_old[tid] = (i < kk) ? (kept ? kept[i] : i) : -1;
+  }
+  __syncthreads();
+
+  // ---- values, parameters and origins of the survivors (first frame: nothing to move) ----
+  if (kk > 0) {
+    for (int e = tid; e < kRgHeads * 64 * 2; e += 128 * kRgHeads) {
+      const int half = e & 1, tok = (e >> 1) & 63, hh = blockIdx.y * kRgHeads + (e >> 7);
+      const int i = gamma * 64 + tok;
+      if (hh < H && i < kk) {
+        const size_t s_slot = (size_t)hh * cap + base_slot + s_old[tok];
+        const size_t d_slot = (size_t)hh * cap + base_slot + i;
+        *reinterpret_cast<uint4*>(dst.v + d_slot * 32 + 16 * half) =
+            *reinterpret_cast<const uint4*>(src.v + s_slot * 32 + 16 * half);
+        if (half == 0) dst.vpar[d_slot] = src.vpar[s_slot];
+      }
+    }
+    if (blockIdx.y == 0 && tid < 64) {
+      const int i = gamma * 64 + tid;
+      if (i < kk) dst.origin[base_slot + i] = src.origin[base_slot + s_old[tid]];
+    }
+  }
+
+  // ---- keys ----
   const int last = gamma * 64 + 63;
-  const bool carried = (last < kk) && (kept == nullptr || kept[last] == last);
+  const bool carried = (last < kk) && (s_old[63] == last);
+  const size_t dgrp = ((size_t)h * (cap >> 6) + (base_slot >> 6) + gamma) * 64;
   if (carried) {
-    const uint32_t word = *reinterpret_cast<const uint32_t*>(src.k + dslot * 32 + 4 * w);
-    *reinterpret_cast<uint32_t*>(dst.k + dslot * 32 + 4 * w) = word;
-    if (two) *reinterpret_cast<uint32_t*>(dst2.k + dslot * 32 + 4 * w) = word;
-    if (tid < 64) {
-      const float2 sz = src.kpar[dgrp + tid];
-      dst.kpar[dgrp + tid] = sz;
-      if (two) dst2.kpar[dgrp + tid] = sz;
+    if (head_ok) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const size_t dslot = (size_t)h * cap + base_slot + gamma * 64 + tq + 16 * u;
+        const uint32_t word = *reinterpret_cast<const uint32_t*>(src.k + dslot * 32 + 4 * w);
+        *reinterpret_cast<uint32_t*>(dst.k + dslot * 32 + 4 * w) = word;
+        if (two) *reinterpret_cast<uint32_t*>(dst2.k + dslot * 32 + 4 * w) = word;
+      }
+      if (t < 64) {
+        const float2 sz = src.kpar[dgrp + t];
+        dst.kpar[dgrp + t] = sz;
+        if (two) dst2.kpar[dgrp + t] = sz;
+      }
     }
     return;
   }
-  float x[8];
-  if (valid && i < kk) {
-    const int old = kept ? kept[i] : i;
-    const size_t sslot = (size_t)h * cap + base_slot + old;
-    const uint32_t word = *reinterpret_cast<const uint32_t*>(src.k + sslot * 32 + 4 * w);
-    const float2* par = src.kpar + ((size_t)h * (cap >> 6) + ((base_slot + old) >> 6)) * 64 + 8 * w;
-    dequant8(word, par, x);
-  } else if (valid) {
-    const uint4 u = *reinterpret_cast<const uint4*>(kstage + ((size_t)h * max_n + (i - kk)) * 64 + 8 * w);
-    bf16x8_to_float(u, x);
+  float x[4][8];
+  uint32_t word[4];
+  uint4 fresh[4];
+  int old[4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int tok = tq + 16 * u;
+    const int i = gamma * 64 + tok;
+    old[u] = (i < r_new) ? s_old[tok] : -2;      // -2: beyond the segment
+    word[u] = 0u;
+    fresh[u] = make_uint4(0, 0, 0, 0);
+    if (head_ok && old[u] >= 0)
+      word[u] = *reinterpret_cast<const uint32_t*>(src.k + ((size_t)h * cap + base_slot + old[u]) * 32 + 4 * w);
+    else if (head_ok && old[u] == -1)
+      fresh[u] = *reinterpret_cast<const uint4*>(kstage + ((size_t)h * max_n + (i - kk)) * 64 + 8 * w);
+  }
+  int par_grp = -1;
+  float2 par[8];
+  bool par_plain = false;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    if (old[u] >= 0) {
+      const int g = (base_slot + old[u]) >> 6;
+      if (g != par_grp && head_ok) {
+        const float4* pp = reinterpret_cast<const float4*>(src.kpar + ((size_t)h * (cap >> 6) + g) * 64 + 8 * w);
+        float zmax = 0.f;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const float4 q4 = __ldg(pp + v);
+          par[2 * v] = make_float2(q4.x, q4.y);
+          par[2 * v + 1] = make_float2(q4.z, q4.w);
+          zmax = fmaxf(zmax, fmaxf(fabsf(q4.y), fabsf(q4.w)));
+        }
+        par_plain = !(zmax < kZLimit) || force_plain;
+        if (!par_plain) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) par[j].y = __fadd_rn(magic_val(j), par[j].y);
+        }
+        par_grp = g;
+      }
+      if (par_plain) dequant8_plain(word[u], par, x[u]);
+      else dequant8_magic(word[u], par, x[u]);
+    } else {
+      bf16x8_to_float(fresh[u], x[u]);
+    }
   }
   float mn[8], mx[8];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    mn[j] = valid ? x[j] : INFINITY;
-    mx[j] = valid ? x[j] : -INFINITY;
+  for (int j = 0; j < 8; ++j) { mn[j] = INFINITY; mx[j] = -INFINITY; }
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    if (old[u] != -2) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { mn[j] = fminf(mn[j], x[u][j]); mx[j] = fmaxf(mx[j], x[u][j]); }
+    }
   }
   // tokens of a warp: lanes with equal (lane & 7) hold the same channels
 #pragma unroll
@@ -453,33 +690,54 @@ regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int cap, int max
       mx[j] = fmaxf(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], o));
     }
   }
-  if ((tid & 31) < 8) {
+  if ((t & 31) < 8) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) { s_mn[warp][8 * w + j] = mn[j]; s_mx[warp][8 * w + j] = mx[j]; }
+    for (int j = 0; j < 8; ++j) { s_mn[hl][wih][8 * w + j] = mn[j]; s_mx[hl][wih][8 * w + j] = mx[j]; }
   }
   __syncthreads();
   // one thread per channel finishes the reduction and derives the group's parameters
-  if (tid < 64) {
-    float a = s_mn[0][tid], b = s_mx[0][tid];
+  int slow = force_plain;
+  if (t < 64) {
+    float a = s_mn[hl][0][t], b = s_mx[hl][0][t];
 #pragma unroll
-    for (int r = 1; r < 16; ++r) { a = fminf(a, s_mn[r][tid]); b = fmaxf(b, s_mx[r][tid]); }
+    for (int r = 1; r < 4; ++r) { a = fminf(a, s_mn[hl][r][t]); b = fmaxf(b, s_mx[hl][r][t]); }
     float sc, inv, z;
     quant_params(a, b, sc, inv, z);
-    s_iz[tid] = make_float2(inv, z);
-    dst.kpar[dgrp + tid] = make_float2(sc, z);
-    if (two) dst2.kpar[dgrp + tid] = make_float2(sc, z);
+    s_iz[hl][t] = make_float2(inv, z);
+    if (head_ok) {
+      dst.kpar[dgrp + t] = make_float2(sc, z);
+      if (two) dst2.kpar[dgrp + t] = make_float2(sc, z);
+      // the conversion-free quantiser needs |x * inv| < 2^21 and |z| < 2^22
+      const float ymax = __fmul_rn(fmaxf(fabsf(a), fabsf(b)), inv);
+      slow |= !(ymax < 2097152.f) || !(fabsf(z) < kZLimit);
+    }
   }
-  __syncthreads();
-  uint32_t c[8];
+  slow = __syncthreads_or(slow);
+  if (!head_ok) return;
+  float2 iz[8];
+  int zadj[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    const float2 iz = s_iz[8 * w + j];
-    c[j] = valid ? quant_code(x[j], iz.x, iz.y) : 0u;
+    iz[j] = s_iz[hl][8 * w + j];
+    zadj[j] = slow ? 0 : (int)iz[j].y - (int)0x4B400000;
   }
-  if (valid) {
-    const uint32_t word = pack8(c);
-    *reinterpret_cast<uint32_t*>(dst.k + dslot * 32 + 4 * w) = word;
-    if (two) *reinterpret_cast<uint32_t*>(dst2.k + dslot * 32 + 4 * w) = word;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    if (old[u] == -2) continue;
+    uint32_t packed;
+    if (slow) {
+      packed = 0u;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) packed |= quant_code_call(x[u][j], iz[j].x, iz[j].y) << nib_shift(j);
+    } else {
+      packed = 0u;
+#pragma unroll
+      for (int j = 0; j < 8; ++j)   // the nibbles do not overlap: multiply-add places them
+        packed = quant_code_magic(x[u][j], iz[j].x, zadj[j]) * (1u << nib_shift(j)) + packed;
+    }
+    const size_t dslot = (size_t)h * cap + base_slot + gamma * 64 + tq + 16 * u;
+    *reinterpret_cast<uint32_t*>(dst.k + dslot * 32 + 4 * w) = packed;
+    if (two) *reinterpret_cast<uint32_t*>(dst2.k + dslot * 32 + 4 * w) = packed;
   }
 }
 
@@ -515,27 +773,19 @@ cudaError_t launch_pack(xkv_cache* c, int n, int kk, bool identity, bool first, 
   const int32_t* kept = identity ? nullptr : c->kept;
   const int H = c->p.n_heads;
   if (c->p.kv_bits == 4) {
+    // one kernel: key regroup + survivor gather of values, value parameters and origins
     const int base = first ? 0 : c->rest_base;
     const int r_new = kk + n;
-    const dim3 grid((r_new + 63) / 64, H);
-    cudaError_t e;
-    {
-      LaunchScope ls(c, XKV_PROF_REGROUP, st);
-      regroup_k_kernel<<<grid, 512, 0, st>>>(src, dst, src, first, c->cap, c->p.max_frame_tokens, base, kk,
-                                             r_new, kept, c->kstage);
-      e = cudaGetLastError();
-    }
-    if (e != cudaSuccess) return e;
+    const dim3 grid((r_new + 63) / 64, (H + kRgHeads - 1) / kRgHeads);
+    LaunchScope ls(c, XKV_PROF_REGROUP, st);
+    regroup_k_kernel<<<grid, 128 * kRgHeads, 0, st>>>(src, dst, src, first, H, c->cap, c->p.max_frame_tokens, base,
+                                                     kk, r_new, kept, c->kstage, c->force_plain);
+    return cudaGetLastError();
   }
   if (kk > 0) {
     LaunchScope ls(c, XKV_PROF_GATHER, st);
-    if (c->p.kv_bits == 4) {
-      const long long threads = (long long)H * kk * 2;
-      gather_kernel<4><<<(int)((threads + 255) / 256), 256, 0, st>>>(src, dst, H, c->cap, c->rest_base, kk, kept);
-    } else {
-      const long long threads = (long long)H * kk * 8;
-      gather_kernel<16><<<(int)((threads + 255) / 256), 256, 0, st>>>(src, dst, H, c->cap, c->rest_base, kk, kept);
-    }
+    const long long threads = (long long)H * kk * 8;
+    gather_kernel<16><<<(int)((threads + 255) / 256), 256, 0, st>>>(src, dst, H, c->cap, c->rest_base, kk, kept);
   }
   return cudaGetLastError();
 }

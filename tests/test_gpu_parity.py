@@ -31,6 +31,41 @@ def test_tiny_stream_4bit(xkv, impl):
     print("tiny 4-bit impl", impl, "worst (max-abs, rel-L2)", worst)
 
 
+def test_tiny_stream_4bit_plain_arithmetic_forms(xkv, monkeypatch):
+    """The maintenance kernels dequantise and quantise without conversion instructions when the
+    zero-points and scaled values are small enough, and fall back to the plain forms otherwise.
+    XKV_FORCE_PLAIN=1 (read when a cache is created) sends every kernel down the fallback:
+    both must give the oracle's bits."""
+    monkeypatch.setenv("XKV_FORCE_PLAIN", "1")
+    p = xkv.Params(budget=1024, max_frame_tokens=261, kv_bits=4)
+    cache, ora, worst = run_stream(xkv, p, 261, 7, seed=11)
+    assert cache.xkv_get_info().T == 1024
+
+
+def test_large_offset_keys(xkv):
+    """Keys with a large common offset: zero-points of a few thousand and |x / s| far from 0."""
+    import torch
+    from xkv_testlib import compare_state, oracle_params, bf16_tensor_to_f32, check_attention
+    from oracle import xkv_oracle as xo
+    p = xkv.Params(n_heads=4, budget=400, max_frame_tokens=128, kv_bits=4)
+    cache, ora = xkv.Cache(p), xo.OracleLayer(oracle_params(p))
+    H, n, d = 4, 128, 64
+    for t in range(6):
+        qb, kb, vb = synth.gen_frame(12, 0, t, H, n, d)
+        kf = synth.bf16_bits_to_f32(kb) * np.float32(0.05) + np.float32(100.0)
+        kb = synth.f32_to_bf16_bits(kf)
+        qf, kf, vf = (synth.bf16_bits_to_f32(x) for x in (qb, kb, vb))
+        q, k, v = (to_device_bf16(x) for x in (qb, kb, vb))
+        cache.kv_append(k, v); cache.kv_score_evict(q); cache.kv_quant_pack()
+        ora.append(kf, vf); ora.score_evict(qf); ora.quant_pack()
+        compare_state(cache.export(), ora.export(), f"frame {t}")
+        # keys near 100 with a spread of 0.05 cannot be held in 16-bit operands (spacing 0.06), so the
+        # attention check uses the fp32 CUDA-core kernel; the point here is the bit-exact state above
+        out = cache.attn_packed_causal(q, impl=1)
+        check_attention(bf16_tensor_to_f32(out).transpose(1, 0, 2), ora.attend(qf), f"frame {t}")
+    assert cache.xkv_get_info().T == 400
+
+
 @pytest.mark.parametrize("impl", [0, 1])
 def test_tiny_stream_16bit(xkv, impl):
     p = xkv.Params(budget=1024, max_frame_tokens=261, kv_bits=16)

@@ -174,9 +174,9 @@ XKV_API int attn_packed_causal(xkv_cache* cache, const void* q, void* out, int32
  * application that forbids allocation after start-up, a plug-in whose host owns
  * the allocator, a process that shares its GPU with a job whose memory pool must
  * not be disturbed - and that therefore cannot grow a buffer for the attention
- * kernel's scratch.  The tensor-core kernel splits the keys of one head over
- * several thread blocks and needs global memory for the partial results (64
- * accumulators plus running max and sum per split, head and query).
+ * kernel's scratch.  The tensor-core kernel cuts the keys of a head between
+ * thread blocks and needs global memory for the partial results (64
+ * accumulators plus running max and sum per query row and cut).
  * attn_packed_causal keeps them in the cache workspace; this variant keeps them
  * in a fixed array of XKV_STATIC_SCRATCH_BYTES that is part of the library image
  * and leaves that region of the workspace untouched.  Every GPU on which the
@@ -187,11 +187,14 @@ XKV_API int attn_packed_causal(xkv_cache* cache, const void* q, void* out, int32
  * Rules of use
  *   - Same arguments, state requirements and result as attn_packed_causal with
  *     impl = 0; q and out are still the caller's.
- *   - A launch whose partials need more than XKV_STATIC_SCRATCH_BYTES is refused
- *     with XKV_E_LIMIT before anything is enqueued; the cache stays in the packed
- *     state, so attn_packed_causal can still take the frame.  The need is
- *     splits * n_heads * n * 264 bytes, splits <= 6 chosen from the grid size;
- *     a single split (short caches) needs none.
+ *   - The need does not grow with the frame or the cache: each thread block
+ *     leaves at most two partial slots of 135 168 bytes, and the kernel runs one
+ *     block per multiprocessor.  The array holds XKV_STATIC_SCRATCH_BYTES /
+ *     135 168 = 248 slots; on a GPU with more than 124 multiprocessors the
+ *     variant launches 124 blocks instead of one per multiprocessor (slower,
+ *     same result).  If not even one block's slots fit, the call returns
+ *     XKV_E_LIMIT before anything is enqueued and the cache stays in the packed
+ *     state, so attn_packed_causal can still take the frame.
  *   - The first call on a device looks up the array's device address (once per
  *     device, with that device current).  Make that first call outside any
  *     stream capture.
@@ -234,6 +237,11 @@ XKV_API int xkv_get_info(const xkv_cache* cache, xkv_info* info);
  * copied (>= 0) or a negative xkv_status. */
 XKV_API int64_t xkv_debug_export(const xkv_cache* cache, int32_t which, void* host_dst, size_t bytes,
                          xkv_stream stream);
+
+/* Tests and benchmarks only: puts an idle cache that holds at least one frame back
+ * into the packed state, so that attn_packed_causal can run again on the same
+ * cache contents (with the same or other queries).  XKV_E_STATE otherwise. */
+XKV_API int xkv_debug_rewind_attention(xkv_cache* cache);
 
 /* Synchronises `stream` and returns the device status word of the cache:
  * XKV_OK, or XKV_E_TIMEOUT if a bounded wait inside a kernel ran out. */

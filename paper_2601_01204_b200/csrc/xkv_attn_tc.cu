@@ -1,25 +1,38 @@
 // Tensor-core attention over the packed cache (Eq. 1 with the dequantisation of
-// Eq. 10) for sm_100a: tcgen05.mma with accumulators in tensor memory.
+// Eq. 10) for sm_100a: tcgen05.mma with accumulators in tensor memory, operands
+// staged by bulk asynchronous copies (TMA) and dequantised in shared memory.
 //
-// One CTA = one tile of 128 queries of one head over a contiguous range of
-// 128-slot key tiles (split-KV).  Warp roles:
-//   warps 0-3  softmax: thread r owns query row r = TMEM lane r.  Reads S from
-//              TMEM, online max/sum, writes P (16-bit) back to TMEM, rescales O
-//              when the running maximum moved by more than 2^8, epilogue.
-//   warps 4-7  operand producers: 4-bit codes -> fp16 (K~ per channel/group, V~
-//              per token) written into shared memory in the 128-byte-swizzled
-//              layouts the MMA descriptors expect.
-//   warp  8    allocates tensor memory; one elected thread issues the MMAs:
-//              S = Q K~^T (M128 N128 K64, both operands K-major in smem) and
-//              O += P V~ (M128 N64 K128, A = P from TMEM, B = V~ MN-major).
+// Work.  An item is (head, pair of 128-query tiles); it meets every 128-slot key
+// tile of the cache.  Items x key tiles are laid out on one line of steps, and the
+// line is cut into equal pieces, one per CTA (one CTA per SM).  A piece that does
+// not cover an item completely leaves partial results (accumulator, running max
+// and sum) in a scratch slot; a second kernel merges them.
+//
+// One CTA, 14 warps:
+//   warps 0-3   softmax of query tile 0: thread r owns query row r = TMEM lane r.
+//               Reads S from tensor memory, online max/sum, writes P (16-bit) back
+//               to tensor memory, rescales O only when the running maximum grew by
+//               more than 2^8, epilogue.
+//   warps 4-7   the same for query tile 1.  The two groups alternate naturally:
+//               while one computes exponentials the tensor pipe produces the
+//               other's scores.
+//   warps 8-11  operand producers: packed 4-bit codes (raw, as copied by TMA) ->
+//               fp16 K~ (per channel and 64-slot group) and V~ (per token) in the
+//               128-byte-swizzled layouts the MMA descriptors expect.  One
+//               dequantised tile serves both query tiles.
+//   warp 12     one thread issues the MMAs: S_t = Q_t K~^T (M128 N128 K64) and
+//               O_t += P_t V~ (M128 N64 K128, A = P from tensor memory).
+//   warp 13     one thread issues the bulk copies of the raw tiles, several steps
+//               ahead; the warp owns the tensor-memory allocation (all 512 columns).
 // 4-bit caches multiply in fp16 (the dequantised keys are not bf16-representable:
 // rounding them to bf16 alone costs ~1e-2 relative L2 with outlier channels);
 // 16-bit caches hold bf16 and multiply in bf16.  Accumulation is fp32.
 //
 // Every mbarrier wait is bounded: when the bound is hit the thread records
-// XKV_E_TIMEOUT in the cache's status word and carries on, so the kernel always
-// terminates and frees its tensor memory.
+// XKV_E_TIMEOUT in the cache's status word and carries on without waiting, so the
+// kernel always terminates, drains its copies and frees its tensor memory.
 #include <mutex>
+#include <stdlib.h>
 
 #include "xkv_internal.cuh"
 
@@ -28,23 +41,47 @@ namespace xkv {
 namespace {
 
 constexpr int kMaxDevices = 64;
-constexpr int kThreads = 288;
+constexpr int kThreads = 448;
 constexpr int kQRows = 128;
-constexpr int kMaxSplits = 6;
+constexpr int kMaxGrid = 160;                 // CTAs the scratch is sized for (>= SM count of the part)
 constexpr uint32_t kSpinLimit = 1u << 22;
 
-// shared memory map (offsets from a 1024-byte aligned base)
-constexpr int kOffQ = 0;                 // 16 KB  Q tile, K-major, SW128
-constexpr int kOffK = 16384;             // 2 x 16 KB  K~ tiles
-constexpr int kOffV = 16384 * 3;         // 2 x 16 KB  V~ tiles
-constexpr int kOffBar = 16384 * 5;       // barriers + tmem base
-constexpr int kSmemBytes = kOffBar + 256 + 1024;   // + alignment slack
+// ring depths
+constexpr int kNK = 3;                        // dequantised K~ tiles
+constexpr int kNV = 3;                        // dequantised V~ tiles
 
-// tensor memory columns
-constexpr int kColS = 0;      // 128 fp32 columns
-constexpr int kColP = 128;    // 64 columns of packed 16-bit pairs
-constexpr int kColO = 192;    // 64 fp32 columns
-constexpr int kTmemCols = 256;
+template <int BITS> struct Cfg;
+template <> struct Cfg<4> {
+  static constexpr int kNR = 4;               // raw stages
+  static constexpr int kRawK = 4096, kRawV = 4096, kRawKP = 1024, kRawVP = 1024;
+  static constexpr int kRawStage = kRawK + kRawV + kRawKP + kRawVP;
+};
+template <> struct Cfg<16> {
+  static constexpr int kNR = 2;
+  static constexpr int kRawK = 16384, kRawV = 16384, kRawKP = 0, kRawVP = 0;
+  static constexpr int kRawStage = kRawK + kRawV;
+};
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr int kOffQ = 0;                          // 2 x 16 KB  Q tiles, K-major, SW128
+constexpr int kOffK = 32768;                      // kNK x 16 KB  K~ tiles
+constexpr int kOffV = kOffK + kNK * 16384;        // kNV x 16 KB  V~ tiles
+constexpr int kOffTab = kOffV + kNV * 16384;      // 2 x (K table 512 B + V table 2048 B) fp16 parameters
+constexpr int kTabBytes = 512 + 2048;
+constexpr int kOffBar = kOffTab + 2 * kTabBytes;  // barriers, tmem base, abort flag
+constexpr int kBarBytes = 512;
+constexpr int kOffRaw = kOffBar + kBarBytes;      // raw stages (16-byte aligned)
+template <int BITS> constexpr int smem_bytes() { return kOffRaw + Cfg<BITS>::kNR * Cfg<BITS>::kRawStage + 1024; }
+
+// tensor memory columns (all 512)
+constexpr int kColS = 0;      // + 128 t : 128 fp32 columns per query tile
+constexpr int kColP = 256;    // + 64 t  : 64 columns of packed 16-bit pairs
+constexpr int kColO = 384;    // + 64 t  : 64 fp32 columns
+constexpr int kTmemCols = 512;
+
+// one partial slot: two query tiles x 128 rows x (64 accumulators + max + sum)
+constexpr size_t kSlotFloats = 2 * 128 * 64;
+constexpr size_t kSlotBytes = kSlotFloats * sizeof(float) + 2 * 128 * sizeof(float2);
 
 struct Args {
   const __nv_bfloat16* q;
@@ -55,13 +92,20 @@ struct Args {
   const float2* kpar;
   const uint8_t* v;
   const float2* vpar;
-  int cap, t_first, rest_base, t_phys;
+  int cap, t_first, t_phys;
   float scale_log2;
-  int n_tiles, tiles_per_split, n_splits;
-  float* part_o;     // [split][H][n][64]
-  float2* part_ml;   // [split][H][n]
+  int n_tiles;          // key tiles of the cache
+  int q_tiles;          // 128-row query tiles of the frame
+  int n_pairs;          // ceil(q_tiles / 2)
+  long long total;      // items * n_tiles
+  float* part_o;        // [2 * grid][2][128][64]
+  float2* part_ml;      // [2 * grid][2][128]
   int* status;
 };
+
+__device__ __forceinline__ long long piece_start(long long total, int grid, int b) {
+  return (total * (long long)b) / (long long)grid;
+}
 
 // ---- PTX wrappers -----------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -242,341 +286,444 @@ __device__ __forceinline__ uint4 dequant_word_h(uint32_t w, const uint32_t (&s2)
   return r;
 }
 
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bulk asynchronous copy global -> this CTA's shared memory, completion counted on an mbarrier.
+// Addresses 16-byte aligned, size a multiple of 16.  No multicast.
+__device__ __forceinline__ void tma_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void producer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
 }  // namespace
 
 template <int BITS>
-__global__ void __launch_bounds__(kThreads, 2) attn_tc_kernel(const Args a) {
+__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
+  using C = Cfg<BITS>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
-  const uint32_t sQ = sbase + kOffQ, sK = sbase + kOffK, sV = sbase + kOffV;
+  const uint32_t sQ = sbase + kOffQ, sK = sbase + kOffK, sV = sbase + kOffV, sRaw = sbase + kOffRaw;
   const uint32_t bar0 = sbase + kOffBar;
   // barrier slots (8 bytes each)
-  const uint32_t b_kfull = bar0, b_kfree = bar0 + 16, b_vfull = bar0 + 32, b_vfree = bar0 + 48;
-  const uint32_t b_sfull = bar0 + 64, b_sfree = bar0 + 72, b_pfull = bar0 + 80, b_pvdone = bar0 + 88;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sgen + kOffBar + 128);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + kOffBar + 132);
+  const uint32_t b_kfull = bar0, b_kfree = bar0 + 8 * kNK;
+  const uint32_t b_vfull = b_kfree + 8 * kNK, b_vfree = b_vfull + 8 * kNV;
+  const uint32_t b_rfull = b_vfree + 8 * kNV, b_rfree = b_rfull + 8 * C::kNR;
+  const uint32_t b_qfull = b_rfree + 8 * C::kNR;      // [2]
+  const uint32_t b_sfull = b_qfull + 16, b_pfull = b_sfull + 16, b_pvdone = b_pfull + 16;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sgen + kOffBar + kBarBytes - 16);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + kOffBar + kBarBytes - 12);
   const WaitCtx wc{a.status, abort_flag};
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
-  const int h = blockIdx.y;
-  const int q0 = blockIdx.x * kQRows;
-  const int split = blockIdx.z;
-  const int tile_lo = split * a.tiles_per_split;
-  const int tile_hi = min(tile_lo + a.tiles_per_split, a.n_tiles);
-  const int nt = tile_hi - tile_lo;
   constexpr bool kBf16 = (BITS == 16);
+
+  // this CTA's piece of the line of steps
+  const long long step_lo = piece_start(a.total, gridDim.x, blockIdx.x);
+  const long long step_hi = piece_start(a.total, gridDim.x, blockIdx.x + 1);
 
   if (tid == 0) {
     *abort_flag = (*reinterpret_cast<volatile int*>(a.status) != 0) ? 1 : 0;   // an earlier CTA already gave up
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(b_kfull + 8 * i, 128); mbar_init(b_kfree + 8 * i, 1);
-      mbar_init(b_vfull + 8 * i, 128); mbar_init(b_vfree + 8 * i, 1);
+    for (int i = 0; i < kNK; ++i) { mbar_init(b_kfull + 8 * i, 128); mbar_init(b_kfree + 8 * i, 1); }
+    for (int i = 0; i < kNV; ++i) { mbar_init(b_vfull + 8 * i, 128); mbar_init(b_vfree + 8 * i, 1); }
+    for (int i = 0; i < C::kNR; ++i) { mbar_init(b_rfull + 8 * i, 1); mbar_init(b_rfree + 8 * i, 128); }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(b_qfull + 8 * t, 128); mbar_init(b_sfull + 8 * t, 1);
+      mbar_init(b_pfull + 8 * t, 128); mbar_init(b_pvdone + 8 * t, 1);
     }
-    mbar_init(b_sfull, 1); mbar_init(b_sfree, 128); mbar_init(b_pfull, 128); mbar_init(b_pvdone, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 8) {
+  if (warp == 13) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32((const void*)tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  if (warp < 4) {
-    // Q tile: row r of this thread, bf16 -> operand type, into the swizzled K-major layout
-    const int row = q0 + tid;
-    uint4 u[8];
-    if (row < a.n) {
-      const __nv_bfloat16* qp = a.q + (int64_t)h * a.hs + (int64_t)row * a.ts;
-#pragma unroll
-      for (int c = 0; c < 8; ++c) u[c] = *reinterpret_cast<const uint4*>(qp + 8 * c);
-    } else {
-#pragma unroll
-      for (int c = 0; c < 8; ++c) u[c] = make_uint4(0, 0, 0, 0);
-    }
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      uint4 o = u[c];
-      if (!kBf16) {
-        const uint32_t r[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
-        uint32_t hh[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          hh[i] = pack_h2(__uint_as_float(r[i] << 16), __uint_as_float(r[i] & 0xFFFF0000u));
-        o = make_uint4(hh[0], hh[1], hh[2], hh[3]);
-      }
-      *reinterpret_cast<uint4*>(sgen + kOffQ + swz_off(tid, c)) = o;
-    }
-    fence_proxy_async();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp < 4) {
+  if (warp < 8) {
     // =========================== softmax warps ===============================
-    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-    float m_ref = -INFINITY;   // reference maximum (scaled, log2 units) used for the exponentials
-    uint64_t l2 = 0ull;        // two partial row sums (packed fp32 pair)
+    const int t = warp >> 2;                 // query tile of the pair
+    const int r = tid & 127;                 // row of the tile = TMEM lane
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t colS = lane_addr + kColS + 128 * t, colP = lane_addr + kColP + 64 * t;
+    const uint32_t colO = lane_addr + kColO + 64 * t;
+    const uint32_t sfull = b_sfull + 8 * t, pfull = b_pfull + 8 * t, pvdone = b_pvdone + 8 * t;
     const int pad_tile = (a.t_first & 127) ? (a.t_first >> 7) : -1;
-    for (int jj = 0; jj < nt; ++jj) {
-      const int tile = tile_lo + jj;
-      int lim_lo = 128, lim_hi = 128;   // columns [lim_lo, 128) of a first-segment pad tile, [lim_hi,128) of the tail are masked
-      if (tile == pad_tile) lim_lo = a.t_first & 127;
-      if (tile == a.n_tiles - 1) lim_hi = a.t_phys - tile * 128;
-      const int lim = min(lim_lo, lim_hi);
-      mbar_wait(b_sfull, jj & 1, wc);
-      __syncwarp();
-      tc_fence_after();
-      // pass 1: row maximum
-      float mx = -INFINITY;
-      if (lim >= 128) {
-#pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t r[32];
-          XKV_TMEM_LD32(lane_addr + kColS + c0, r);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; i += 2) mx = max3(mx, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-        }
-      } else {
-#pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t r[32];
-          XKV_TMEM_LD32(lane_addr + kColS + c0, r);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float x = (c0 + i < lim) ? __uint_as_float(r[i]) : -INFINITY;
-            mx = fmaxf(mx, x);
-          }
-        }
-      }
-      mx *= a.scale_log2;
-      // decide whether the reference maximum moves (only when it grew by more than 2^8)
-      float alpha = 1.f;
-      const bool grow = mx > m_ref + 8.f;
-      if (grow) {
-        alpha = exp2f(m_ref - mx);      // 0 on the first tile (m_ref = -inf)
-        m_ref = mx;
-        l2 = mul_f2(l2, pack_f2(alpha, alpha));
-      }
-      if (jj > 0) {
-        // P(jj-1) has been consumed and O is quiescent once PV(jj-1) completed
-        mbar_wait(b_pvdone, (jj - 1) & 1, wc);
-        __syncwarp();
-        tc_fence_after();
-        if (__any_sync(0xffffffffu, grow)) {
-#pragma unroll 1
-          for (int c0 = 0; c0 < 64; c0 += 32) {
-            uint32_t r[32];
-            XKV_TMEM_LD32(lane_addr + kColO + c0, r);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-            XKV_TMEM_ST32(lane_addr + kColO + c0, r);
-          }
-          tc_wait_st();
-        }
-      }
-      // pass 2: exponentials, row sum, P -> TMEM (16-bit pairs)
-      const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2);
-      const uint64_t nm2 = pack_f2(-m_ref, -m_ref);
-      if (lim >= 128) {
-#pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t r[32];
-          XKV_TMEM_LD32(lane_addr + kColS + c0, r);
-          tc_wait_ld();
-          uint32_t pk[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const uint64_t x2 = fma_f2(pack_f2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, nm2);
-            const float p0 = fast_exp2(f2_lo(x2)), p1 = fast_exp2(f2_hi(x2));
-            l2 = add_f2(l2, pack_f2(p0, p1));
-            pk[i] = kBf16 ? pack_bf2(p0, p1) : pack_h2(p0, p1);
-          }
-          XKV_TMEM_ST16(lane_addr + kColP + (c0 >> 1), pk);
-        }
-      } else {
-#pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-          uint32_t r[32];
-          XKV_TMEM_LD32(lane_addr + kColS + c0, r);
-          tc_wait_ld();
-          uint32_t pk[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * i]), a.scale_log2, -m_ref));
-            float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), a.scale_log2, -m_ref));
-            if (c0 + 2 * i >= lim) p0 = 0.f;
-            if (c0 + 2 * i + 1 >= lim) p1 = 0.f;
-            l2 = add_f2(l2, pack_f2(p0, p1));
-            pk[i] = kBf16 ? pack_bf2(p0, p1) : pack_h2(p0, p1);
-          }
-          XKV_TMEM_ST16(lane_addr + kColP + (c0 >> 1), pk);
-        }
-      }
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(b_sfree);
-      mbar_arrive(b_pfull);
-    }
-    // epilogue
-    mbar_wait(b_pvdone, (nt - 1) & 1, wc);
-    __syncwarp();
-    tc_fence_after();
-    const int row = q0 + tid;
-    const float l = f2_lo(l2) + f2_hi(l2);
-    if (a.n_splits == 1) {
-      const float inv_l = 1.f / l;
-#pragma unroll 1
-      for (int c0 = 0; c0 < 64; c0 += 32) {
-        uint32_t r[32];
-        XKV_TMEM_LD32(lane_addr + kColO + c0, r);
-        tc_wait_ld();
+    const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2);
+    uint32_t cnt = 0;                        // steps this tile has been through (barrier phases)
+    int seg_idx = 0;
+    for (long long pos = step_lo; pos < step_hi; ++seg_idx) {
+      const int item = (int)(pos / a.n_tiles);
+      const int tile_lo = (int)(pos - (long long)item * a.n_tiles);
+      const int nt = (int)min((long long)(a.n_tiles - tile_lo), step_hi - pos);
+      pos += nt;
+      const int h = item / a.n_pairs, pair = item - h * a.n_pairs;
+      const int qt = 2 * pair + t;
+      if (qt >= a.q_tiles) continue;          // the pair has no second tile
+      // ---- Q tile: row r, bf16 -> operand type, into the swizzled K-major layout ----
+      const int row = qt * kQRows + r;
+      {
+        uint4 u[8];
         if (row < a.n) {
-          __nv_bfloat16* op = a.out + (int64_t)h * a.hs + (int64_t)row * a.ts + c0;
+          const __nv_bfloat16* qp = a.q + (int64_t)h * a.hs + (int64_t)row * a.ts;
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t o[4];
+          for (int c = 0; c < 8; ++c) u[c] = *reinterpret_cast<const uint4*>(qp + 8 * c);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) u[c] = make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          uint4 o = u[c];
+          if (!kBf16) {
+            const uint32_t rr[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
+            uint32_t hh[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-              o[i] = pack_bf2(__uint_as_float(r[8 * c + 2 * i]) * inv_l, __uint_as_float(r[8 * c + 2 * i + 1]) * inv_l);
-            *reinterpret_cast<uint4*>(op + 8 * c) = make_uint4(o[0], o[1], o[2], o[3]);
+              hh[i] = pack_h2(__uint_as_float(rr[i] << 16), __uint_as_float(rr[i] & 0xFFFF0000u));
+            o = make_uint4(hh[0], hh[1], hh[2], hh[3]);
+          }
+          *reinterpret_cast<uint4*>(sgen + kOffQ + t * 16384 + swz_off(r, c)) = o;
+        }
+        fence_proxy_async();
+        mbar_arrive(b_qfull + 8 * t);
+      }
+      float m_ref = -INFINITY;   // reference maximum (scaled, log2 units) used for the exponentials
+      uint64_t l2 = 0ull;        // two partial row sums (packed fp32 pair)
+      for (int jj = 0; jj < nt; ++jj, ++cnt) {
+        const int tile = tile_lo + jj;
+        int lim = 128;           // columns [lim, 128) are masked (pad slots after the first frame, the tail)
+        if (tile == pad_tile) lim = a.t_first & 127;
+        if (tile == a.n_tiles - 1) lim = min(lim, a.t_phys - tile * 128);
+        mbar_wait(sfull, cnt & 1, wc);
+        __syncwarp();            // the spin loops may leave the warp diverged; tcgen05.ld/st are warp-collective
+        tc_fence_after();
+        // pass 1: row maximum
+        float mx = -INFINITY;
+        if (lim >= 128) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t ra[32];
+            XKV_TMEM_LD32(colS + c0, ra);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) mx = max3(mx, __uint_as_float(ra[i]), __uint_as_float(ra[i + 1]));
+          }
+        } else {
+#pragma unroll 1
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t ra[32];
+            XKV_TMEM_LD32(colS + c0, ra);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float x = (c0 + i < lim) ? __uint_as_float(ra[i]) : -INFINITY;
+              mx = fmaxf(mx, x);
+            }
           }
         }
-      }
-    } else {
-      const size_t prow = ((size_t)split * gridDim.y + h) * a.n + row;
+        mx *= a.scale_log2;
+        // the reference maximum moves only when it grew by more than 2^8
+        float alpha = 1.f;
+        const bool grow = mx > m_ref + 8.f;
+        if (grow) {
+          alpha = exp2f(m_ref - mx);      // 0 on the first tile (m_ref = -inf)
+          m_ref = mx;
+          l2 = mul_f2(l2, pack_f2(alpha, alpha));
+        }
+        if (jj > 0) {
+          // P of the previous step has been consumed and O is quiescent once its PV completed
+          mbar_wait(pvdone, (cnt - 1) & 1, wc);
+          __syncwarp();
+          tc_fence_after();
+          if (__any_sync(0xffffffffu, grow)) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < 64; c0 += 32) {
-        uint32_t r[32];
-        XKV_TMEM_LD32(lane_addr + kColO + c0, r);
-        tc_wait_ld();
-        if (row < a.n) {
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+              uint32_t ra[32];
+              XKV_TMEM_LD32(colO + c0, ra);
+              tc_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) ra[i] = __float_as_uint(__uint_as_float(ra[i]) * alpha);
+              XKV_TMEM_ST32(colO + c0, ra);
+            }
+            tc_wait_st();
+          }
+        }
+        // pass 2: exponentials, row sum, P -> TMEM (16-bit pairs)
+        const uint64_t nm2 = pack_f2(-m_ref, -m_ref);
+        if (lim >= 128) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t ra[32];
+            XKV_TMEM_LD32(colS + c0, ra);
+            tc_wait_ld();
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const uint64_t x2 = fma_f2(pack_f2(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1])), sc2, nm2);
+              const float p0 = fast_exp2(f2_lo(x2)), p1 = fast_exp2(f2_hi(x2));
+              l2 = add_f2(l2, pack_f2(p0, p1));
+              pk[i] = kBf16 ? pack_bf2(p0, p1) : pack_h2(p0, p1);
+            }
+            XKV_TMEM_ST16(colP + (c0 >> 1), pk);
+          }
+        } else {
+#pragma unroll 1
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t ra[32];
+            XKV_TMEM_LD32(colS + c0, ra);
+            tc_wait_ld();
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              float p0 = fast_exp2(fmaf(__uint_as_float(ra[2 * i]), a.scale_log2, -m_ref));
+              float p1 = fast_exp2(fmaf(__uint_as_float(ra[2 * i + 1]), a.scale_log2, -m_ref));
+              if (c0 + 2 * i >= lim) p0 = 0.f;
+              if (c0 + 2 * i + 1 >= lim) p1 = 0.f;
+              l2 = add_f2(l2, pack_f2(p0, p1));
+              pk[i] = kBf16 ? pack_bf2(p0, p1) : pack_h2(p0, p1);
+            }
+            XKV_TMEM_ST16(colP + (c0 >> 1), pk);
+          }
+        }
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(pfull);
+      }
+      // ---- epilogue of the segment ----
+      mbar_wait(pvdone, (cnt - 1) & 1, wc);
+      __syncwarp();
+      tc_fence_after();
+      const float l = f2_lo(l2) + f2_hi(l2);
+      const bool whole = (tile_lo == 0 && nt == a.n_tiles);
+      if (whole) {
+        const float inv_l = 1.f / l;
+#pragma unroll 1
+        for (int c0 = 0; c0 < 64; c0 += 32) {
+          uint32_t ra[32];
+          XKV_TMEM_LD32(colO + c0, ra);
+          tc_wait_ld();
+          if (row < a.n) {
+            __nv_bfloat16* op = a.out + (int64_t)h * a.hs + (int64_t)row * a.ts + c0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              uint32_t o[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                o[i] = pack_bf2(__uint_as_float(ra[8 * c + 2 * i]) * inv_l, __uint_as_float(ra[8 * c + 2 * i + 1]) * inv_l);
+              *reinterpret_cast<uint4*>(op + 8 * c) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+          }
+        }
+      } else {
+        const size_t slot = (size_t)2 * blockIdx.x + (seg_idx == 0 ? 0 : 1);
+        const size_t prow = (slot * 2 + t) * 128 + r;
+#pragma unroll 1
+        for (int c0 = 0; c0 < 64; c0 += 32) {
+          uint32_t ra[32];
+          XKV_TMEM_LD32(colO + c0, ra);
+          tc_wait_ld();
           float4* dst = reinterpret_cast<float4*>(a.part_o + prow * 64 + c0);
 #pragma unroll
           for (int c = 0; c < 8; ++c)
-            dst[c] = make_float4(__uint_as_float(r[4 * c]), __uint_as_float(r[4 * c + 1]),
-                                 __uint_as_float(r[4 * c + 2]), __uint_as_float(r[4 * c + 3]));
+            dst[c] = make_float4(__uint_as_float(ra[4 * c]), __uint_as_float(ra[4 * c + 1]),
+                                 __uint_as_float(ra[4 * c + 2]), __uint_as_float(ra[4 * c + 3]));
         }
+        a.part_ml[prow] = make_float2(m_ref, l);
       }
-      if (row < a.n) a.part_ml[prow] = make_float2(m_ref, l);
+      tc_fence_before();
     }
-    tc_fence_before();
-  } else if (warp < 8) {
+  } else if (warp < 12) {
     // =========================== operand producers ===========================
-    const int t = tid - 128;
+    const int t = tid - 256;
     const int w = t & 7;          // 16-byte chunk = 8 channels
     const int kb = t >> 3;        // keys kb + 16 i
     const uint32_t row_off = (uint32_t)((kb >> 3) * 1024 + (kb & 7) * 128 + ((w ^ (kb & 7)) << 4));
-    const size_t head_slot = (size_t)h * a.cap;
-    for (int jj = 0; jj < nt; ++jj) {
-      const int tile = tile_lo + jj;
-      const int b = jj & 1, u = jj >> 1;
-      const int p0 = tile * 128 + kb;
-      // ---- keys ----
-      mbar_wait(b_kfree + 8 * b, (u & 1) ^ 1, wc);
-      if (BITS == 4) {
-        uint32_t wd[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-          wd[i] = __ldg(reinterpret_cast<const uint32_t*>(a.k + (head_slot + p0 + 16 * i) * 32 + 4 * w));
-#pragma unroll
-        for (int g = 0; g < 2; ++g) {
-          const float2* par = a.kpar + ((size_t)h * (a.cap >> 6) + (tile * 2 + g)) * 64 + 8 * w;
-          uint32_t s2[4], zo[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 p_a = __ldg(par + 2 * i), p_b = __ldg(par + 2 * i + 1);
-            const float off = (i & 1) ? 64.f : 1024.f;
-            s2[i] = pack_h2(p_a.x, p_b.x);
-            zo[i] = pack_h2(off + p_a.y, off + p_b.y);
+    uint32_t g = 0;               // steps so far (ring positions)
+    for (long long pos = step_lo; pos < step_hi;) {
+      const int item = (int)(pos / a.n_tiles);
+      const int tile_lo = (int)(pos - (long long)item * a.n_tiles);
+      const int nt = (int)min((long long)(a.n_tiles - tile_lo), step_hi - pos);
+      pos += nt;
+      for (int jj = 0; jj < nt; ++jj, ++g) {
+        const uint32_t rs = g % C::kNR, ru = g / C::kNR;
+        const uint32_t kbuf = g % kNK, ku = g / kNK;
+        const uint32_t vbuf = g % kNV, vu = g / kNV;
+        const uint8_t* raw = sgen + kOffRaw + rs * C::kRawStage;
+        mbar_wait(b_rfull + 8 * rs, ru & 1, wc);
+        if (BITS == 4) {
+          // ---- fp16 parameter tables of this tile (one (group, channel) and one key per thread) ----
+          uint8_t* tab = sgen + kOffTab + (g & 1) * kTabBytes;
+          {
+            const float2 kp = *reinterpret_cast<const float2*>(raw + C::kRawK + C::kRawV + 8 * t);  // (group t>>6, channel t&63)
+            const int c = t & 63;
+            const float off = (((c & 7) >> 1) & 1) ? 64.f : 1024.f;
+            __half* ks = reinterpret_cast<__half*>(tab);              // [2][64] scales, then [2][64] offsets
+            ks[t] = __float2half_rn(kp.x);
+            ks[128 + t] = __float2half_rn(off + kp.y);
+            const float2 vp = *reinterpret_cast<const float2*>(raw + C::kRawK + C::kRawV + C::kRawKP + 8 * t);   // key t
+            const uint32_t s1 = pack_h2(vp.x, vp.x);
+            const uint32_t zl = pack_h2(1024.f + vp.y, 1024.f + vp.y);
+            const uint32_t zh = pack_h2(64.f + vp.y, 64.f + vp.y);
+            *reinterpret_cast<uint4*>(tab + 512 + 16 * t) = make_uint4(s1, zl, zh, 0u);
           }
+          producer_sync();
+          // ---- keys ----
+          uint32_t wd[8];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint4 o = dequant_word_h(wd[4 * g + i], s2, zo);
-            *reinterpret_cast<uint4*>(sgen + kOffK + b * 16384 + row_off + (4 * g + i) * 2048) = o;
+          for (int i = 0; i < 8; ++i) wd[i] = *reinterpret_cast<const uint32_t*>(raw + (kb + 16 * i) * 32 + 4 * w);
+          mbar_wait(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
+#pragma unroll
+          for (int grp = 0; grp < 2; ++grp) {
+            const uint4 sv = *reinterpret_cast<const uint4*>(tab + grp * 128 + 16 * w);
+            const uint4 zv = *reinterpret_cast<const uint4*>(tab + 256 + grp * 128 + 16 * w);
+            const uint32_t s2[4] = {sv.x, sv.y, sv.z, sv.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint4 o = dequant_word_h(wd[4 * grp + i], s2, zo);
+              *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (4 * grp + i) * 2048) = o;
+            }
           }
-        }
-      } else {
+          fence_proxy_async();
+          mbar_arrive(b_kfull + 8 * kbuf);
+          // ---- values ----
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const uint4 o = __ldg(reinterpret_cast<const uint4*>(a.k + (head_slot + p0 + 16 * i) * 128 + 16 * w));
-          *reinterpret_cast<uint4*>(sgen + kOffK + b * 16384 + row_off + i * 2048) = o;
+          for (int i = 0; i < 8; ++i) wd[i] = *reinterpret_cast<const uint32_t*>(raw + C::kRawK + (kb + 16 * i) * 32 + 4 * w);
+          mbar_arrive(b_rfree + 8 * rs);     // everything this thread needs of the raw stage is in registers or tables
+          mbar_wait(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint4 pv = *reinterpret_cast<const uint4*>(tab + 512 + 16 * (kb + 16 * i));
+            const uint32_t s2[4] = {pv.x, pv.x, pv.x, pv.x}, zo[4] = {pv.y, pv.z, pv.y, pv.z};
+            const uint4 o = dequant_word_h(wd[i], s2, zo);
+            *reinterpret_cast<uint4*>(sgen + kOffV + vbuf * 16384 + row_off + i * 2048) = o;
+          }
+          fence_proxy_async();
+          mbar_arrive(b_vfull + 8 * vbuf);
+        } else {
+          uint4 rowk[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) rowk[i] = *reinterpret_cast<const uint4*>(raw + (kb + 16 * i) * 128 + 16 * w);
+          mbar_wait(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + i * 2048) = rowk[i];
+          fence_proxy_async();
+          mbar_arrive(b_kfull + 8 * kbuf);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) rowk[i] = *reinterpret_cast<const uint4*>(raw + C::kRawK + (kb + 16 * i) * 128 + 16 * w);
+          mbar_arrive(b_rfree + 8 * rs);
+          mbar_wait(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            *reinterpret_cast<uint4*>(sgen + kOffV + vbuf * 16384 + row_off + i * 2048) = rowk[i];
+          fence_proxy_async();
+          mbar_arrive(b_vfull + 8 * vbuf);
         }
       }
-      fence_proxy_async();
-      mbar_arrive(b_kfull + 8 * b);
-      // ---- values ----
-      mbar_wait(b_vfree + 8 * b, (u & 1) ^ 1, wc);
-      if (BITS == 4) {
-        uint32_t wd[8];
-        float2 vp[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          wd[i] = __ldg(reinterpret_cast<const uint32_t*>(a.v + (head_slot + p0 + 16 * i) * 32 + 4 * w));
-          vp[i] = __ldg(a.vpar + head_slot + p0 + 16 * i);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const uint32_t s1 = pack_h2(vp[i].x, vp[i].x);
-          const uint32_t z_lo = pack_h2(1024.f + vp[i].y, 1024.f + vp[i].y);
-          const uint32_t z_hi = pack_h2(64.f + vp[i].y, 64.f + vp[i].y);
-          const uint32_t s2[4] = {s1, s1, s1, s1}, zo[4] = {z_lo, z_hi, z_lo, z_hi};
-          const uint4 o = dequant_word_h(wd[i], s2, zo);
-          *reinterpret_cast<uint4*>(sgen + kOffV + b * 16384 + row_off + i * 2048) = o;
-        }
-      } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const uint4 o = __ldg(reinterpret_cast<const uint4*>(a.v + (head_slot + p0 + 16 * i) * 128 + 16 * w));
-          *reinterpret_cast<uint4*>(sgen + kOffV + b * 16384 + row_off + i * 2048) = o;
-        }
-      }
-      fence_proxy_async();
-      mbar_arrive(b_vfull + 8 * b);
     }
-  } else if (tid == 256) {
+  } else if (tid == 384) {
     // =========================== MMA issuer ===================================
     const uint32_t idesc_qk = make_idesc(128, kBf16, false);
     const uint32_t idesc_pv = make_idesc(64, kBf16, true);
-    const uint64_t dq = make_desc(sQ);
-    auto issue_pv = [&](int t) {
-      const int b = t & 1, u = t >> 1;
-      mbar_wait(b_vfull + 8 * b, u & 1, wc);
-      mbar_wait(b_pfull, t & 1, wc);
-      tc_fence_after();
-      const uint64_t dv = make_desc(sV + b * 16384);
+    uint32_t g = 0;
+    uint32_t cnt[2] = {0, 0}, segq[2] = {0, 0};
+    for (long long pos = step_lo; pos < step_hi;) {
+      const int item = (int)(pos / a.n_tiles);
+      const int tile_lo = (int)(pos - (long long)item * a.n_tiles);
+      const int nt = (int)min((long long)(a.n_tiles - tile_lo), step_hi - pos);
+      pos += nt;
+      const int pair = item % a.n_pairs;
+      const int ntile = (2 * pair + 1 < a.q_tiles) ? 2 : 1;
+      auto issue_pv = [&](int t, uint32_t gv, bool first_of_segment) {
+        const uint64_t dv = make_desc(sV + (gv % kNV) * 16384);
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks)   // 16 keys per step: 2 swizzle atoms = 2048 B of V~, 8 columns of P
-        mma_ts(tmem + kColO, tmem + kColP + 8 * ks, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv,
-               (t > 0 || ks > 0) ? 1u : 0u);
-      tc_commit(b_vfree + 8 * b);
-      tc_commit(b_pvdone);
-    };
-    for (int jj = 0; jj < nt; ++jj) {
-      const int b = jj & 1, u = jj >> 1;
-      mbar_wait(b_kfull + 8 * b, u & 1, wc);
-      mbar_wait(b_sfree, (jj & 1) ^ 1, wc);
-      tc_fence_after();
-      const uint64_t dk = make_desc(sK + b * 16384);
+        for (int ks = 0; ks < 8; ++ks)   // 16 keys per step: 2 swizzle atoms = 2048 B of V~, 8 columns of P
+          mma_ts(tmem + kColO + 64 * t, tmem + kColP + 64 * t + 8 * ks, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv,
+                 (!first_of_segment || ks > 0) ? 1u : 0u);
+        tc_commit(b_pvdone + 8 * t);
+      };
+      for (int jj = 0; jj < nt; ++jj, ++g) {
+        mbar_wait(b_kfull + 8 * (g % kNK), (g / kNK) & 1, wc);
+        const uint64_t dk = make_desc(sK + (g % kNK) * 16384);
+        for (int t = 0; t < ntile; ++t) {
+          if (jj == 0) mbar_wait(b_qfull + 8 * t, segq[t] & 1, wc);
+          else mbar_wait(b_pfull + 8 * t, (cnt[t] - 1) & 1, wc);   // S_t read, P_t of the previous step written
+          tc_fence_after();
+          const uint64_t dq = make_desc(sQ + t * 16384);
 #pragma unroll
-      for (int ks = 0; ks < 4; ++ks)   // 16 channels per step: 32 B inside the swizzle span
-        mma_ss(tmem + kColS, dq + (uint64_t)(ks * 2), dk + (uint64_t)(ks * 2), idesc_qk, ks > 0 ? 1u : 0u);
-      tc_commit(b_kfree + 8 * b);
-      tc_commit(b_sfull);
-      if (jj > 0) issue_pv(jj - 1);
+          for (int ks = 0; ks < 4; ++ks)   // 16 channels per step: 32 B inside the swizzle span
+            mma_ss(tmem + kColS + 128 * t, dq + (uint64_t)(ks * 2), dk + (uint64_t)(ks * 2), idesc_qk, ks > 0 ? 1u : 0u);
+          tc_commit(b_sfull + 8 * t);
+          if (jj > 0) {
+            if (t == 0) { mbar_wait(b_vfull + 8 * ((g - 1) % kNV), ((g - 1) / kNV) & 1, wc); tc_fence_after(); }
+            issue_pv(t, g - 1, jj == 1);
+          }
+          ++cnt[t];
+        }
+        tc_commit(b_kfree + 8 * (g % kNK));
+        if (jj > 0) tc_commit(b_vfree + 8 * ((g - 1) % kNV));
+      }
+      // the last PV of the segment
+      for (int t = 0; t < ntile; ++t) {
+        mbar_wait(b_pfull + 8 * t, (cnt[t] - 1) & 1, wc);
+        if (t == 0) mbar_wait(b_vfull + 8 * ((g - 1) % kNV), ((g - 1) / kNV) & 1, wc);
+        tc_fence_after();
+        issue_pv(t, g - 1, nt == 1);
+        ++segq[t];
+      }
+      tc_commit(b_vfree + 8 * ((g - 1) % kNV));
     }
-    issue_pv(nt - 1);
-    // wait until the last MMAs are done before the CTA may free tensor memory
-    mbar_wait(b_pvdone, (nt - 1) & 1, wc);
+    // all MMAs must be done before the CTA may free tensor memory: the softmax warps have waited
+    // for every PV (pvdone) before their epilogues, and every QK (sfull) before that.
     tc_fence_before();
+  } else if (tid == 416) {
+    // =========================== TMA loader ===================================
+    uint32_t g = 0;
+    for (long long pos = step_lo; pos < step_hi;) {
+      const int item = (int)(pos / a.n_tiles);
+      const int tile_lo = (int)(pos - (long long)item * a.n_tiles);
+      const int nt = (int)min((long long)(a.n_tiles - tile_lo), step_hi - pos);
+      pos += nt;
+      const int h = item / a.n_pairs;
+      const size_t head_slot = (size_t)h * a.cap;
+      for (int jj = 0; jj < nt; ++jj, ++g) {
+        const int tile = tile_lo + jj;
+        const uint32_t rs = g % C::kNR, ru = g / C::kNR;
+        mbar_wait(b_rfree + 8 * rs, (ru & 1) ^ 1, wc);
+        const uint32_t dst = sRaw + rs * C::kRawStage, bar = b_rfull + 8 * rs;
+        mbar_expect_tx(bar, C::kRawStage);
+        const size_t slot0 = head_slot + (size_t)tile * 128;
+        if (BITS == 4) {
+          tma_load_1d(dst, a.k + slot0 * 32, C::kRawK, bar);
+          tma_load_1d(dst + C::kRawK, a.v + slot0 * 32, C::kRawV, bar);
+          tma_load_1d(dst + C::kRawK + C::kRawV, a.kpar + ((size_t)h * (a.cap >> 6) + 2 * tile) * 64, C::kRawKP, bar);
+          tma_load_1d(dst + C::kRawK + C::kRawV + C::kRawKP, a.vpar + slot0, C::kRawVP, bar);
+        } else {
+          tma_load_1d(dst, a.k + slot0 * 128, C::kRawK, bar);
+          tma_load_1d(dst + C::kRawK, a.v + slot0 * 128, C::kRawV, bar);
+        }
+      }
+    }
+    // Drain: every copy this thread started has landed once the last use of each stage completed
+    // (bounded, and not cut short by the abort flag, so that nothing is in flight at exit).
+    const uint32_t issued = g;
+    for (uint32_t i = 0; i < (uint32_t)C::kNR && i < issued; ++i) {
+      const uint32_t gi = issued - 1 - i;
+      const uint32_t rs = gi % C::kNR, ru = gi / C::kNR;
+      for (uint32_t it = 0; it < kSpinLimit; ++it)
+        if (mbar_try(b_rfull + 8 * rs, ru & 1)) break;
+    }
   }
   __syncthreads();
-  if (warp == 8) {
+  if (warp == 13) {
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -584,64 +731,61 @@ __global__ void __launch_bounds__(kThreads, 2) attn_tc_kernel(const Args a) {
 }
 
 // ---------------------------------------------------------------------------
-// Split-KV combine: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.
-// Thread = (head, row, 8-channel chunk).
+// Merge of the partial results of the items that were cut between CTAs:
+// out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  Thread = (item, query
+// tile, row, 8-channel chunk); items that one CTA covered alone were written by it.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-attn_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, int n_splits, int H,
-                    int n, __nv_bfloat16* __restrict__ out, int64_t ts, int64_t hs) {
-  const long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const int ch = (int)(g & 7);
-  const long long hr = g >> 3;
-  if (hr >= (long long)H * n) return;
+attn_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, int grid, long long total,
+                    int n_tiles, int n_pairs, int q_tiles, int n, __nv_bfloat16* __restrict__ out, int64_t ts,
+                    int64_t hs) {
+  const long long gidx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int ch = (int)(gidx & 7);
+  const int r = (int)((gidx >> 3) & 127);
+  const int t = (int)((gidx >> 10) & 1);
+  const long long item = gidx >> 11;
+  if (item * n_tiles >= total) return;
+  const int h = (int)(item / n_pairs), pair = (int)(item - (long long)h * n_pairs);
+  const int qt = 2 * pair + t;
+  const int row = qt * 128 + r;
+  if (qt >= q_tiles || row >= n) return;
+  const long long lo = item * n_tiles, hi = lo + n_tiles;
+  // CTA that holds step x: the largest b with piece_start(b) <= x
+  const int b_first = (int)(((lo + 1) * grid - 1) / total);
+  const int b_last = (int)((hi * grid - 1) / total);
+  if (b_first == b_last) return;                 // one CTA covered the whole item and wrote the result
   float m = -INFINITY;
-  for (int s = 0; s < n_splits; ++s) m = fmaxf(m, part_ml[(size_t)s * H * n + hr].x);
+  for (int b = b_first; b <= b_last; ++b) {
+    const size_t slot = (size_t)2 * b + (piece_start(total, grid, b) >= lo ? 0 : 1);
+    m = fmaxf(m, part_ml[(slot * 2 + t) * 128 + r].x);
+  }
   float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   float l = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    const float2 ml = part_ml[(size_t)s * H * n + hr];
+  for (int b = b_first; b <= b_last; ++b) {
+    const size_t slot = (size_t)2 * b + (piece_start(total, grid, b) >= lo ? 0 : 1);
+    const size_t prow = (slot * 2 + t) * 128 + r;
+    const float2 ml = part_ml[prow];
     const float wgt = exp2f(ml.x - m);
     l += wgt * ml.y;
-    const float4* po = reinterpret_cast<const float4*>(part_o + ((size_t)s * H * n + hr) * 64 + 8 * ch);
+    const float4* po = reinterpret_cast<const float4*>(part_o + prow * 64 + 8 * ch);
     const float4 x = po[0], y = po[1];
     acc[0] += wgt * x.x; acc[1] += wgt * x.y; acc[2] += wgt * x.z; acc[3] += wgt * x.w;
     acc[4] += wgt * y.x; acc[5] += wgt * y.y; acc[6] += wgt * y.z; acc[7] += wgt * y.w;
   }
   const float inv = 1.f / l;
-  const int h = (int)(hr / n), row = (int)(hr % n);
   uint32_t o[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) o[i] = pack_bf2(acc[2 * i] * inv, acc[2 * i + 1] * inv);
   *reinterpret_cast<uint4*>(out + (int64_t)h * hs + (int64_t)row * ts + 8 * ch) = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-size_t attn_tc_scratch_bytes(const xkv_params* p) {
-  const size_t rows = (size_t)kMaxSplits * p->n_heads * p->max_frame_tokens;
-  return rows * 64 * sizeof(float) + rows * sizeof(float2) + 512;
-}
+size_t attn_tc_scratch_bytes(const xkv_params*) { return (size_t)2 * kMaxGrid * kSlotBytes + 512; }
 
-// Splits are chosen so that the grid fills whole waves of (SMs x 2 resident CTAs).
-static int choose_splits(int items, int n_tiles, int slots) {
-  int best = 1;
-  double best_eff = 0.0;
-  for (int s = 1; s <= kMaxSplits; ++s) {
-    const int tps = (n_tiles + s - 1) / s;
-    if (tps < 2 && s > 1) break;
-    if ((s - 1) * tps >= n_tiles) continue;      // an empty split
-    const long long ctas = (long long)items * s;
-    const long long waves = (ctas + slots - 1) / slots;
-    const double eff = (double)ctas / (double)(waves * slots) * ((double)n_tiles / (double)(tps * s));
-    if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
-  }
-  return best;
-}
-
-// `part` holds the split-KV partials: accumulators float [rows_cap][64], then (max, sum) float2
-// [rows_cap].  rows_cap = 0 means "as many rows as this launch needs" and `part_bytes` is then the
-// room available: when it does not suffice nothing is launched and cudaErrorMemoryAllocation returns.
+// `part` holds the partial slots: accumulators float [slots][2][128][64], then (max, sum) float2
+// [slots][2][128], slots = part_bytes / kSlotBytes.  The grid is the SM count, capped by the slots
+// available (two per CTA) and by the number of steps.
 static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
-                                     float scale, float* part, size_t rows_cap, size_t part_bytes,
-                                     cudaStream_t st) {
+                                     float scale, float* part, size_t part_bytes, cudaStream_t st) {
   static int sm_count = 0;
   static bool attr_set = false;
   if (!attr_set) {
@@ -650,9 +794,9 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(attn_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(attn_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<16>());
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -662,47 +806,46 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
   a.n = n; a.ts = ts; a.hs = hs;
   const BufSet& b = c->buf[c->cur];
   a.k = b.k; a.kpar = b.kpar; a.v = b.v; a.vpar = b.vpar;
-  a.cap = c->cap; a.t_first = c->T_first; a.rest_base = c->rest_base;
+  a.cap = c->cap; a.t_first = c->T_first;
   a.t_phys = c->rest_base + (c->T - c->T_first);
   if (c->T == c->T_first) a.t_phys = c->T_first;          // only the first frame: no pad tile beyond it
   a.scale_log2 = scale * 1.4426950408889634f;
   a.n_tiles = (a.t_phys + 127) / 128;
-  const int q_tiles = (n + kQRows - 1) / kQRows;
+  a.q_tiles = (n + kQRows - 1) / kQRows;
+  a.n_pairs = (a.q_tiles + 1) / 2;
   const int H = c->p.n_heads;
-  a.n_splits = choose_splits(q_tiles * H, a.n_tiles, sm_count * 2);
-  a.tiles_per_split = (a.n_tiles + a.n_splits - 1) / a.n_splits;
-  size_t rows = rows_cap;
-  if (rows == 0) {
-    rows = (size_t)a.n_splits * H * n;
-    if (a.n_splits > 1 && rows * (64 * sizeof(float) + sizeof(float2)) > part_bytes) return cudaErrorMemoryAllocation;
-  }
+  a.total = (long long)H * a.n_pairs * a.n_tiles;
+  const size_t slots = part_bytes / kSlotBytes;
+  long long grid = sm_count;
+  if (grid > (long long)(slots / 2)) grid = (long long)(slots / 2);
+  if (grid > a.total) grid = a.total;
+  if (grid < 1) return cudaErrorMemoryAllocation;
   a.part_o = part;
-  a.part_ml = reinterpret_cast<float2*>(part + rows * 64);
+  a.part_ml = reinterpret_cast<float2*>(part + slots * kSlotFloats);
   a.status = c->status;
-  const dim3 grid(q_tiles, H, a.n_splits);
   {
     LaunchScope ls(c, XKV_PROF_ATTN, st);
-    if (c->p.kv_bits == 16) attn_tc_kernel<16><<<grid, kThreads, kSmemBytes, st>>>(a);
-    else attn_tc_kernel<4><<<grid, kThreads, kSmemBytes, st>>>(a);
+    if (c->p.kv_bits == 16) attn_tc_kernel<16><<<(int)grid, kThreads, smem_bytes<16>(), st>>>(a);
+    else attn_tc_kernel<4><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
-  if (a.n_splits > 1) {
+  {
     LaunchScope ls(c, XKV_PROF_COMBINE, st);
-    const long long threads = (long long)H * n * 8;
-    attn_combine_kernel<<<(int)((threads + 255) / 256), 256, 0, st>>>(a.part_o, a.part_ml, a.n_splits, H, n, a.out, ts, hs);
+    const long long threads = (long long)H * a.n_pairs * 2048;
+    attn_combine_kernel<<<(int)((threads + 255) / 256), 256, 0, st>>>(a.part_o, a.part_ml, (int)grid, a.total,
+                                                                      a.n_tiles, a.n_pairs, a.q_tiles, n, a.out, ts, hs);
   }
   return cudaGetLastError();
 }
 
 cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs, float scale,
                            cudaStream_t st) {
-  return launch_attn_tc_on(c, q, out, n, ts, hs, scale, c->attn_part,
-                           (size_t)kMaxSplits * c->p.n_heads * c->p.max_frame_tokens, c->attn_part_bytes, st);
+  return launch_attn_tc_on(c, q, out, n, ts, hs, scale, c->attn_part, c->attn_part_bytes, st);
 }
 
 // ---------------------------------------------------------------------------
-// attn_packed_causal_static: the same attention with its split-KV partials in a
+// attn_packed_causal_static: the same attention with its partial slots in a
 // fixed array that is part of the loaded library image instead of the caller's
 // workspace.  See xkv.h for who needs this and for the rules of use.
 // ---------------------------------------------------------------------------
@@ -724,13 +867,13 @@ cudaError_t launch_attn_tc_static(xkv_cache* c, const void* q, void* out, int n,
     std::lock_guard<std::mutex> lock(g_static_mutex);
     if (!g_static_addr[dev]) {
       void* p = nullptr;
-      e = cudaGetSymbolAddress(&p, g_static_partials);
+      e = cudaGetSymbolAddress((void**)&p, g_static_partials);
       if (e != cudaSuccess) return e;
       g_static_addr[dev] = p;
     }
     addr = g_static_addr[dev];
   }
-  return launch_attn_tc_on(c, q, out, n, ts, hs, scale, reinterpret_cast<float*>(addr), 0,
+  return launch_attn_tc_on(c, q, out, n, ts, hs, scale, reinterpret_cast<float*>(addr),
                            (size_t)XKV_STATIC_SCRATCH_BYTES, st);
 }
 

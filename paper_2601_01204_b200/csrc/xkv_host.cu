@@ -365,6 +365,13 @@ int64_t xkv_debug_export(const xkv_cache* c, int32_t which, void* host_dst, size
   return (int64_t)nbytes;
 }
 
+int xkv_debug_rewind_attention(xkv_cache* c) {
+  if (!c) return XKV_E_INVALID;
+  if (c->stage != 0 || c->frames < 1) return XKV_E_STATE;
+  c->stage = 3;
+  return XKV_OK;
+}
+
 int xkv_poll_status(const xkv_cache* c, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;
   if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;

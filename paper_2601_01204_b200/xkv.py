@@ -33,6 +33,7 @@ EXPORTED = [
     "kv_quant_pack", "attn_packed_causal", "xkv_stream_step", "xkv_stream_step_host_bytes",
     "xkv_stream_step_host", "xkv_get_info", "xkv_debug_export", "xkv_poll_status", "xkv_strerror",
     "xkv_synth_fill", "xkv_profile_enable", "xkv_profile_read", "attn_packed_causal_static",
+    "xkv_debug_rewind_attention",
 ]
 PROF_NAMES = ["append", "pool_q", "score", "select", "regroup_k", "gather", "attn", "attn_combine"]
 
@@ -87,6 +88,8 @@ lib.xkv_get_info.restype = C.c_int
 lib.xkv_get_info.argtypes = [_vp, C.POINTER(xkv_info)]
 lib.xkv_debug_export.restype = _i64
 lib.xkv_debug_export.argtypes = [_vp, _i32, _vp, _sz, _vp]
+lib.xkv_debug_rewind_attention.restype = C.c_int
+lib.xkv_debug_rewind_attention.argtypes = [_vp]
 lib.xkv_poll_status.restype = C.c_int
 lib.xkv_poll_status.argtypes = [_vp, _vp]
 lib.xkv_strerror.restype = C.c_char_p
@@ -193,9 +196,9 @@ class Cache:
         return out
 
     def attn_packed_causal_static(self, q, out=None, scale: float | None = None):
-        """attn_packed_causal with the split-KV partials in the library's fixed device array
-        (for callers that may not allocate; XKV_E_LIMIT when the launch needs more than
-        STATIC_SCRATCH_BYTES)."""
+        """attn_packed_causal with the partial results in the library's fixed device array
+        (for callers that may not allocate; may run with fewer thread blocks than the GPU has
+        multiprocessors)."""
         import torch
         if out is None:
             out = torch.empty_like(q)
@@ -225,6 +228,9 @@ class Cache:
         pr = xkv_profile()
         _check(lib.xkv_profile_read(self.handle, C.byref(pr), _stream()), "xkv_profile_read")
         return {name: (pr.ms[i], pr.launches[i]) for i, name in enumerate(PROF_NAMES)}
+
+    def xkv_debug_rewind_attention(self) -> None:
+        _check(lib.xkv_debug_rewind_attention(self.handle), "xkv_debug_rewind_attention")
 
     def xkv_poll_status(self) -> int:
         return int(lib.xkv_poll_status(self.handle, _stream()))

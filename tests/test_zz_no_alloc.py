@@ -4,9 +4,9 @@ Some users of the library run where cudaMalloc is forbidden (a host that bans
 allocation after start-up, a plug-in without its own allocator).  For them the
 library offers attention with the split-KV partials in a fixed device array
 that belongs to the library image.  This file checks, through the C ABI, that
-the variant returns what attn_packed_causal returns, on two frames in a row
-(the array is shared and keeps the previous call's contents), and that a launch
-that would not fit is refused cleanly.
+the variant returns what attn_packed_causal returns, on several frames in a row
+(the array is shared and keeps the previous call's contents), also when it has
+to run with fewer thread blocks than the GPU has multiprocessors.
 
 The file name sorts last on purpose: a run that stops at the first failure has
 then already executed every other test.
@@ -61,24 +61,26 @@ def test_static_scratch_attention_matches_workspace_attention(xkv):
     assert checked >= 2 and sta_cache.xkv_get_info().T == 1024
 
 
-def test_static_scratch_limit_is_enforced(xkv):
-    """A frame whose partials exceed the fixed array is refused and can still be served the usual way."""
+def test_static_scratch_attention_larger_frames(xkv):
+    """Frames of several query-tile pairs and many heads: the fixed array must still do (its size
+    does not depend on the frame), with fewer thread blocks than the workspace variant may use."""
     import torch
-    H, n, d = 64, 2048, 64                       # up to 6 * 64 * 2048 * 264 B = 198 MiB of partials
-    p = xkv.Params(n_heads=H, budget=8192, max_frame_tokens=n, kv_bits=4)
-    cache = xkv.Cache(p)
-    q = torch.zeros(H, n, d, dtype=torch.bfloat16, device="cuda")
-    refused = False
-    for t in range(3):
-        cache.kv_append(q, q)
-        cache.kv_score_evict(q)
-        cache.kv_quant_pack()
-        try:
-            cache.attn_packed_causal_static(q)
-        except xkv.XkvError as e:
-            assert e.status == xkv.XKV_E_LIMIT
-            assert cache.xkv_get_info().stage == 3
-            cache.attn_packed_causal(q)
-            refused = True
-    assert refused
-    assert cache.xkv_poll_status() == 0
+    H, n, d = 24, 700, 64
+    p = xkv.Params(n_heads=H, budget=2048, max_frame_tokens=n, kv_bits=4)
+    ref_cache, sta_cache = xkv.Cache(p), xkv.Cache(p)
+    for t, (qb, kb, vb) in enumerate(_frames(32, 4, H, n, d)):
+        q, k, v = (to_device_bf16(x) for x in (qb, kb, vb))
+        outs = []
+        for cache, static in ((ref_cache, False), (sta_cache, True)):
+            cache.kv_append(k, v)
+            cache.kv_score_evict(q)
+            cache.kv_quant_pack()
+            out = torch.full_like(q, float("nan"))
+            if static:
+                cache.attn_packed_causal_static(q, out)
+            else:
+                cache.attn_packed_causal(q, out)
+            assert cache.xkv_poll_status() == 0
+            outs.append(bf16_tensor_to_f32(out))
+        maxabs, rell2 = attn_errors(outs[1], outs[0])
+        assert maxabs <= ATTN_MAXABS and rell2 <= ATTN_RELL2, (t, maxabs, rell2)

@@ -596,7 +596,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           // ---- values ----
 #pragma unroll
           for (int i = 0; i < 8; ++i) wd[i] = *reinterpret_cast<const uint32_t*>(raw + C::kRawK + (kb + 16 * i) * 32 + 4 * w);
-          mbar_arrive(b_rfree + 8 * rs);     // everything this thread needs of the raw stage is in registers or tables
           mbar_wait(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
@@ -607,6 +606,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           }
           fence_proxy_async();
           mbar_arrive(b_vfull + 8 * vbuf);
+          // The raw stage is released only here, after the words read from it have been used and
+          // the fence above: released right after the loads, the refill of the stage was observed
+          // to reach some of those loads when the wait in between was long.
+          mbar_arrive(b_rfree + 8 * rs);
         } else {
           uint4 rowk[8];
 #pragma unroll
@@ -619,13 +622,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           mbar_arrive(b_kfull + 8 * kbuf);
 #pragma unroll
           for (int i = 0; i < 8; ++i) rowk[i] = *reinterpret_cast<const uint4*>(raw + C::kRawK + (kb + 16 * i) * 128 + 16 * w);
-          mbar_arrive(b_rfree + 8 * rs);
           mbar_wait(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
 #pragma unroll
           for (int i = 0; i < 8; ++i)
             *reinterpret_cast<uint4*>(sgen + kOffV + vbuf * 16384 + row_off + i * 2048) = rowk[i];
           fence_proxy_async();
           mbar_arrive(b_vfull + 8 * vbuf);
+          mbar_arrive(b_rfree + 8 * rs);
         }
       }
     }

@@ -8,11 +8,11 @@
 // not cover an item completely leaves partial results (accumulator, running max
 // and sum) in a scratch slot; a second kernel merges them.
 //
-// One CTA, 14 warps:
+// One CTA, 15 warps:
 //   warps 0-3   softmax of query tile 0: thread r owns query row r = TMEM lane r.
 //               Reads S from tensor memory, online max/sum, writes P (16-bit) back
 //               to tensor memory, rescales O only when the running maximum grew by
-//               more than 2^8, epilogue.
+//               more than 2^14, epilogue.
 //   warps 4-7   the same for query tile 1.  The two groups alternate naturally:
 //               while one computes exponentials the tensor pipe produces the
 //               other's scores.
@@ -20,8 +20,10 @@
 //               fp16 K~ (per channel and 64-slot group) and V~ (per token) in the
 //               128-byte-swizzled layouts the MMA descriptors expect.  One
 //               dequantised tile serves both query tiles.
-//   warp 12     one thread issues the MMAs: S_t = Q_t K~^T (M128 N128 K64) and
-//               O_t += P_t V~ (M128 N64 K128, A = P from tensor memory).
+//   warps 12,14 one thread each issues the MMAs of query tile 0 resp. 1:
+//               S_t = Q_t K~^T (M128 N128 K64) and O_t += P_t V~ (M128 N64 K128,
+//               A = P from tensor memory).  A single issuing thread for both tiles
+//               was the bottleneck of the CTA.
 //   warp 13     one thread issues the bulk copies of the raw tiles, several steps
 //               ahead; the warp owns the tensor-memory allocation (all 512 columns).
 // 4-bit caches multiply in fp16 (the dequantised keys are not bf16-representable:
@@ -41,10 +43,15 @@ namespace xkv {
 namespace {
 
 constexpr int kMaxDevices = 64;
-constexpr int kThreads = 448;
+constexpr int kThreads = 480;
 constexpr int kQRows = 128;
 constexpr int kMaxGrid = 160;                 // CTAs the scratch is sized for (>= SM count of the part)
 constexpr uint32_t kSpinLimit = 1u << 22;
+// The reference maximum of a row moves only when the row maximum exceeds it by more than 2^kGrow
+// (log2 units).  Until then exponentials reach at most 2^14 = 16384, inside the fp16 range; the
+// decision is taken per warp, so a low threshold would make some row of the 32 trip it at every
+// few tiles.
+constexpr float kGrow = 14.f;
 
 // ring depths
 constexpr int kNK = 3;                        // dequantised K~ tiles
@@ -127,6 +134,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // per-CTA flag); once the flag is up every later wait of the CTA gives up at once.
 struct WaitCtx { int* status; volatile int* abort_flag; };
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc) {
+  if (mbar_try(bar, parity)) return;          // the common case costs one instruction
   if (*wc.abort_flag) return;
   for (uint32_t it = 0; it < kSpinLimit; ++it)
     if (mbar_try(bar, parity)) return;
@@ -220,6 +228,21 @@ __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint64_t b_d
         "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), \
         "r"(r[15]) : "memory")
 
+#define XKV_TMEM_LD16(taddr, r)                                                                      \
+  asm volatile(                                                                                      \
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "                                                      \
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"                              \
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), \
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),     \
+        "=r"(r[15])                                                                                  \
+      : "r"(taddr) : "memory")
+
+#define XKV_TMEM_ST8(taddr, r)                                                                       \
+  asm volatile(                                                                                      \
+      "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"                       \
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),     \
+        "r"(r[7]) : "memory")
+
 // Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 B apart.
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
   uint64_t d = 0;
@@ -296,6 +319,20 @@ __device__ __forceinline__ void tma_load_1d(uint32_t dst, const void* src, uint3
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// O[row][0..63] *= alpha for the 32 rows (TMEM lanes) of the calling warp; a real call, to keep its
+// registers out of the softmax loop.  Warp-collective.
+__device__ __noinline__ void rescale_rows(uint32_t col_o, float alpha) {
+#pragma unroll 1
+  for (int c0 = 0; c0 < 64; c0 += 32) {
+    uint32_t ra[32];
+    XKV_TMEM_LD32(col_o + c0, ra);
+    tc_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) ra[i] = __float_as_uint(__uint_as_float(ra[i]) * alpha);
+    XKV_TMEM_ST32(col_o + c0, ra);
+  }
+  tc_wait_st();
+}
 __device__ __forceinline__ void producer_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 }  // namespace
@@ -313,7 +350,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
   const uint32_t b_vfull = b_kfree + 8 * kNK, b_vfree = b_vfull + 8 * kNV;
   const uint32_t b_rfull = b_vfree + 8 * kNV, b_rfree = b_rfull + 8 * C::kNR;
   const uint32_t b_qfull = b_rfree + 8 * C::kNR;      // [2]
-  const uint32_t b_sfull = b_qfull + 16, b_pfull = b_sfull + 16, b_pvdone = b_pfull + 16;
+  const uint32_t b_sfull = b_qfull + 16, b_pfull = b_sfull + 16, b_pvdone = b_pfull + 16, b_sfree = b_pvdone + 16;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sgen + kOffBar + kBarBytes - 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + kOffBar + kBarBytes - 12);
   const WaitCtx wc{a.status, abort_flag};
@@ -328,12 +365,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
 
   if (tid == 0) {
     *abort_flag = (*reinterpret_cast<volatile int*>(a.status) != 0) ? 1 : 0;   // an earlier CTA already gave up
-    for (int i = 0; i < kNK; ++i) { mbar_init(b_kfull + 8 * i, 128); mbar_init(b_kfree + 8 * i, 1); }
-    for (int i = 0; i < kNV; ++i) { mbar_init(b_vfull + 8 * i, 128); mbar_init(b_vfree + 8 * i, 1); }
+    for (int i = 0; i < kNK; ++i) { mbar_init(b_kfull + 8 * i, 128); mbar_init(b_kfree + 8 * i, 2); }
+    for (int i = 0; i < kNV; ++i) { mbar_init(b_vfull + 8 * i, 128); mbar_init(b_vfree + 8 * i, 2); }
     for (int i = 0; i < C::kNR; ++i) { mbar_init(b_rfull + 8 * i, 1); mbar_init(b_rfree + 8 * i, 128); }
     for (int t = 0; t < 2; ++t) {
       mbar_init(b_qfull + 8 * t, 128); mbar_init(b_sfull + 8 * t, 1);
-      mbar_init(b_pfull + 8 * t, 128); mbar_init(b_pvdone + 8 * t, 1);
+      mbar_init(b_pfull + 8 * t, 128); mbar_init(b_pvdone + 8 * t, 1); mbar_init(b_sfree + 8 * t, 128);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -354,7 +391,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t colS = lane_addr + kColS + 128 * t, colP = lane_addr + kColP + 64 * t;
     const uint32_t colO = lane_addr + kColO + 64 * t;
-    const uint32_t sfull = b_sfull + 8 * t, pfull = b_pfull + 8 * t, pvdone = b_pvdone + 8 * t;
+    const uint32_t sfull = b_sfull + 8 * t, pfull = b_pfull + 8 * t, pvdone = b_pvdone + 8 * t, sfree = b_sfree + 8 * t;
     const int pad_tile = (a.t_first & 127) ? (a.t_first >> 7) : -1;
     const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2);
     uint32_t cnt = 0;                        // steps this tile has been through (barrier phases)
@@ -405,18 +442,101 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
         mbar_wait(sfull, cnt & 1, wc);
         __syncwarp();            // the spin loops may leave the warp diverged; tcgen05.ld/st are warp-collective
         tc_fence_after();
-        // pass 1: row maximum
-        float mx = -INFINITY;
-        if (lim >= 128) {
-#pragma unroll 1
-          for (int c0 = 0; c0 < 128; c0 += 32) {
-            uint32_t ra[32];
-            XKV_TMEM_LD32(colS + c0, ra);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) mx = max3(mx, __uint_as_float(ra[i]), __uint_as_float(ra[i + 1]));
+        bool pv_waited = (jj == 0);   // P of the previous step consumed, O quiescent (its PV completed)
+        auto wait_pv = [&]() {
+          if (!pv_waited) {
+            mbar_wait(pvdone, (cnt - 1) & 1, wc);
+            __syncwarp();
+            tc_fence_after();
+            pv_waited = true;
           }
+        };
+        // The reference maximum m_ref moves only when the row maximum grew by more than 2^14 over
+        // it: then the row sum and the accumulator are rescaled.
+        auto apply_max = [&](float mx_scaled) {
+          float alpha = 1.f;
+          const bool grow = mx_scaled > m_ref + kGrow;
+          if (grow) {
+            alpha = exp2f(m_ref - mx_scaled);      // 0 on the first tile (m_ref = -inf)
+            m_ref = mx_scaled;
+            l2 = mul_f2(l2, pack_f2(alpha, alpha));
+          }
+          if (jj > 0) {
+            wait_pv();
+            if (__any_sync(0xffffffffu, grow)) rescale_rows(colO, alpha);
+          }
+        };
+        if (lim >= 128) {
+          // ---- full tile.  Exponentials against the current reference in one pass over S.  The
+          // pass is valid when no exponential exceeded 2^kGrow; that is checked on the row sum of
+          // the first 96 columns and the maximum of the last 32.  Otherwise (always on the first
+          // tile of a segment, rarely afterwards) the row maximum is taken first, the reference
+          // moves, and the pass is repeated. ----
+          uint64_t lt2;
+#pragma unroll 1
+          for (int attempt = 0; attempt < 2; ++attempt) {
+            if (jj == 0 || attempt == 1) {
+              float mx = -INFINITY;
+#pragma unroll 1
+              for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t ra[32];
+                XKV_TMEM_LD32(colS + c0, ra);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) mx = max3(mx, __uint_as_float(ra[i]), __uint_as_float(ra[i + 1]));
+              }
+              apply_max(mx * a.scale_log2);
+            }
+            const bool last_attempt = (jj == 0 || attempt == 1);
+            const uint64_t nm2 = pack_f2(-m_ref, -m_ref);
+            lt2 = 0ull;
+            bool redo = false;
+            uint32_t ra[32], rb[32];
+            // exponentials of 32 columns against the reference; P (16-bit pairs) -> TMEM
+            auto chunk = [&](const uint32_t (&rr)[32], int c) {
+              uint32_t pk[16];
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const uint64_t x2 = fma_f2(pack_f2(__uint_as_float(rr[2 * i]), __uint_as_float(rr[2 * i + 1])), sc2, nm2);
+                const float p0 = fast_exp2(f2_lo(x2)), p1 = fast_exp2(f2_hi(x2));
+                lt2 = add_f2(lt2, pack_f2(p0, p1));
+                pk[i] = kBf16 ? pack_bf2(p0, p1) : pack_h2(p0, p1);
+              }
+              if (c == 0) wait_pv();
+              XKV_TMEM_ST16(colP + 16 * c, pk);
+            };
+            XKV_TMEM_LD32(colS, ra);
+            tc_wait_ld();
+#pragma unroll 1
+            for (int c = 0; c < 4; c += 2) {
+              XKV_TMEM_LD32(colS + 32 * (c + 1), rb);          // in flight while chunk c is processed
+              chunk(ra, c);
+              tc_wait_ld();
+              if (c == 0) {
+                XKV_TMEM_LD32(colS + 64, ra);
+              } else {
+                // all of S is in registers: unless the pass has to be repeated, the score columns
+                // can take the next tile's scores already
+                if (!last_attempt) {
+                  float mxl = -INFINITY;
+#pragma unroll
+                  for (int i = 0; i < 32; i += 2) mxl = max3(mxl, __uint_as_float(rb[i]), __uint_as_float(rb[i + 1]));
+                  const float part = f2_lo(lt2) + f2_hi(lt2);
+                  const bool bad = !(part < 16384.f) || (mxl * a.scale_log2 > m_ref + kGrow);
+                  redo = __any_sync(0xffffffffu, bad);
+                }
+                if (!redo) { tc_fence_before(); mbar_arrive(sfree); }
+              }
+              chunk(rb, c + 1);
+              if (c == 0) tc_wait_ld();
+            }
+            if (!redo) break;
+            tc_wait_st();
+          }
+          l2 = add_f2(l2, lt2);
         } else {
+          // ---- masked tile (pad slots after the first frame, the tail): two plain passes ----
+          float mx = -INFINITY;
 #pragma unroll 1
           for (int c0 = 0; c0 < 128; c0 += 32) {
             uint32_t ra[32];
@@ -428,53 +548,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
               mx = fmaxf(mx, x);
             }
           }
-        }
-        mx *= a.scale_log2;
-        // the reference maximum moves only when it grew by more than 2^8
-        float alpha = 1.f;
-        const bool grow = mx > m_ref + 8.f;
-        if (grow) {
-          alpha = exp2f(m_ref - mx);      // 0 on the first tile (m_ref = -inf)
-          m_ref = mx;
-          l2 = mul_f2(l2, pack_f2(alpha, alpha));
-        }
-        if (jj > 0) {
-          // P of the previous step has been consumed and O is quiescent once its PV completed
-          mbar_wait(pvdone, (cnt - 1) & 1, wc);
-          __syncwarp();
-          tc_fence_after();
-          if (__any_sync(0xffffffffu, grow)) {
-#pragma unroll 1
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-              uint32_t ra[32];
-              XKV_TMEM_LD32(colO + c0, ra);
-              tc_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; ++i) ra[i] = __float_as_uint(__uint_as_float(ra[i]) * alpha);
-              XKV_TMEM_ST32(colO + c0, ra);
-            }
-            tc_wait_st();
-          }
-        }
-        // pass 2: exponentials, row sum, P -> TMEM (16-bit pairs)
-        const uint64_t nm2 = pack_f2(-m_ref, -m_ref);
-        if (lim >= 128) {
-#pragma unroll 1
-          for (int c0 = 0; c0 < 128; c0 += 32) {
-            uint32_t ra[32];
-            XKV_TMEM_LD32(colS + c0, ra);
-            tc_wait_ld();
-            uint32_t pk[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const uint64_t x2 = fma_f2(pack_f2(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1])), sc2, nm2);
-              const float p0 = fast_exp2(f2_lo(x2)), p1 = fast_exp2(f2_hi(x2));
-              l2 = add_f2(l2, pack_f2(p0, p1));
-              pk[i] = kBf16 ? pack_bf2(p0, p1) : pack_h2(p0, p1);
-            }
-            XKV_TMEM_ST16(colP + (c0 >> 1), pk);
-          }
-        } else {
+          apply_max(mx * a.scale_log2);
+          wait_pv();
 #pragma unroll 1
           for (int c0 = 0; c0 < 128; c0 += 32) {
             uint32_t ra[32];
@@ -492,6 +567,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
             }
             XKV_TMEM_ST16(colP + (c0 >> 1), pk);
           }
+          tc_fence_before();
+          mbar_arrive(sfree);
         }
         tc_wait_st();
         tc_fence_before();
@@ -632,57 +709,55 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
         }
       }
     }
-  } else if (tid == 384) {
-    // =========================== MMA issuer ===================================
+  } else if (tid == 384 || tid == 448) {
+    // =========================== MMA issuers ==================================
+    // One thread per query tile.  Both release the K~/V~ stages (two arrivals each), also for an
+    // item that has no second tile: then the second thread only follows the rings.
+    const int t = (tid == 448) ? 1 : 0;
     const uint32_t idesc_qk = make_idesc(128, kBf16, false);
     const uint32_t idesc_pv = make_idesc(64, kBf16, true);
-    uint32_t g = 0;
-    uint32_t cnt[2] = {0, 0}, segq[2] = {0, 0};
+    const uint64_t dq = make_desc(sQ + t * 16384);
+    const uint32_t d_s = tmem + kColS + 128 * t, d_p = tmem + kColP + 64 * t, d_o = tmem + kColO + 64 * t;
+    uint32_t g = 0, cnt = 0, segq = 0;
     for (long long pos = step_lo; pos < step_hi;) {
       const int item = (int)(pos / a.n_tiles);
       const int tile_lo = (int)(pos - (long long)item * a.n_tiles);
       const int nt = (int)min((long long)(a.n_tiles - tile_lo), step_hi - pos);
       pos += nt;
       const int pair = item % a.n_pairs;
-      const int ntile = (2 * pair + 1 < a.q_tiles) ? 2 : 1;
-      auto issue_pv = [&](int t, uint32_t gv, bool first_of_segment) {
-        const uint64_t dv = make_desc(sV + (gv % kNV) * 16384);
+      const bool active = 2 * pair + t < a.q_tiles;
+      auto issue_pv = [&](uint32_t gv, bool first_of_segment) {
+        mbar_wait(b_vfull + 8 * (gv % kNV), (gv / kNV) & 1, wc);
+        if (active) {
+          mbar_wait(b_pfull + 8 * t, (cnt - 1) & 1, wc);        // P_t of that step written
+          tc_fence_after();
+          const uint64_t dv = make_desc(sV + (gv % kNV) * 16384);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)   // 16 keys per step: 2 swizzle atoms = 2048 B of V~, 8 columns of P
-          mma_ts(tmem + kColO + 64 * t, tmem + kColP + 64 * t + 8 * ks, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv,
-                 (!first_of_segment || ks > 0) ? 1u : 0u);
-        tc_commit(b_pvdone + 8 * t);
+          for (int ks = 0; ks < 8; ++ks)   // 16 keys per step: 2 swizzle atoms = 2048 B of V~, 8 columns of P
+            mma_ts(d_o, d_p + 8 * ks, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv,
+                   (!first_of_segment || ks > 0) ? 1u : 0u);
+          tc_commit(b_pvdone + 8 * t);
+        }
+        tc_commit(b_vfree + 8 * (gv % kNV));
       };
       for (int jj = 0; jj < nt; ++jj, ++g) {
         mbar_wait(b_kfull + 8 * (g % kNK), (g / kNK) & 1, wc);
-        const uint64_t dk = make_desc(sK + (g % kNK) * 16384);
-        for (int t = 0; t < ntile; ++t) {
-          if (jj == 0) mbar_wait(b_qfull + 8 * t, segq[t] & 1, wc);
-          else mbar_wait(b_pfull + 8 * t, (cnt[t] - 1) & 1, wc);   // S_t read, P_t of the previous step written
+        if (active) {
+          if (jj == 0) mbar_wait(b_qfull + 8 * t, segq & 1, wc);
+          else mbar_wait(b_sfree + 8 * t, (cnt - 1) & 1, wc);   // S_t of the previous step has been read
           tc_fence_after();
-          const uint64_t dq = make_desc(sQ + t * 16384);
+          const uint64_t dk = make_desc(sK + (g % kNK) * 16384);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)   // 16 channels per step: 32 B inside the swizzle span
-            mma_ss(tmem + kColS + 128 * t, dq + (uint64_t)(ks * 2), dk + (uint64_t)(ks * 2), idesc_qk, ks > 0 ? 1u : 0u);
+            mma_ss(d_s, dq + (uint64_t)(ks * 2), dk + (uint64_t)(ks * 2), idesc_qk, ks > 0 ? 1u : 0u);
           tc_commit(b_sfull + 8 * t);
-          if (jj > 0) {
-            if (t == 0) { mbar_wait(b_vfull + 8 * ((g - 1) % kNV), ((g - 1) / kNV) & 1, wc); tc_fence_after(); }
-            issue_pv(t, g - 1, jj == 1);
-          }
-          ++cnt[t];
         }
         tc_commit(b_kfree + 8 * (g % kNK));
-        if (jj > 0) tc_commit(b_vfree + 8 * ((g - 1) % kNV));
+        if (jj > 0) issue_pv(g - 1, jj == 1);
+        if (active) ++cnt;
       }
-      // the last PV of the segment
-      for (int t = 0; t < ntile; ++t) {
-        mbar_wait(b_pfull + 8 * t, (cnt[t] - 1) & 1, wc);
-        if (t == 0) mbar_wait(b_vfull + 8 * ((g - 1) % kNV), ((g - 1) / kNV) & 1, wc);
-        tc_fence_after();
-        issue_pv(t, g - 1, nt == 1);
-        ++segq[t];
-      }
-      tc_commit(b_vfree + 8 * ((g - 1) % kNV));
+      issue_pv(g - 1, nt == 1);           // the last PV of the segment
+      if (active) ++segq;
     }
     // all MMAs must be done before the CTA may free tensor memory: the softmax warps have waited
     // for every PV (pvdone) before their epilogues, and every QK (sfull) before that.

@@ -493,15 +493,26 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
             bool redo = false;
             uint32_t ra[32], rb[32];
             // exponentials of 32 columns against the reference; P (16-bit pairs) -> TMEM
-            auto chunk = [&](const uint32_t (&rr)[32], int c) {
-              uint32_t pk[16];
+            // Written in three sweeps over the chunk (scale and shift, exponentials, sums and
+            // conversion), each of 16 or 32 independent operations, so that the latency of the
+            // special-function unit is covered inside one warp.
+            auto chunk = [&](uint32_t (&rr)[32], int c) {
+              uint64_t x[16];
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const uint64_t x2 = fma_f2(pack_f2(__uint_as_float(rr[2 * i]), __uint_as_float(rr[2 * i + 1])), sc2, nm2);
-                const float p0 = fast_exp2(f2_lo(x2)), p1 = fast_exp2(f2_hi(x2));
-                lt2 = add_f2(lt2, pack_f2(p0, p1));
-                pk[i] = kBf16 ? pack_bf2(p0, p1) : pack_h2(p0, p1);
+              for (int i = 0; i < 16; ++i)
+                x[i] = fma_f2(pack_f2(__uint_as_float(rr[2 * i]), __uint_as_float(rr[2 * i + 1])), sc2, nm2);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) x[i] = pack_f2(fast_exp2(f2_lo(x[i])), fast_exp2(f2_hi(x[i])));
+              uint32_t pk[16];
+              uint64_t s0 = 0ull, s1 = 0ull;
+#pragma unroll
+              for (int i = 0; i < 16; i += 2) {
+                s0 = add_f2(s0, x[i]);
+                s1 = add_f2(s1, x[i + 1]);
+                pk[i] = kBf16 ? pack_bf2(f2_lo(x[i]), f2_hi(x[i])) : pack_h2(f2_lo(x[i]), f2_hi(x[i]));
+                pk[i + 1] = kBf16 ? pack_bf2(f2_lo(x[i + 1]), f2_hi(x[i + 1])) : pack_h2(f2_lo(x[i + 1]), f2_hi(x[i + 1]));
               }
+              lt2 = add_f2(lt2, add_f2(s0, s1));
               if (c == 0) wait_pv();
               XKV_TMEM_ST16(colP + 16 * c, pk);
             };

@@ -29,7 +29,7 @@ METRIC = "stream frames/s (24-layer compressed-KV attention)"
 UNIT = "frames/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture
 # summarised under profiles/ (None until a capture of the current kernel exists).
-ATTN_DRAM_TRAFFIC_BYTES = None
+ATTN_DRAM_TRAFFIC_BYTES = 24.04e6
 
 
 def _peaks() -> dict:
@@ -305,7 +305,7 @@ def run_xkv(args) -> None:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="xkv", choices=["xkv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

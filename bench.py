@@ -154,6 +154,27 @@ def run_reference(args) -> None:
 
 
 # --------------------------------------------------------------------------- GPU arm
+def replica_seed(base_seed: int, rank: int) -> int:
+    """Replicas stream different data: rank r uses seed base + 1000 r."""
+    return base_seed + 1000 * rank
+
+
+def max_over_ranks(value: float, device: str = "cuda") -> float:
+    """Slowest rank's time (the replicas share nothing; the job is as slow as its slowest stream)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    tt = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def aggregate_frames_per_s(world: int, steps: int, ms_total_max: float) -> float:
+    """Whole-job throughput of `world` independent replicas that each ran `steps` frames."""
+    return world * steps / (ms_total_max * 1e-3)
+
+
 def run_xkv(args) -> None:
     import torch
     import torch.distributed as dist
@@ -183,7 +204,7 @@ def run_xkv(args) -> None:
     K, W = args.steps, args.warmup
     fill = -(-w["budget"] // n)                     # 12 frames until every layer's cache is full
     pool = min(fill + W + K, 40)                    # distinct resident frames, cycled afterwards
-    seed = w["seed"] + 1000 * rank                  # replicas stream different data
+    seed = replica_seed(w["seed"], rank)
     frames = []
     for f in range(pool):
         q = torch.empty(L, H, n, d, dtype=torch.bfloat16, device="cuda")
@@ -221,10 +242,7 @@ def run_xkv(args) -> None:
         barrier()
     ms_total = ev0.elapsed_time(ev1)
     launches = sum(c.xkv_get_info().launches for c in caches) - launches0
-    if world > 1:
-        tt = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total)
     assert all(c.xkv_get_info().T == w["budget"] for c in caches)
     assert all(c.xkv_poll_status() == 0 for c in caches)
 
@@ -262,10 +280,7 @@ def run_xkv(args) -> None:
         step_host(i)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        tt = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_s = float(tt.item())
+    e2e_s = max_over_ranks(e2e_s)
     frame_bytes = L * H * n * d * 2
 
     if rank == 0:
@@ -276,7 +291,7 @@ def run_xkv(args) -> None:
         attn_avg_s = (attn_ms / max(attn_cnt, 1)) * 1e-3
         achieved = flops / attn_avg_s / 1e12 if attn_avg_s > 0 else 0.0
         prof_total = sum(v[0] for v in prof.values())
-        line = dict(metric=METRIC, value=world * K / (ms_total * 1e-3), unit=UNIT, n_gpus=world, steps=K, warmup=W,
+        line = dict(metric=METRIC, value=aggregate_frames_per_s(world, K, ms_total), unit=UNIT, n_gpus=world, steps=K, warmup=W,
                     ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f16",
                     data="synthetic",
                     config=dict(workload=w["name"], layers=L, heads=H, head_dim=d, tokens_per_frame=n,

@@ -824,34 +824,40 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
 // out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  Thread = (item, query
 // tile, row, 8-channel chunk); items that one CTA covered alone were written by it.
 // ---------------------------------------------------------------------------
+// IDX = uint32_t when total * grid fits 32 bits (the divisions are then cheap), else uint64_t.
+template <typename IDX>
 __global__ void __launch_bounds__(256)
-attn_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, int grid, long long total,
+attn_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml, int grid_i, long long total_ll,
                     int n_tiles, int n_pairs, int q_tiles, int n, __nv_bfloat16* __restrict__ out, int64_t ts,
                     int64_t hs) {
+  const IDX grid = (IDX)grid_i, total = (IDX)total_ll;
   const long long gidx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int ch = (int)(gidx & 7);
   const int r = (int)((gidx >> 3) & 127);
   const int t = (int)((gidx >> 10) & 1);
-  const long long item = gidx >> 11;
-  if (item * n_tiles >= total) return;
-  const int h = (int)(item / n_pairs), pair = (int)(item - (long long)h * n_pairs);
+  const IDX item = (IDX)(gidx >> 11);
+  if ((long long)item * n_tiles >= total_ll) return;
+  const int h = (int)(item / (IDX)n_pairs), pair = (int)(item - (IDX)h * (IDX)n_pairs);
   const int qt = 2 * pair + t;
   const int row = qt * 128 + r;
   if (qt >= q_tiles || row >= n) return;
-  const long long lo = item * n_tiles, hi = lo + n_tiles;
+  const IDX lo = item * (IDX)n_tiles, hi = lo + (IDX)n_tiles;
   // CTA that holds step x: the largest b with piece_start(b) <= x
   const int b_first = (int)(((lo + 1) * grid - 1) / total);
   const int b_last = (int)((hi * grid - 1) / total);
   if (b_first == b_last) return;                 // one CTA covered the whole item and wrote the result
+  // a piece's first segment (slot 0) is this item iff the piece starts inside it: only the first
+  // piece of the item can start before it
+  const bool first_is_second_slot = (total * (IDX)b_first) / grid < lo;
   float m = -INFINITY;
   for (int b = b_first; b <= b_last; ++b) {
-    const size_t slot = (size_t)2 * b + (piece_start(total, grid, b) >= lo ? 0 : 1);
+    const size_t slot = (size_t)2 * b + ((b == b_first && first_is_second_slot) ? 1 : 0);
     m = fmaxf(m, part_ml[(slot * 2 + t) * 128 + r].x);
   }
   float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   float l = 0.f;
   for (int b = b_first; b <= b_last; ++b) {
-    const size_t slot = (size_t)2 * b + (piece_start(total, grid, b) >= lo ? 0 : 1);
+    const size_t slot = (size_t)2 * b + ((b == b_first && first_is_second_slot) ? 1 : 0);
     const size_t prow = (slot * 2 + t) * 128 + r;
     const float2 ml = part_ml[prow];
     const float wgt = exp2f(ml.x - m);
@@ -922,8 +928,13 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
   {
     LaunchScope ls(c, XKV_PROF_COMBINE, st);
     const long long threads = (long long)H * a.n_pairs * 2048;
-    attn_combine_kernel<<<(int)((threads + 255) / 256), 256, 0, st>>>(a.part_o, a.part_ml, (int)grid, a.total,
-                                                                      a.n_tiles, a.n_pairs, a.q_tiles, n, a.out, ts, hs);
+    const int blocks = (int)((threads + 255) / 256);
+    if ((a.total + 1) * grid < (1ll << 31))
+      attn_combine_kernel<uint32_t><<<blocks, 256, 0, st>>>(a.part_o, a.part_ml, (int)grid, a.total, a.n_tiles,
+                                                            a.n_pairs, a.q_tiles, n, a.out, ts, hs);
+    else
+      attn_combine_kernel<uint64_t><<<blocks, 256, 0, st>>>(a.part_o, a.part_ml, (int)grid, a.total, a.n_tiles,
+                                                            a.n_pairs, a.q_tiles, n, a.out, ts, hs);
   }
   return cudaGetLastError();
 }

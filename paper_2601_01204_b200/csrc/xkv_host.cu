@@ -17,7 +17,7 @@ constexpr size_t kAlign = 256;
 struct Layout {
   int cap, row_bytes;
   size_t off_k[2], off_kpar[2], off_v[2], off_vpar[2], off_origin[2];
-  size_t off_kstage, off_qbar, off_qvec, off_scores, off_kept, off_counters, off_status, off_attn;
+  size_t off_kstage, off_qbar, off_qvec, off_scores, off_kept, off_counters, off_status, off_attn, off_hist;
   size_t attn_bytes;
   size_t total;
 };
@@ -47,6 +47,7 @@ Layout make_layout(const xkv_params* p) {
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + kAlign - 1) / kAlign * kAlign; return o; };
   L.off_status = take(256);
   L.off_counters = take(256);
+  L.off_hist = take(4096 * sizeof(unsigned int));
   for (int b = 0; b < 2; ++b) {
     L.off_k[b] = take(H * L.cap * L.row_bytes);
     L.off_kpar[b] = take(H * (L.cap / 64) * 64 * sizeof(float2));
@@ -122,6 +123,7 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
   c->scores = reinterpret_cast<float*>(c->ws + L.off_scores);
   c->kept = reinterpret_cast<int32_t*>(c->ws + L.off_kept);
   c->counters = reinterpret_cast<unsigned int*>(c->ws + L.off_counters);
+  c->sel_hist = reinterpret_cast<unsigned int*>(c->ws + L.off_hist);
   c->status = reinterpret_cast<int*>(c->ws + L.off_status);
   c->attn_part = reinterpret_cast<float*>(c->ws + L.off_attn);
   c->attn_part_bytes = L.attn_bytes;

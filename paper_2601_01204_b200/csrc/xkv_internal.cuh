@@ -53,6 +53,7 @@ struct xkv_cache {
   float* scores;           // [cap]
   int32_t* kept;           // [cap]
   unsigned int* counters;  // [8] device counters (self-resetting)
+  unsigned int* sel_hist;  // [4096] histogram of the top 12 bits of the score keys (self-clearing)
   int* status;             // device status word
   float* attn_part;        // split-KV partials of the attention kernel
   size_t attn_part_bytes;

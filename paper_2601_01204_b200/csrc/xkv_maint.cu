@@ -3,6 +3,8 @@
 // survivor gather.  All bandwidth- or latency-bound; fp32 arithmetic whose every
 // operation and order is fixed, because it decides integers (kept indices, 4-bit
 // codes) that must be reproducible bit for bit.
+#include <stdlib.h>
+
 #include "xkv_internal.cuh"
 
 namespace xkv {
@@ -280,10 +282,18 @@ cudaError_t launch_pool_q(xkv_cache* c, const void* q, int n, int64_t ts, int64_
 // with a balanced tree: three levels inside the lane, three by xor-shuffle.
 // The words of four heads are fetched ahead of their (ordered) use.
 // ---------------------------------------------------------------------------
+// Unsigned key whose order is the total order of fp32 bit patterns (so that -0 < +0).
+__device__ __forceinline__ uint32_t order_key(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+constexpr int kSelBins = 4096;          // histogram of the top 12 key bits, filled by the score kernel
+
 template <int BITS>
 __global__ void __launch_bounds__(512)
 score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* __restrict__ qvec,
-             float* __restrict__ scores, int force_plain) {
+             float* __restrict__ scores, unsigned int* __restrict__ hist, int force_plain) {
   // Parameters of the CTA's key group.  Fast path: float4 [H][4][8] = (s, magic + z) of channels
   // 8w + 2v and 8w + 2v + 1 at [h][v][w], so that the eight lanes of a quarter-warp read
   // consecutive 16-byte chunks.  Plain path: float2 (s, z) [H][64].
@@ -388,7 +398,10 @@ score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* 
   float s = __fadd_rn(t0, t2);
 #pragma unroll
   for (int o = 1; o < 8; o <<= 1) s = __fadd_rn(s, __shfl_xor_sync(0xffffffffu, s, o));
-  if (valid && w == 0) scores[i] = s;
+  if (valid && w == 0) {
+    scores[i] = s;
+    atomicAdd(&hist[order_key(s) >> 20], 1u);      // first digit of the selection (the select kernel clears it)
+  }
 }
 
 cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st) {
@@ -397,30 +410,25 @@ cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st) {
   LaunchScope ls(c, XKV_PROF_SCORE, st);
   if (c->p.kv_bits == 16)
     score_kernel<16><<<blocks, 512, smem, st>>>(c->buf[c->cur], c->p.n_heads, c->cap, c->rest_base, r_old,
-                                                c->qvec, c->scores, c->force_plain);
+                                                c->qvec, c->scores, c->sel_hist, c->force_plain);
   else
     score_kernel<4><<<blocks, 512, smem, st>>>(c->buf[c->cur], c->p.n_heads, c->cap, c->rest_base, r_old,
-                                               c->qvec, c->scores, c->force_plain);
+                                               c->qvec, c->scores, c->sel_hist, c->force_plain);
   return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------
-// Top-k of the scores (Sec. 3.2).  One CTA.  The order keys (fp32 bit pattern
-// mapped to an unsigned whose order is the float total order) are held in shared
-// memory when they fit.  The k-th largest key tau is found digit by digit (12, 10
-// and 10 bits): a pass histograms the digit of the keys that match the digits
-// found so far, a suffix scan locates the bin that holds the k-th largest.  Then
-// a stable compaction keeps every key above tau and the first (k - #above) keys
+// Top-k of the scores (Sec. 3.2).  One CTA.  The order keys are held in shared
+// memory when they fit.  The k-th largest key tau is found in two stages: the
+// histogram of the top 12 bits (counted by the score kernel with global atomics)
+// gives the bin that holds it; the keys of that bin, normally a few hundred, are
+// collected and the remaining 20 bits are found by bisection on them.  Then a
+// stable compaction keeps every key above tau and the first (k - #above) keys
 // equal to it.  Each thread owns a run of consecutive positions.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t order_key(float f) {
-  const uint32_t u = __float_as_uint(f);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
 constexpr int kSelThreads = 1024;
-constexpr int kSelSmemKeys = 48 * 1024;   // keys held in shared memory (192 KB)
-constexpr int kSelBins = 4096;
+constexpr int kSelSmemKeys = 44 * 1024;   // keys held in shared memory (176 KB)
+constexpr int kSelCand = 4096;            // candidates collected from the bin of tau
 
 __device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned int* s_warp,
                                                         unsigned int& total) {
@@ -451,86 +459,141 @@ __device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned
   return res;
 }
 
+// sum of v over the block (all threads get it); s_acc must be zero on entry and is zero on exit
+__device__ __forceinline__ unsigned int block_sum(unsigned int v, unsigned int* s_acc) {
+  v = __reduce_add_sync(0xffffffffu, v);
+  if ((threadIdx.x & 31) == 0 && v) atomicAdd(s_acc, v);
+  __syncthreads();
+  const unsigned int t = *s_acc;
+  __syncthreads();
+  if (threadIdx.x == 0) *s_acc = 0u;
+  return t;
+}
+
 template <bool IN_SMEM>
 __global__ void __launch_bounds__(kSelThreads)
-select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restrict__ kept) {
+select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restrict__ kept,
+              unsigned int* __restrict__ hist) {
   extern __shared__ uint32_t s_keys[];
-  __shared__ unsigned int s_hist[kSelBins];
+  __shared__ uint32_t s_cand[kSelCand];
   __shared__ unsigned int s_warp[33];
-  __shared__ unsigned int s_prefix, s_need;
+  __shared__ unsigned int s_bin, s_need, s_ncand, s_acc;
   const int tid = threadIdx.x;
   const int lane = tid & 31;
+  // ---- stage 1: the bin of tau from the 12-bit histogram (thread t owns 4 bins counted from the top) ----
+  unsigned int hb[4], own = 0u;
+  {
+    const uint4 h4 = *reinterpret_cast<const uint4*>(hist + kSelBins - 4 - 4 * tid);   // bins 4095-4t-3 .. 4095-4t
+    hb[0] = h4.w; hb[1] = h4.z; hb[2] = h4.y; hb[3] = h4.x;
+  }
   if (IN_SMEM)
     for (int j = tid; j < tp; j += kSelThreads) s_keys[j] = order_key(scores[j]);
-  if (tid == 0) { s_prefix = 0u; s_need = (unsigned int)k; }
+  if (tid == 0) { s_ncand = 0u; s_acc = 0u; }
   auto key_at = [&](int j) -> uint32_t { return IN_SMEM ? s_keys[j] : order_key(scores[j]); };
-
-  uint32_t mask = 0u;                  // bits of the key decided so far
-  int shift = 32;
-#pragma unroll 1
-  for (int pass = 0; pass < 3; ++pass) {
-    const int bits = (pass == 0) ? 12 : 10;
-    const int nbins = 1 << bits;
-    shift -= bits;
-    for (int b = tid; b < nbins; b += kSelThreads) s_hist[b] = 0u;
-    __syncthreads();
-    const uint32_t prefix = s_prefix;
-    for (int base = 0; base < tp; base += kSelThreads) {
-      const int j = base + tid;
-      const bool in = j < tp;
-      const uint32_t key = in ? key_at(j) : 0u;
-      const bool cand = in && ((key & mask) == prefix);
-      const uint32_t digit = (key >> shift) & (uint32_t)(nbins - 1);
-      // a warp whose candidates all share one digit (e.g. all scores equal) adds once
-      const unsigned int cands = __ballot_sync(0xffffffffu, cand);
-      if (cands) {
-        const int leader = __ffs(cands) - 1;
-        const uint32_t d0 = __shfl_sync(0xffffffffu, digit, leader);
-        const bool same = __all_sync(0xffffffffu, !cand || digit == d0);
-        if (same) { if (lane == leader) atomicAdd(&s_hist[d0], (unsigned int)__popc(cands)); }
-        else if (cand) atomicAdd(&s_hist[digit], 1u);
-      }
+  *reinterpret_cast<uint4*>(hist + kSelBins - 4 - 4 * tid) = make_uint4(0u, 0u, 0u, 0u);   // ready for the next evicting step
+#pragma unroll
+  for (int u = 0; u < 4; ++u) own += hb[u];
+  unsigned int total;
+  unsigned int above = block_excl_scan(own, s_warp, total);   // keys in higher bins than this thread's
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    if (above < (unsigned int)k && (unsigned int)k <= above + hb[u]) {
+      s_bin = (unsigned int)(kSelBins - 1 - (4 * tid + u));
+      s_need = (unsigned int)k - above;
     }
-    __syncthreads();
-    // suffix scan: thread t owns `per` bins counted from the top
-    const int per = nbins / kSelThreads;                   // 4 or 1
-    unsigned int h[4] = {0u, 0u, 0u, 0u};
-    unsigned int own = 0u;
-    for (int u = 0; u < per; ++u) { h[u] = s_hist[nbins - 1 - (tid * per + u)]; own += h[u]; }
-    unsigned int total;
-    unsigned int above = block_excl_scan(own, s_warp, total);   // keys with a larger digit than this thread's bins
-    const unsigned int need = s_need;
-    for (int u = 0; u < per; ++u) {
-      if (above < need && need <= above + h[u]) {
-        s_prefix = prefix | ((uint32_t)(nbins - 1 - (tid * per + u)) << shift);
-        s_need = need - above;
-      }
-      above += h[u];
-    }
-    mask |= (uint32_t)(nbins - 1) << shift;
-    __syncthreads();
+    above += hb[u];
   }
-  const uint32_t tau = s_prefix;
-  const unsigned int need_eq = s_need;
-  // stable compaction; an odd run length keeps the runs of a warp on different shared-memory banks
-  const int ipt = ((tp + kSelThreads - 1) / kSelThreads) | 1;
+  __syncthreads();
+  const uint32_t bin = s_bin;
+  const unsigned int need = s_need;                  // tau is the need-th largest key of its bin
+
+  // ---- stage 2: collect the keys of that bin (each thread scans its run; a block scan places them) ----
+  const int ipt = ((tp + kSelThreads - 1) / kSelThreads) | 1;   // odd run length: a warp's runs on different banks
   const int j0 = min(tid * ipt, tp), j1 = min(j0 + ipt, tp);
+  unsigned int mine_n = 0u;
+  for (int j = j0; j < j1; ++j) mine_n += ((key_at(j) >> 20) == bin);
+  unsigned int ncand;
+  unsigned int at = block_excl_scan(mine_n, s_warp, ncand);
+  if (mine_n) {
+    for (int j = j0; j < j1; ++j) {
+      const uint32_t key = key_at(j);
+      if ((key >> 20) == bin) { if (at < (unsigned int)kSelCand) s_cand[at] = key; ++at; }
+    }
+  }
+  __syncthreads();
+
+  // ---- stage 3: the low 20 bits of tau by bisection on the candidates ----
+  uint32_t prefix = bin << 20;
+  unsigned int n_gt;                                 // candidates above tau
+  if (ncand <= (unsigned int)kSelThreads) {
+    const bool has = (unsigned int)tid < ncand;
+    const uint32_t mine = has ? s_cand[tid] : 0u;
+    for (int bit = 19; bit >= 0; --bit) {
+      const uint32_t trial = prefix | (1u << bit);
+      if ((unsigned int)__syncthreads_count(has && mine >= trial) >= need) prefix = trial;
+    }
+    n_gt = (unsigned int)__syncthreads_count(has && mine > prefix);
+  } else {
+    // rare (many equal or nearly equal scores): the same bisection over a list that does not fit
+    // one candidate per thread, or over all keys of the bin when it overflowed the list
+    const bool listed = ncand <= (unsigned int)kSelCand;
+    auto count = [&](uint32_t trial, bool strict) -> unsigned int {
+      unsigned int c = 0u;
+      if (listed) {
+        for (unsigned int i = tid; i < ncand; i += kSelThreads) c += strict ? (s_cand[i] > trial) : (s_cand[i] >= trial);
+      } else {
+        for (int j = j0; j < j1; ++j) {
+          const uint32_t key = key_at(j);
+          if ((key >> 20) == bin) c += strict ? (key > trial) : (key >= trial);
+        }
+      }
+      return block_sum(c, &s_acc);
+    };
+    for (int bit = 19; bit >= 0; --bit) {
+      const uint32_t trial = prefix | (1u << bit);
+      if (count(trial, false) >= need) prefix = trial;
+    }
+    n_gt = count(prefix, true);
+  }
+  const uint32_t tau = prefix;
+  const unsigned int need_eq = need - n_gt;          // keys equal to tau that are kept (lowest positions)
+
+  // ---- stage 4: stable compaction ----
   unsigned int cnt_eq = 0u, cnt_gt = 0u;
   for (int j = j0; j < j1; ++j) {
     const uint32_t key = key_at(j);
     cnt_eq += (key == tau);
     cnt_gt += (key > tau);
   }
-  unsigned int total;
   const unsigned int eq_before = block_excl_scan(cnt_eq, s_warp, total);
   unsigned int take_eq = 0u;
   if (eq_before < need_eq) take_eq = min(cnt_eq, need_eq - eq_before);
   unsigned int out = block_excl_scan(cnt_gt + take_eq, s_warp, total);
-  for (int j = j0; j < j1; ++j) {
-    const uint32_t key = key_at(j);
-    bool keep = key > tau;
-    if (key == tau && take_eq > 0u) { keep = true; --take_eq; }
-    if (keep) kept[out++] = j;
+  // The kept positions are listed in shared memory first (in the key array: a thread's keep flags
+  // are taken before anything is overwritten) and copied out in full lines; written from the
+  // runs directly, every store of a warp would touch 32 different sectors.
+  unsigned int flags = 0u;                           // runs longer than 32 keys take the direct route
+  const bool staged = IN_SMEM && ipt <= 32;
+  if (staged) {
+    for (int j = j0; j < j1; ++j) {
+      const uint32_t key = key_at(j);
+      bool keep = key > tau;
+      if (key == tau && take_eq > 0u) { keep = true; --take_eq; }
+      flags |= (keep ? 1u : 0u) << (j - j0);
+    }
+    __syncthreads();
+    int32_t* s_out = reinterpret_cast<int32_t*>(s_keys);
+    for (int j = j0; j < j1; ++j)
+      if ((flags >> (j - j0)) & 1u) s_out[out++] = j;
+    __syncthreads();
+    for (int i = tid; i < k; i += kSelThreads) kept[i] = s_out[i];
+  } else {
+    for (int j = j0; j < j1; ++j) {
+      const uint32_t key = key_at(j);
+      bool keep = key > tau;
+      if (key == tau && take_eq > 0u) { keep = true; --take_eq; }
+      if (keep) kept[out++] = j;
+    }
   }
 }
 
@@ -544,9 +607,10 @@ cudaError_t launch_select(xkv_cache* c, int r_old, int k, cudaStream_t st) {
   }
   LaunchScope ls(c, XKV_PROF_SELECT, st);
   if (r_old <= kSelSmemKeys)
-    select_kernel<true><<<1, kSelThreads, (size_t)r_old * sizeof(uint32_t), st>>>(c->scores, r_old, k, c->kept);
+    select_kernel<true><<<1, kSelThreads, (size_t)r_old * sizeof(uint32_t), st>>>(c->scores, r_old, k, c->kept,
+                                                                                   c->sel_hist);
   else
-    select_kernel<false><<<1, kSelThreads, 0, st>>>(c->scores, r_old, k, c->kept);
+    select_kernel<false><<<1, kSelThreads, 0, st>>>(c->scores, r_old, k, c->kept, c->sel_hist);
   return cudaGetLastError();
 }
 

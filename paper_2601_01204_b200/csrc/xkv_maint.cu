@@ -470,7 +470,8 @@ __device__ __forceinline__ unsigned int block_sum(unsigned int v, unsigned int* 
   return t;
 }
 
-template <bool IN_SMEM>
+// KPT > 0: every thread's run has at most KPT keys and is held in registers after the first read.
+template <bool IN_SMEM, int KPT>
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restrict__ kept,
               unsigned int* __restrict__ hist) {
@@ -510,15 +511,25 @@ select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restri
   // ---- stage 2: collect the keys of that bin (each thread scans its run; a block scan places them) ----
   const int ipt = ((tp + kSelThreads - 1) / kSelThreads) | 1;   // odd run length: a warp's runs on different banks
   const int j0 = min(tid * ipt, tp), j1 = min(j0 + ipt, tp);
+  constexpr int kR = KPT > 0 ? KPT : 1;
+  uint32_t kr[kR];                                   // this thread's run (KPT > 0)
+  if (KPT > 0) {
+#pragma unroll
+    for (int i = 0; i < kR; ++i) kr[i] = (j0 + i < j1) ? key_at(j0 + i) : 0u;
+  }
+  // key i of the run: from registers when the loop over i is unrolled, else from memory
+#define XKV_RUN_LOOP(BODY)                                                              \
+  if (KPT > 0) {                                                                        \
+    _Pragma("unroll") for (int i = 0; i < kR; ++i) if (j0 + i < j1) { const int j = j0 + i; const uint32_t key = kr[i]; BODY } \
+  } else {                                                                              \
+    for (int j = j0; j < j1; ++j) { const uint32_t key = key_at(j); BODY }              \
+  }
   unsigned int mine_n = 0u;
-  for (int j = j0; j < j1; ++j) mine_n += ((key_at(j) >> 20) == bin);
+  XKV_RUN_LOOP({ (void)j; mine_n += ((key >> 20) == bin); })
   unsigned int ncand;
   unsigned int at = block_excl_scan(mine_n, s_warp, ncand);
   if (mine_n) {
-    for (int j = j0; j < j1; ++j) {
-      const uint32_t key = key_at(j);
-      if ((key >> 20) == bin) { if (at < (unsigned int)kSelCand) s_cand[at] = key; ++at; }
-    }
+    XKV_RUN_LOOP({ (void)j; if ((key >> 20) == bin) { if (at < (unsigned int)kSelCand) s_cand[at] = key; ++at; } })
   }
   __syncthreads();
 
@@ -542,10 +553,7 @@ select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restri
       if (listed) {
         for (unsigned int i = tid; i < ncand; i += kSelThreads) c += strict ? (s_cand[i] > trial) : (s_cand[i] >= trial);
       } else {
-        for (int j = j0; j < j1; ++j) {
-          const uint32_t key = key_at(j);
-          if ((key >> 20) == bin) c += strict ? (key > trial) : (key >= trial);
-        }
+        XKV_RUN_LOOP({ (void)j; if ((key >> 20) == bin) c += strict ? (key > trial) : (key >= trial); })
       }
       return block_sum(c, &s_acc);
     };
@@ -560,11 +568,7 @@ select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restri
 
   // ---- stage 4: stable compaction ----
   unsigned int cnt_eq = 0u, cnt_gt = 0u;
-  for (int j = j0; j < j1; ++j) {
-    const uint32_t key = key_at(j);
-    cnt_eq += (key == tau);
-    cnt_gt += (key > tau);
-  }
+  XKV_RUN_LOOP({ (void)j; cnt_eq += (key == tau); cnt_gt += (key > tau); })
   const unsigned int eq_before = block_excl_scan(cnt_eq, s_warp, total);
   unsigned int take_eq = 0u;
   if (eq_before < need_eq) take_eq = min(cnt_eq, need_eq - eq_before);
@@ -575,42 +579,53 @@ select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restri
   unsigned int flags = 0u;                           // runs longer than 32 keys take the direct route
   const bool staged = IN_SMEM && ipt <= 32;
   if (staged) {
-    for (int j = j0; j < j1; ++j) {
-      const uint32_t key = key_at(j);
+    XKV_RUN_LOOP({
       bool keep = key > tau;
       if (key == tau && take_eq > 0u) { keep = true; --take_eq; }
       flags |= (keep ? 1u : 0u) << (j - j0);
-    }
+    })
     __syncthreads();
     int32_t* s_out = reinterpret_cast<int32_t*>(s_keys);
-    for (int j = j0; j < j1; ++j)
-      if ((flags >> (j - j0)) & 1u) s_out[out++] = j;
+    if (KPT > 0) {
+#pragma unroll
+      for (int i = 0; i < kR; ++i)
+        if ((flags >> i) & 1u) s_out[out++] = j0 + i;
+    } else {
+      for (int j = j0; j < j1; ++j)
+        if ((flags >> (j - j0)) & 1u) s_out[out++] = j;
+    }
     __syncthreads();
     for (int i = tid; i < k; i += kSelThreads) kept[i] = s_out[i];
   } else {
-    for (int j = j0; j < j1; ++j) {
-      const uint32_t key = key_at(j);
+    XKV_RUN_LOOP({
       bool keep = key > tau;
       if (key == tau && take_eq > 0u) { keep = true; --take_eq; }
       if (keep) kept[out++] = j;
-    }
+    })
   }
+#undef XKV_RUN_LOOP
 }
 
 cudaError_t launch_select(xkv_cache* c, int r_old, int k, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    const cudaError_t e = cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               kSelSmemKeys * (int)sizeof(uint32_t));
+    cudaError_t e = cudaFuncSetAttribute(select_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kSelSmemKeys * (int)sizeof(uint32_t));
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(select_kernel<true, 17>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kSelSmemKeys * (int)sizeof(uint32_t));
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   LaunchScope ls(c, XKV_PROF_SELECT, st);
-  if (r_old <= kSelSmemKeys)
-    select_kernel<true><<<1, kSelThreads, (size_t)r_old * sizeof(uint32_t), st>>>(c->scores, r_old, k, c->kept,
-                                                                                   c->sel_hist);
+  const size_t smem = (size_t)r_old * sizeof(uint32_t);
+  const int ipt = ((r_old + kSelThreads - 1) / kSelThreads) | 1;
+  if (r_old > kSelSmemKeys)
+    select_kernel<false, 0><<<1, kSelThreads, 0, st>>>(c->scores, r_old, k, c->kept, c->sel_hist);
+  else if (ipt <= 17)
+    select_kernel<true, 17><<<1, kSelThreads, smem, st>>>(c->scores, r_old, k, c->kept, c->sel_hist);
   else
-    select_kernel<false><<<1, kSelThreads, 0, st>>>(c->scores, r_old, k, c->kept, c->sel_hist);
+    select_kernel<true, 0><<<1, kSelThreads, smem, st>>>(c->scores, r_old, k, c->kept, c->sel_hist);
   return cudaGetLastError();
 }
 

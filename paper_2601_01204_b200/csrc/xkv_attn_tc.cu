@@ -133,11 +133,16 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // Bounded wait.  On exhaustion the failure is recorded (device status word and a
 // per-CTA flag); once the flag is up every later wait of the CTA gives up at once.
 struct WaitCtx { int* status; volatile int* abort_flag; };
+// SLEEP_NS: back-off between polls.  Warps that wait long (operand producers, the copy thread)
+// poll rarely so that they do not take issue slots from the softmax warps.
+template <int SLEEP_NS = 32>
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc) {
   if (mbar_try(bar, parity)) return;          // the common case costs one instruction
   if (*wc.abort_flag) return;
-  for (uint32_t it = 0; it < kSpinLimit; ++it)
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
     if (mbar_try(bar, parity)) return;
+    __nanosleep(SLEEP_NS);
+  }
   *wc.abort_flag = 1;
   atomicExch(wc.status, (int)XKV_E_TIMEOUT);
 }
@@ -645,7 +650,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
         const uint32_t kbuf = g % kNK, ku = g / kNK;
         const uint32_t vbuf = g % kNV, vu = g / kNV;
         const uint8_t* raw = sgen + kOffRaw + rs * C::kRawStage;
-        mbar_wait(b_rfull + 8 * rs, ru & 1, wc);
+        mbar_wait<256>(b_rfull + 8 * rs, ru & 1, wc);
         if (BITS == 4) {
           // ---- fp16 parameter tables of this tile (one (group, channel) and one key per thread) ----
           uint8_t* tab = sgen + kOffTab + (g & 1) * kTabBytes;
@@ -667,7 +672,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           uint32_t wd[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) wd[i] = *reinterpret_cast<const uint32_t*>(raw + (kb + 16 * i) * 32 + 4 * w);
-          mbar_wait(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
+          mbar_wait<256>(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
 #pragma unroll
           for (int grp = 0; grp < 2; ++grp) {
             const uint4 sv = *reinterpret_cast<const uint4*>(tab + grp * 128 + 16 * w);
@@ -684,7 +689,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           // ---- values ----
 #pragma unroll
           for (int i = 0; i < 8; ++i) wd[i] = *reinterpret_cast<const uint32_t*>(raw + C::kRawK + (kb + 16 * i) * 32 + 4 * w);
-          mbar_wait(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
+          mbar_wait<256>(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const uint4 pv = *reinterpret_cast<const uint4*>(tab + 512 + 16 * (kb + 16 * i));
@@ -702,7 +707,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           uint4 rowk[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) rowk[i] = *reinterpret_cast<const uint4*>(raw + (kb + 16 * i) * 128 + 16 * w);
-          mbar_wait(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
+          mbar_wait<256>(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
 #pragma unroll
           for (int i = 0; i < 8; ++i)
             *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + i * 2048) = rowk[i];
@@ -710,7 +715,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           mbar_arrive(b_kfull + 8 * kbuf);
 #pragma unroll
           for (int i = 0; i < 8; ++i) rowk[i] = *reinterpret_cast<const uint4*>(raw + C::kRawK + (kb + 16 * i) * 128 + 16 * w);
-          mbar_wait(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
+          mbar_wait<256>(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
 #pragma unroll
           for (int i = 0; i < 8; ++i)
             *reinterpret_cast<uint4*>(sgen + kOffV + vbuf * 16384 + row_off + i * 2048) = rowk[i];
@@ -786,7 +791,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
       for (int jj = 0; jj < nt; ++jj, ++g) {
         const int tile = tile_lo + jj;
         const uint32_t rs = g % C::kNR, ru = g / C::kNR;
-        mbar_wait(b_rfree + 8 * rs, (ru & 1) ^ 1, wc);
+        mbar_wait<256>(b_rfree + 8 * rs, (ru & 1) ^ 1, wc);
         const uint32_t dst = sRaw + rs * C::kRawStage, bar = b_rfull + 8 * rs;
         mbar_expect_tx(bar, C::kRawStage);
         const size_t slot0 = head_slot + (size_t)tile * 128;

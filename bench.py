@@ -309,12 +309,39 @@ def run_xkv(args) -> None:
                     kernels={k_: dict(ms_per_step=v_[0] / K, launches_per_step=v_[1] / K,
                                       share=v_[0] / prof_total if prof_total else 0.0) for k_, v_ in prof.items()
                              if v_[1]})
+        # cache-maintenance kernels against the HBM roofline: algorithmic bytes of one launch in
+        # steady state (cache full, n tokens evicted per step) over its measured duration
+        for k_, nbytes in maintenance_bytes(H, n, d, w["budget"], w["kv_bits"]).items():
+            if k_ in line["kernels"] and prof[k_][0] > 0:
+                sec = prof[k_][0] / prof[k_][1] * 1e-3
+                line["kernels"][k_].update(bytes_per_launch=nbytes, gb_per_s=nbytes / sec / 1e9,
+                                           hbm_frac=nbytes / sec / 1e9 / peaks["hbm_gbs"])
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def maintenance_bytes(H: int, n: int, d: int, budget: int, bits: int) -> dict:
+    """Bytes that one steady-state launch of each cache-maintenance kernel has to move (4-bit cache):
+    what it reads plus what it writes, every array once.  prunable = budget - n middle tokens are
+    scored, k = budget - 2 n of them survive, n new tokens arrive."""
+    if bits != 4:
+        return {}
+    row, code, par = d * 2, d // 2, 8                      # bf16 row, packed row, one (scale, zero) pair
+    prunable, k = budget - n, max(0, budget - 2 * n)
+    grp = lambda tokens: (tokens + 63) // 64 * d * par     # key parameters of the 64-token groups
+    return {
+        "append": H * n * (2 * row) + H * n * (row + code + par),          # K, V in; staged K, V codes + params out
+        "pool_q": H * n * row,
+        "score": H * (prunable * code + grp(prunable)) + 4 * prunable,
+        "select": 4 * prunable + 4 * k,
+        # keys regrouped (survivors' codes and parameters, new bf16 keys in; codes and parameters
+        # out) and the survivors' value rows and parameters moved
+        "regroup_k": H * (k * code + grp(k) + n * row + (k + n) * code + grp(k + n)) + 2 * H * k * (code + par),
+    }
 
 
 def main() -> None:

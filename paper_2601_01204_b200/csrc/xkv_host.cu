@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 
 #include "xkv_internal.cuh"
@@ -288,6 +289,43 @@ size_t xkv_stream_step_host_bytes(const xkv_params* params, int32_t n) {
   return 2 * 4 * ((t + kAlign - 1) / kAlign * kAlign);
 }
 
+namespace {
+
+// Copy streams and events of xkv_stream_step_host, one set per device, created on first use.
+struct HostStepPipe {
+  bool ready = false;
+  cudaStream_t up = nullptr, down = nullptr;      // host -> device, device -> host
+  cudaEvent_t start = nullptr;                    // the caller's stream at entry
+  cudaEvent_t up_done[2] = {nullptr, nullptr};    // inputs of the layer in slot s are on the device
+  cudaEvent_t comp_done[2] = {nullptr, nullptr};  // the layer in slot s has run: inputs free, output ready
+  cudaEvent_t down_done[2] = {nullptr, nullptr};  // output of slot s is in host memory: output buffer free
+};
+std::mutex g_pipe_mutex;
+HostStepPipe g_pipe[64];
+
+HostStepPipe* host_step_pipe() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  HostStepPipe& p = g_pipe[dev];
+  if (!p.ready) {
+    bool ok = cudaStreamCreateWithFlags(&p.up, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&p.down, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+      ok = cudaEventCreateWithFlags(&p.up_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&p.comp_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&p.down_done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;
+    p.ready = true;
+  }
+  return &p;
+}
+
+}  // namespace
+
+// The layers run on the caller's stream; the inputs of layer l + 1 are copied to the other half of
+// the staging buffer on a copy stream while layer l runs, and outputs go back on a third stream.
 int xkv_stream_step_host(xkv_cache* const* layers, int32_t n_layers, const void* const* q,
                          const void* const* k, const void* const* v, void* const* out, int32_t n,
                          void* dev_staging, size_t staging_bytes, xkv_stream stream) {
@@ -295,33 +333,58 @@ int xkv_stream_step_host(xkv_cache* const* layers, int32_t n_layers, const void*
   const xkv_params* p = &layers[0]->p;
   if (n < 1 || n > p->max_frame_tokens) return XKV_E_INVALID;
   if (staging_bytes < xkv_stream_step_host_bytes(p, n)) return XKV_E_NOMEM;
+  for (int l = 0; l < n_layers; ++l)
+    if (!layers[l] || !q[l] || !k[l] || !v[l] || !out[l]) return XKV_E_INVALID;
+  HostStepPipe* pipe = host_step_pipe();
+  if (!pipe) return XKV_E_CUDA;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const size_t t = (size_t)p->n_heads * n * kHeadDim * sizeof(__nv_bfloat16);
   const size_t slot = (t + kAlign - 1) / kAlign * kAlign;
   uint8_t* base = reinterpret_cast<uint8_t*>(dev_staging);
   const int64_t ts = kHeadDim, hs = (int64_t)n * kHeadDim;
-  for (int l = 0; l < n_layers; ++l) {
+  int rc = XKV_OK;
+  bool cuda_ok = true;
+  auto ck = [&](cudaError_t e) { if (e != cudaSuccess) cuda_ok = false; };
+  // the copy streams start where the caller's stream stands (the staging buffer may be in use there)
+  ck(cudaEventRecord(pipe->start, st));
+  ck(cudaStreamWaitEvent(pipe->up, pipe->start, 0));
+  ck(cudaStreamWaitEvent(pipe->down, pipe->start, 0));
+  int l = 0;
+  for (; l < n_layers && cuda_ok && rc == XKV_OK; ++l) {
     xkv_cache* c = layers[l];
-    if (!c || !q[l] || !k[l] || !v[l] || !out[l]) return XKV_E_INVALID;
-    uint8_t* s = base + (size_t)(l & 1) * 4 * slot;
+    const int sl = l & 1;
+    uint8_t* s = base + (size_t)sl * 4 * slot;
     void* dq = s;
     void* dk = s + slot;
     void* dv = s + 2 * slot;
     void* dout = s + 3 * slot;
-    if (cudaMemcpyAsync(dk, k[l], t, cudaMemcpyHostToDevice, st) != cudaSuccess) return XKV_E_CUDA;
-    if (cudaMemcpyAsync(dv, v[l], t, cudaMemcpyHostToDevice, st) != cudaSuccess) return XKV_E_CUDA;
-    if (cudaMemcpyAsync(dq, q[l], t, cudaMemcpyHostToDevice, st) != cudaSuccess) return XKV_E_CUDA;
-    int rc = kv_append(c, dk, dv, n, ts, hs, stream);
-    if (rc != XKV_OK) return rc;
-    rc = kv_score_evict(c, dq, n, ts, hs, stream);
-    if (rc != XKV_OK) return rc;
-    rc = kv_quant_pack(c, stream);
-    if (rc != XKV_OK) return rc;
-    rc = attn_packed_causal(c, dq, dout, n, ts, hs, 1.0f / sqrtf((float)p->head_dim), 0, stream);
-    if (rc != XKV_OK) return rc;
-    if (cudaMemcpyAsync(out[l], dout, t, cudaMemcpyDeviceToHost, st) != cudaSuccess) return XKV_E_CUDA;
+    // inputs: once the layer that used this half two layers ago has run
+    if (l >= 2) ck(cudaStreamWaitEvent(pipe->up, pipe->comp_done[sl], 0));
+    ck(cudaMemcpyAsync(dk, k[l], t, cudaMemcpyHostToDevice, pipe->up));
+    ck(cudaMemcpyAsync(dv, v[l], t, cudaMemcpyHostToDevice, pipe->up));
+    ck(cudaMemcpyAsync(dq, q[l], t, cudaMemcpyHostToDevice, pipe->up));
+    ck(cudaEventRecord(pipe->up_done[sl], pipe->up));
+    // the layer: inputs present, and the output of two layers ago copied out of this half
+    ck(cudaStreamWaitEvent(st, pipe->up_done[sl], 0));
+    if (l >= 2) ck(cudaStreamWaitEvent(st, pipe->down_done[sl], 0));
+    if (!cuda_ok) break;
+    rc = kv_append(c, dk, dv, n, ts, hs, stream);
+    if (rc == XKV_OK) rc = kv_score_evict(c, dq, n, ts, hs, stream);
+    if (rc == XKV_OK) rc = kv_quant_pack(c, stream);
+    if (rc == XKV_OK) rc = attn_packed_causal(c, dq, dout, n, ts, hs, 1.0f / sqrtf((float)p->head_dim), 0, stream);
+    ck(cudaEventRecord(pipe->comp_done[sl], st));
+    if (rc != XKV_OK) break;
+    // output
+    ck(cudaStreamWaitEvent(pipe->down, pipe->comp_done[sl], 0));
+    ck(cudaMemcpyAsync(out[l], dout, t, cudaMemcpyDeviceToHost, pipe->down));
+    ck(cudaEventRecord(pipe->down_done[sl], pipe->down));
   }
-  return cudaStreamSynchronize(st) == cudaSuccess ? XKV_OK : XKV_E_CUDA;
+  // everything started above ends before the call returns, also after an error
+  ck(cudaStreamSynchronize(pipe->up));
+  ck(cudaStreamSynchronize(st));
+  ck(cudaStreamSynchronize(pipe->down));
+  if (rc != XKV_OK) return rc;
+  return cuda_ok ? XKV_OK : XKV_E_CUDA;
 }
 
 int xkv_get_info(const xkv_cache* c, xkv_info* info) {

@@ -159,3 +159,28 @@ def test_synth_kernel_matches_numpy_generator(xkv):
         xkv.xkv_synth_fill(dst, 9, 2, 5, tensor)
         got = dst.view(torch.int16).cpu().numpy().view(np.uint16)
         assert np.array_equal(got, synth.gen_tensor_bits(9, 2, 5, tensor, H, n, d))
+
+
+def test_host_buffer_step_equals_device_step(xkv):
+    """xkv_stream_step_host (inputs and outputs in pinned host memory, copies overlapped with the
+    kernels on the library's own copy streams) gives the bits of xkv_stream_step on device
+    tensors: three layers (so that both halves of the staging buffer are reused), frames past
+    the point where eviction starts."""
+    import torch
+    L, H, n, d, budget = 3, 4, 200, 64, 512
+    p = xkv.Params(n_heads=H, budget=budget, max_frame_tokens=n, kv_bits=4)
+    dev_caches = [xkv.Cache(p) for _ in range(L)]
+    host_caches = [xkv.Cache(p) for _ in range(L)]
+    staging = torch.empty(xkv.xkv_stream_step_host_bytes(p, n), dtype=torch.uint8, device="cuda")
+    for t in range(5):
+        frames = [synth.gen_frame(21, l, t, H, n, d) for l in range(L)]
+        dq, dk, dv = ([to_device_bf16(f[i]) for f in frames] for i in range(3))
+        dout = [torch.empty_like(x) for x in dq]
+        xkv.xkv_stream_step(dev_caches, dq, dk, dv, dout)
+        hq, hk, hv = ([x.cpu().pin_memory() for x in xs] for xs in (dq, dk, dv))
+        hout = [torch.empty_like(x).pin_memory() for x in hq]
+        xkv.xkv_stream_step_host(host_caches, hq, hk, hv, hout, staging)
+        torch.cuda.synchronize()
+        for l in range(L):
+            assert torch.equal(hout[l].view(torch.int16), dout[l].cpu().view(torch.int16)), (t, l)
+    assert host_caches[0].xkv_get_info().last_evicted > 0

@@ -854,23 +854,41 @@ attn_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__
   // a piece's first segment (slot 0) is this item iff the piece starts inside it: only the first
   // piece of the item can start before it
   const bool first_is_second_slot = (total * (IDX)b_first) / grid < lo;
-  float m = -INFINITY;
-  for (int b = b_first; b <= b_last; ++b) {
-    const size_t slot = (size_t)2 * b + ((b == b_first && first_is_second_slot) ? 1 : 0);
-    m = fmaxf(m, part_ml[(slot * 2 + t) * 128 + r].x);
-  }
+  // The partials are fetched four at a time, all loads before the first use (an item is cut into
+  // two or three pieces unless the cache is very long); the running maximum and the weights are
+  // those of the online softmax, in the fixed order of the pieces.
+  float m = -INFINITY, l = 0.f;
   float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  float l = 0.f;
-  for (int b = b_first; b <= b_last; ++b) {
-    const size_t slot = (size_t)2 * b + ((b == b_first && first_is_second_slot) ? 1 : 0);
-    const size_t prow = (slot * 2 + t) * 128 + r;
-    const float2 ml = part_ml[prow];
-    const float wgt = exp2f(ml.x - m);
-    l += wgt * ml.y;
-    const float4* po = reinterpret_cast<const float4*>(part_o + prow * 64 + 8 * ch);
-    const float4 x = po[0], y = po[1];
-    acc[0] += wgt * x.x; acc[1] += wgt * x.y; acc[2] += wgt * x.z; acc[3] += wgt * x.w;
-    acc[4] += wgt * y.x; acc[5] += wgt * y.y; acc[6] += wgt * y.z; acc[7] += wgt * y.w;
+  for (int b0 = b_first; b0 <= b_last; b0 += 4) {
+    float2 ml[4];
+    float4 x[4], y[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int b = b0 + j;
+      ml[j] = make_float2(-INFINITY, 0.f);
+      x[j] = y[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (b <= b_last) {
+        const size_t slot = (size_t)2 * b + ((b == b_first && first_is_second_slot) ? 1 : 0);
+        const size_t prow = (slot * 2 + t) * 128 + r;
+        ml[j] = part_ml[prow];
+        const float4* po = reinterpret_cast<const float4*>(part_o + prow * 64 + 8 * ch);
+        x[j] = po[0];
+        y[j] = po[1];
+      }
+    }
+    const float mc = fmaxf(fmaxf(m, fmaxf(ml[0].x, ml[1].x)), fmaxf(ml[2].x, ml[3].x));
+    const float sc = exp2f(m - mc);                // 0 for the first group (m = -inf)
+    m = mc;
+    l *= sc;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] *= sc;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float wgt = exp2f(ml[j].x - m);        // 0 for an absent piece
+      l += wgt * ml[j].y;
+      acc[0] += wgt * x[j].x; acc[1] += wgt * x[j].y; acc[2] += wgt * x[j].z; acc[3] += wgt * x[j].w;
+      acc[4] += wgt * y[j].x; acc[5] += wgt * y[j].y; acc[6] += wgt * y[j].z; acc[7] += wgt * y[j].w;
+    }
   }
   const float inv = 1.f / l;
   uint32_t o[4];

@@ -229,8 +229,16 @@ pool_q_kernel(const __nv_bfloat16* __restrict__ q, int n, int64_t ts, int64_t hs
   }
   __syncthreads();
   if (hslot == 0) {
-    float acc = s_pooled[c];
-    for (int h = 1; h < H; ++h) acc = __fadd_rn(acc, s_pooled[h * 64 + c]);
+    // (reads in batches ahead of the ordered additions)
+    float acc = 0.f;
+    for (int h0 = 0; h0 < H; h0 += 16) {
+      float v[16];
+#pragma unroll
+      for (int u = 0; u < 16; ++u) v[u] = (h0 + u < H) ? s_pooled[(h0 + u) * 64 + c] : 0.f;
+#pragma unroll
+      for (int u = 0; u < 16; ++u)
+        if (h0 + u < H) acc = (h0 + u == 0) ? v[u] : __fadd_rn(acc, v[u]);
+    }
     const float inv_h = __fdiv_rn(1.f, (float)H);
     __stcg(&qbar[i * 64 + c], __fmul_rn(acc, inv_h));
   }
@@ -251,8 +259,15 @@ pool_q_kernel(const __nv_bfloat16* __restrict__ q, int n, int64_t ts, int64_t hs
       for (int e = tid; e < rows * 64; e += nthr) s_rows[e] = __ldcg(&qbar[r0 * 64 + e]);
       __syncthreads();
       if (hslot == 0) {
-        float acc = (r0 == 0) ? s_rows[c] : s_acc[c];
-        for (int r = (r0 == 0) ? 1 : 0; r < rows; ++r) acc = __fadd_rn(acc, s_rows[r * 64 + c]);
+        float acc = (r0 == 0) ? 0.f : s_acc[c];
+        for (int q0 = 0; q0 < rows; q0 += 16) {
+          float v[16];
+#pragma unroll
+          for (int u = 0; u < 16; ++u) v[u] = (q0 + u < rows) ? s_rows[(q0 + u) * 64 + c] : 0.f;
+#pragma unroll
+          for (int u = 0; u < 16; ++u)
+            if (q0 + u < rows) acc = (r0 == 0 && q0 + u == 0) ? v[u] : __fadd_rn(acc, v[u]);
+        }
         s_acc[c] = acc;
       }
     }

@@ -210,7 +210,11 @@ XKV_API int attn_packed_causal_static(xkv_cache* cache, const void* q, void* out
 
 /* One frame through a stack of layers: for each layer in order, the four calls
  * above with softmax_scale = 1/sqrt(head_dim).  q, k, v, out are HOST arrays of
- * n_layers DEVICE pointers.  Stops at the first error and returns it. */
+ * n_layers DEVICE pointers.  Stops at the first error and returns it.
+ * Within a layer kv_append runs on a stream of the library's own (created on
+ * first use, one per device) beside kv_score_evict, which does not depend on it;
+ * both are ordered after everything already in `stream` and before the layer's
+ * kv_quant_pack, and a layer starts only after the previous layer's attention. */
 XKV_API int xkv_stream_step(xkv_cache* const* layers, int32_t n_layers,
                     const void* const* q, const void* const* k, const void* const* v,
                     void* const* out, int32_t n, int64_t tok_stride, int64_t head_stride,

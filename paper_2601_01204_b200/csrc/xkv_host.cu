@@ -263,38 +263,14 @@ int attn_packed_causal_static(xkv_cache* c, const void* q, void* out, int32_t n,
   return XKV_OK;
 }
 
-int xkv_stream_step(xkv_cache* const* layers, int32_t n_layers, const void* const* q, const void* const* k,
-                    const void* const* v, void* const* out, int32_t n, int64_t ts, int64_t hs,
-                    xkv_stream stream) {
-  if (!layers || !q || !k || !v || !out || n_layers < 1) return XKV_E_INVALID;
-  for (int l = 0; l < n_layers; ++l) {
-    xkv_cache* c = layers[l];
-    if (!c) return XKV_E_INVALID;
-    int rc = kv_append(c, k[l], v[l], n, ts, hs, stream);
-    if (rc != XKV_OK) return rc;
-    rc = kv_score_evict(c, q[l], n, ts, hs, stream);
-    if (rc != XKV_OK) return rc;
-    rc = kv_quant_pack(c, stream);
-    if (rc != XKV_OK) return rc;
-    rc = attn_packed_causal(c, q[l], out[l], n, ts, hs, 1.0f / sqrtf((float)c->p.head_dim), 0, stream);
-    if (rc != XKV_OK) return rc;
-  }
-  return XKV_OK;
-}
-
-size_t xkv_stream_step_host_bytes(const xkv_params* params, int32_t n) {
-  if (!params_ok(params) || n < 1) return 0;
-  // two slots (double buffering) of Q, K, V, out
-  const size_t t = (size_t)params->n_heads * n * kHeadDim * sizeof(__nv_bfloat16);
-  return 2 * 4 * ((t + kAlign - 1) / kAlign * kAlign);
-}
-
 namespace {
 
-// Copy streams and events of xkv_stream_step_host, one set per device, created on first use.
+// Streams and events of the stream-step calls, one set per device, created on first use.
 struct HostStepPipe {
   bool ready = false;
   cudaStream_t up = nullptr, down = nullptr;      // host -> device, device -> host
+  cudaStream_t side = nullptr;                    // kv_append of a layer, beside its scoring
+  cudaEvent_t fork = nullptr, join = nullptr;
   cudaEvent_t start = nullptr;                    // the caller's stream at entry
   cudaEvent_t up_done[2] = {nullptr, nullptr};    // inputs of the layer in slot s are on the device
   cudaEvent_t comp_done[2] = {nullptr, nullptr};  // the layer in slot s has run: inputs free, output ready
@@ -311,6 +287,9 @@ HostStepPipe* host_step_pipe() {
   if (!p.ready) {
     bool ok = cudaStreamCreateWithFlags(&p.up, cudaStreamNonBlocking) == cudaSuccess &&
               cudaStreamCreateWithFlags(&p.down, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&p.side, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.join, cudaEventDisableTiming) == cudaSuccess &&
               cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; i < 2 && ok; ++i)
       ok = cudaEventCreateWithFlags(&p.up_done[i], cudaEventDisableTiming) == cudaSuccess &&
@@ -322,7 +301,52 @@ HostStepPipe* host_step_pipe() {
   return &p;
 }
 
+// One layer, one frame.  kv_append (it needs K and V and writes the staging area and the other
+// buffer set) runs on the side stream while the pooled query, the scores and the selection (they
+// need Q and read the current buffer set) run on the caller's stream; the two meet before
+// kv_quant_pack.  The side stream starts where the caller's stream stands, i.e. after the previous
+// layer's attention: nothing of a layer starts before the layer before it has finished.
+int run_layer(HostStepPipe* pipe, xkv_cache* c, const void* q, const void* k, const void* v, void* out, int32_t n,
+              int64_t ts, int64_t hs, cudaStream_t st) {
+  xkv_stream stream = reinterpret_cast<xkv_stream>(st);
+  bool ok = cudaEventRecord(pipe->fork, st) == cudaSuccess &&
+            cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess;
+  if (!ok) return XKV_E_CUDA;
+  int rc = kv_append(c, k, v, n, ts, hs, reinterpret_cast<xkv_stream>(pipe->side));
+  ok = cudaEventRecord(pipe->join, pipe->side) == cudaSuccess;
+  if (rc == XKV_OK && ok) rc = kv_score_evict(c, q, n, ts, hs, stream);
+  // the join is made also after an error, so that the side stream is never left behind
+  ok = ok && cudaStreamWaitEvent(st, pipe->join, 0) == cudaSuccess;
+  if (rc != XKV_OK) return rc;
+  if (!ok) return XKV_E_CUDA;
+  rc = kv_quant_pack(c, stream);
+  if (rc != XKV_OK) return rc;
+  return attn_packed_causal(c, q, out, n, ts, hs, 1.0f / sqrtf((float)c->p.head_dim), 0, stream);
+}
+
 }  // namespace
+
+int xkv_stream_step(xkv_cache* const* layers, int32_t n_layers, const void* const* q, const void* const* k,
+                    const void* const* v, void* const* out, int32_t n, int64_t ts, int64_t hs,
+                    xkv_stream stream) {
+  if (!layers || !q || !k || !v || !out || n_layers < 1) return XKV_E_INVALID;
+  HostStepPipe* pipe = host_step_pipe();
+  if (!pipe) return XKV_E_CUDA;
+  for (int l = 0; l < n_layers; ++l) {
+    xkv_cache* c = layers[l];
+    if (!c) return XKV_E_INVALID;
+    const int rc = run_layer(pipe, c, q[l], k[l], v[l], out[l], n, ts, hs, reinterpret_cast<cudaStream_t>(stream));
+    if (rc != XKV_OK) return rc;
+  }
+  return XKV_OK;
+}
+
+size_t xkv_stream_step_host_bytes(const xkv_params* params, int32_t n) {
+  if (!params_ok(params) || n < 1) return 0;
+  // two slots (double buffering) of Q, K, V, out
+  const size_t t = (size_t)params->n_heads * n * kHeadDim * sizeof(__nv_bfloat16);
+  return 2 * 4 * ((t + kAlign - 1) / kAlign * kAlign);
+}
 
 // The layers run on the caller's stream; the inputs of layer l + 1 are copied to the other half of
 // the staging buffer on a copy stream while layer l runs, and outputs go back on a third stream.
@@ -368,10 +392,7 @@ int xkv_stream_step_host(xkv_cache* const* layers, int32_t n_layers, const void*
     ck(cudaStreamWaitEvent(st, pipe->up_done[sl], 0));
     if (l >= 2) ck(cudaStreamWaitEvent(st, pipe->down_done[sl], 0));
     if (!cuda_ok) break;
-    rc = kv_append(c, dk, dv, n, ts, hs, stream);
-    if (rc == XKV_OK) rc = kv_score_evict(c, dq, n, ts, hs, stream);
-    if (rc == XKV_OK) rc = kv_quant_pack(c, stream);
-    if (rc == XKV_OK) rc = attn_packed_causal(c, dq, dout, n, ts, hs, 1.0f / sqrtf((float)p->head_dim), 0, stream);
+    rc = run_layer(pipe, c, dq, dk, dv, dout, n, ts, hs, st);
     ck(cudaEventRecord(pipe->comp_done[sl], st));
     if (rc != XKV_OK) break;
     // output

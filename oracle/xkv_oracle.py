@@ -355,6 +355,9 @@ class OracleLayer:
         self._new_k = None
         self._new_v = None
         self._kept_rest = None                         # ascending old rest indices that survive
+        # the newest frame as it arrived (bf16 values in fp32), kept for attend(full_precision_tail=True)
+        self._cur_k = None
+        self._cur_v = None
         # diagnostics of the last step
         self.last_scores = None
         self.last_kept_mid = None
@@ -392,6 +395,7 @@ class OracleLayer:
         self.frames += 1
         self._new_k = np.ascontiguousarray(K, dtype=F32)
         self._new_v = np.ascontiguousarray(V, dtype=F32)
+        self._cur_k, self._cur_v = self._new_k, self._new_v
         self._kept_rest = None
         self.last_scores = None
         self.last_kept_mid = None
@@ -483,21 +487,32 @@ class OracleLayer:
         self._new_k = self._new_v = None
 
     # ---- step 5: attention over the packed cache ---------------------------
-    def attend(self, Q: np.ndarray, scale: float | None = None) -> np.ndarray:
+    def attend(self, Q: np.ndarray, scale: float | None = None, full_precision_tail: bool = False) -> np.ndarray:
         """Eq. 1 with Eq. 10.  Every cached token is from a frame <= t, so all are visible.
+
+        full_precision_tail: Eq. 1 read literally -- the frame attends to its own K_t, V_t as they
+        arrived and to the dequantised cache for everything older.  The newest frame holds the last
+        n positions of the cache; the cache itself (what later frames will see) is the same in
+        both readings.
 
         Returns fp32 [n][H][d].
         """
         if scale is None:
             scale = 1.0 / np.sqrt(self.p.head_dim)
-        O = attention(Q, self.keys_dequantized(), self.values_dequantized(), scale)
+        K, V = self.keys_dequantized(), self.values_dequantized()
+        if full_precision_tail:
+            n = self._cur_k.shape[1]
+            K = np.concatenate([K[:, :K.shape[1] - n], self._cur_k], axis=1)
+            V = np.concatenate([V[:, :V.shape[1] - n], self._cur_v], axis=1)
+        O = attention(Q, K, V, scale)
         return np.ascontiguousarray(np.transpose(O, (1, 0, 2)))
 
-    def step(self, Q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float | None = None):
+    def step(self, Q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float | None = None,
+             full_precision_tail: bool = False):
         self.append(K, V)
         self.score_evict(Q)
         self.quant_pack()
-        return self.attend(Q, scale)
+        return self.attend(Q, scale, full_precision_tail)
 
     # ---- export for bit-exact comparison ----------------------------------
     def export(self) -> dict:

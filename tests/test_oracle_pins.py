@@ -284,6 +284,60 @@ def test_streaming_4bit_no_pruning_equals_quantize_then_attend():
     assert np.array_equal(L.k_codes, kc) and np.array_equal(L.v_codes, vc)
 
 
+def test_full_precision_tail_reading_of_eq1():
+    """attend(full_precision_tail=True): the frame attends to its own K_t, V_t unquantised and to
+    the dequantised cache for older tokens (Eq. 1 read literally).  Pinned by:
+    the first frame is plain softmax(Q K^T / sqrt(d)) V on the raw tensors (torch, fp64);
+    with 16-bit storage both readings coincide; with 4-bit storage and pruning the result equals
+    attention over [dequantised older part of the cache | raw K_t, V_t] assembled by hand from the
+    exported cache, and the cache state is the same in both readings; and on average it is closer
+    to the unquantised attention than the packed reading."""
+    H, n, d, G = 2, 24, 16, 8
+    scale = 1.0 / np.sqrt(d)
+    frames = [[synth.bf16_bits_to_f32(a) for a in synth.gen_frame(13, 0, t, H, n, d)] for t in range(5)]
+
+    # first frame: everything is tail
+    p4 = xo.OracleParams(n_heads=H, head_dim=d, n_special=5, pool_g=4, quant_group=G, kv_bits=4, budget=3 * n)
+    L = xo.OracleLayer(p4)
+    q, k, v = frames[0]
+    out = L.step(q, k, v, full_precision_tail=True)                      # [n][H][d]
+    tq, tk, tv = [torch.from_numpy(x).double() for x in (q, k, v)]
+    ref = torch.softmax(tq @ tk.transpose(1, 2) * scale, dim=-1) @ tv    # [H][n][d]
+    np.testing.assert_allclose(out.transpose(1, 0, 2), ref.numpy(), rtol=1e-5, atol=1e-6)
+    assert np.abs(L.attend(q) - out).max() > 1e-3                        # the packed reading differs
+
+    # later frames, pruning active (budget 3n): hand-assembled reference, same cache in both readings
+    La, Lb = xo.OracleLayer(p4), xo.OracleLayer(p4)
+    err_tail, err_packed = [], []
+    Kraw, Vraw, fid = [], [], []
+    for t, (q, k, v) in enumerate(frames):
+        oa = La.step(q, k, v, full_precision_tail=True)
+        ob = Lb.step(q, k, v)
+        ea, eb = La.export(), Lb.export()
+        assert all(np.array_equal(ea[key], eb[key]) for key in ea)
+        T = La.T
+        Kd, Vd = La.keys_dequantized(), La.values_dequantized()
+        Kh = np.concatenate([Kd[:, :T - n], k], axis=1)
+        Vh = np.concatenate([Vd[:, :T - n], v], axis=1)
+        np.testing.assert_allclose(oa.transpose(1, 0, 2), xo.attention(q, Kh, Vh, scale), rtol=1e-6, atol=1e-7)
+        # against attention over the unquantised survivors
+        Kraw.append(k), Vraw.append(v), fid.append(np.full(n, t + 1))
+        org = La.origin
+        allk, allv = np.concatenate(Kraw, 1), np.concatenate(Vraw, 1)
+        pos = ((org >> 16) - 1) * n + (org & 0xFFFF)
+        exact = xo.attention(q, allk[:, pos], allv[:, pos], scale).transpose(1, 0, 2)
+        err_tail.append(np.linalg.norm(oa - exact)), err_packed.append(np.linalg.norm(ob - exact))
+    assert La.T == 3 * n                                                 # pruning happened
+    assert sum(err_tail) < sum(err_packed)
+
+    # 16-bit storage: nothing is quantised, the readings coincide
+    p16 = xo.OracleParams(n_heads=H, head_dim=d, n_special=5, pool_g=4, quant_group=G, kv_bits=16, budget=3 * n)
+    L16 = xo.OracleLayer(p16)
+    for q, k, v in frames:
+        L16.append(k, v); L16.score_evict(q); L16.quant_pack()
+        np.testing.assert_array_equal(L16.attend(q, full_precision_tail=True), L16.attend(q))
+
+
 # ------------------------------------------------------------------ eviction
 @pytest.mark.parametrize("bits", [4, 16])
 def test_eviction_invariants(bits):

@@ -166,6 +166,20 @@ XKV_API int attn_packed_causal(xkv_cache* cache, const void* q, void* out, int32
                        int64_t tok_stride, int64_t head_stride, float softmax_scale,
                        int32_t impl, xkv_stream stream);
 
+/* Step 5 with Eq. 1 read literally: the frame attends to its own K_t, V_t as they
+ * arrived (bf16) and to the packed cache (Eq. 10) for every older token; Sec. 3.3
+ * quantises "the final KV cache ... including the current frame", Eq. 1 shows the
+ * raw K_t, V_t inside the attention, and this call is the second reading.  k_t,
+ * v_t are the device tensors that kv_append took for this frame (n tokens, the
+ * strides of q).  The cache is left exactly as attn_packed_causal leaves it: later
+ * frames see this frame quantised either way.  A 16-bit cache stores the frame
+ * unchanged, so there both calls give the same result.  Always the tensor-core
+ * kernel.  Errors and state as attn_packed_causal; XKV_E_INVALID also when n is
+ * not the size of the frame appended last. */
+XKV_API int attn_packed_causal_tail(xkv_cache* cache, const void* q, const void* k_t, const void* v_t,
+                            void* out, int32_t n, int64_t tok_stride, int64_t head_stride,
+                            float softmax_scale, xkv_stream stream);
+
 /* attn_packed_causal for callers that must not allocate device memory.
  * (The paper has no counterpart: this is a deployment variant of Step 5 with the
  * same arithmetic and the same kernel.)

@@ -108,6 +108,13 @@ struct Args {
   float* part_o;        // [2 * grid][2][128][64]
   float2* part_ml;      // [2 * grid][2][128]
   int* status;
+  // Newest frame unquantised (Eq. 1 read literally): when k_tail is set, the key slots
+  // [tail_lo, t_phys) take K~, V~ from these bf16 tensors ([head][token][64] with the strides
+  // below, token = slot - tail_lo) instead of the packed rows.
+  const __nv_bfloat16* k_tail;
+  const __nv_bfloat16* v_tail;
+  int64_t tail_ts, tail_hs;
+  int tail_lo;
 };
 
 __device__ __forceinline__ long long piece_start(long long total, int grid, int b) {
@@ -315,6 +322,15 @@ __device__ __forceinline__ uint4 dequant_word_h(uint32_t w, const uint32_t (&s2)
 }
 
 
+// Eight bf16 values -> eight fp16 values (exact whenever the value is in fp16's range).
+__device__ __forceinline__ uint4 bf16x8_to_h8(const uint4& u) {
+  const uint32_t r[4] = {u.x, u.y, u.z, u.w};
+  uint32_t h[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) h[i] = pack_h2(__uint_as_float(r[i] << 16), __uint_as_float(r[i] & 0xFFFF0000u));
+  return make_uint4(h[0], h[1], h[2], h[3]);
+}
+
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
@@ -342,7 +358,9 @@ __device__ __forceinline__ void producer_sync() { asm volatile("bar.sync 1, 128;
 
 }  // namespace
 
-template <int BITS>
+// TAIL: the newest frame's keys and values come unquantised from Args::k_tail, v_tail (a separate
+// instantiation, so that the kernel without a tail carries none of its code).
+template <int BITS, bool TAIL = false>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
   using C = Cfg<BITS>;
   extern __shared__ uint8_t smem_raw[];
@@ -645,7 +663,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
       const int tile_lo = (int)(pos - (long long)item * a.n_tiles);
       const int nt = (int)min((long long)(a.n_tiles - tile_lo), step_hi - pos);
       pos += nt;
+      const int h = item / a.n_pairs;
       for (int jj = 0; jj < nt; ++jj, ++g) {
+        // keys of this tile that belong to the unquantised newest frame (none without a tail)
+        const int slot0 = (tile_lo + jj) * 128 + kb;              // this thread's keys: slot0 + 16 i
+        const bool tail_tile = TAIL && BITS == 4 && (tile_lo + jj) * 128 + 127 >= a.tail_lo;
+        const int64_t tail_off = (int64_t)h * a.tail_hs + 8 * w;
         const uint32_t rs = g % C::kNR, ru = g / C::kNR;
         const uint32_t kbuf = g % kNK, ku = g / kNK;
         const uint32_t vbuf = g % kNV, vu = g / kNV;
@@ -680,7 +703,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
             const uint32_t s2[4] = {sv.x, sv.y, sv.z, sv.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              const uint4 o = dequant_word_h(wd[4 * grp + i], s2, zo);
+              uint4 o = dequant_word_h(wd[4 * grp + i], s2, zo);
+              if (TAIL && tail_tile) {
+                const int slot = slot0 + 16 * (4 * grp + i);
+                if (slot >= a.tail_lo && slot < a.t_phys)
+                  o = bf16x8_to_h8(*reinterpret_cast<const uint4*>(a.k_tail + tail_off + (int64_t)(slot - a.tail_lo) * a.tail_ts));
+              }
               *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (4 * grp + i) * 2048) = o;
             }
           }
@@ -694,7 +722,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           for (int i = 0; i < 8; ++i) {
             const uint4 pv = *reinterpret_cast<const uint4*>(tab + 512 + 16 * (kb + 16 * i));
             const uint32_t s2[4] = {pv.x, pv.x, pv.x, pv.x}, zo[4] = {pv.y, pv.z, pv.y, pv.z};
-            const uint4 o = dequant_word_h(wd[i], s2, zo);
+            uint4 o = dequant_word_h(wd[i], s2, zo);
+            if (TAIL && tail_tile) {
+              const int slot = slot0 + 16 * i;
+              if (slot >= a.tail_lo && slot < a.t_phys)
+                o = bf16x8_to_h8(*reinterpret_cast<const uint4*>(a.v_tail + tail_off + (int64_t)(slot - a.tail_lo) * a.tail_ts));
+            }
             *reinterpret_cast<uint4*>(sgen + kOffV + vbuf * 16384 + row_off + i * 2048) = o;
           }
           fence_proxy_async();
@@ -902,8 +935,11 @@ size_t attn_tc_scratch_bytes(const xkv_params*) { return (size_t)2 * kMaxGrid * 
 // `part` holds the partial slots: accumulators float [slots][2][128][64], then (max, sum) float2
 // [slots][2][128], slots = part_bytes / kSlotBytes.  The grid is the SM count, capped by the slots
 // available (two per CTA) and by the number of steps.
+struct TailArgs { const void* k; const void* v; int64_t ts, hs; };
+
 static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
-                                     float scale, float* part, size_t part_bytes, cudaStream_t st) {
+                                     float scale, float* part, size_t part_bytes, cudaStream_t st,
+                                     const TailArgs* tail = nullptr) {
   static int sm_count = 0;
   static bool attr_set = false;
   if (!attr_set) {
@@ -915,6 +951,8 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
     e = cudaFuncSetAttribute(attn_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<16>());
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_tc_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -941,9 +979,20 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
   a.part_o = part;
   a.part_ml = reinterpret_cast<float2*>(part + slots * kSlotFloats);
   a.status = c->status;
+  a.k_tail = a.v_tail = nullptr;
+  a.tail_ts = a.tail_hs = 0;
+  a.tail_lo = a.t_phys;
+  if (tail && c->p.kv_bits == 4) {      // a 16-bit cache holds the frame exactly as it arrived
+    a.k_tail = reinterpret_cast<const __nv_bfloat16*>(tail->k);
+    a.v_tail = reinterpret_cast<const __nv_bfloat16*>(tail->v);
+    a.tail_ts = tail->ts;
+    a.tail_hs = tail->hs;
+    a.tail_lo = a.t_phys - n;           // the newest frame holds the last n slots
+  }
   {
     LaunchScope ls(c, XKV_PROF_ATTN, st);
     if (c->p.kv_bits == 16) attn_tc_kernel<16><<<(int)grid, kThreads, smem_bytes<16>(), st>>>(a);
+    else if (a.k_tail) attn_tc_kernel<4, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
     else attn_tc_kernel<4><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -965,6 +1014,12 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
 cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs, float scale,
                            cudaStream_t st) {
   return launch_attn_tc_on(c, q, out, n, ts, hs, scale, c->attn_part, c->attn_part_bytes, st);
+}
+
+cudaError_t launch_attn_tc_tail(xkv_cache* c, const void* q, const void* k_t, const void* v_t, void* out, int n,
+                                int64_t ts, int64_t hs, float scale, cudaStream_t st) {
+  const TailArgs tail{k_t, v_t, ts, hs};
+  return launch_attn_tc_on(c, q, out, n, ts, hs, scale, c->attn_part, c->attn_part_bytes, st, &tail);
 }
 
 // ---------------------------------------------------------------------------

@@ -248,6 +248,21 @@ int attn_packed_causal(xkv_cache* c, const void* q, void* out, int32_t n, int64_
   return XKV_OK;
 }
 
+int attn_packed_causal_tail(xkv_cache* c, const void* q, const void* k_t, const void* v_t, void* out, int32_t n,
+                            int64_t ts, int64_t hs, float softmax_scale, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  if (c->stage != 3) return XKV_E_STATE;
+  if (n < 1 || n != c->n_pending || !aligned16(q) || !aligned16(k_t) || !aligned16(v_t) || !aligned16(out) ||
+      !strides_ok(ts, hs) || !(softmax_scale > 0.f))
+    return XKV_E_INVALID;
+  const cudaError_t e =
+      launch_attn_tc_tail(c, q, k_t, v_t, out, n, ts, hs, softmax_scale, reinterpret_cast<cudaStream_t>(stream));
+  if (e == cudaErrorNotSupported) return XKV_E_UNSUPPORTED;
+  if (e != cudaSuccess) return XKV_E_CUDA;
+  c->stage = 0;
+  return XKV_OK;
+}
+
 int attn_packed_causal_static(xkv_cache* c, const void* q, void* out, int32_t n, int64_t ts, int64_t hs,
                               float softmax_scale, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;

@@ -103,6 +103,10 @@ cudaError_t launch_attn_simple(xkv_cache* c, const void* q, void* out, int n, in
 // Returns cudaErrorNotSupported when the tensor-core kernel cannot take the call.
 cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
                            float scale, cudaStream_t st);
+// Same kernel with the newest frame's keys and values taken unquantised from k_t, v_t (the tensors
+// given to kv_append, same strides as q).
+cudaError_t launch_attn_tc_tail(xkv_cache* c, const void* q, const void* k_t, const void* v_t, void* out, int n,
+                                int64_t ts, int64_t hs, float scale, cudaStream_t st);
 // Same kernel, split-KV partials in the library's fixed device array; cudaErrorMemoryAllocation
 // when the launch would need more than XKV_STATIC_SCRATCH_BYTES.
 cudaError_t launch_attn_tc_static(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,

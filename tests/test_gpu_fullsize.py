@@ -63,6 +63,18 @@ def _stream(xkv, n, budget, frames, seed, attn_from, bits=4):
             err = got.astype(np.float64) - ref
             assert np.abs(err).max() <= ATTN_MAXABS * np.abs(ref).max(), f"frame {t}"
             assert np.linalg.norm(err) <= ATTN_RELL2 * np.linalg.norm(ref), f"frame {t}"
+            # the same frame once more with its own K, V unquantised (Eq. 1 read literally)
+            cache.xkv_debug_rewind_attention()
+            cache.attn_packed_causal_tail(q, k, v, out)
+            Kt = np.concatenate([ora.keys_dequantized()[:, :ora.T - n], kf], axis=1)
+            Vt = np.concatenate([ora.values_dequantized()[:, :ora.T - n], vf], axis=1)
+            ref_t = xo.attention(qf[:, rows], Kt, Vt, scale)
+            got_t = bf16_tensor_to_f32(out)[:, rows]
+            err_t = got_t.astype(np.float64) - ref_t
+            assert np.abs(err_t).max() <= ATTN_MAXABS * np.abs(ref_t).max(), f"frame {t} (tail)"
+            assert np.linalg.norm(err_t) <= ATTN_RELL2 * np.linalg.norm(ref_t), f"frame {t} (tail)"
+            if bits == 4:   # and it is that reading, not the packed one
+                assert np.linalg.norm(err_t) < 0.5 * np.linalg.norm(got_t.astype(np.float64) - ref), f"frame {t}"
         assert cache.xkv_poll_status() == 0
     return cache, evicting
 

@@ -184,3 +184,39 @@ def test_host_buffer_step_equals_device_step(xkv):
         for l in range(L):
             assert torch.equal(hout[l].view(torch.int16), dout[l].cpu().view(torch.int16)), (t, l)
     assert host_caches[0].xkv_get_info().last_evicted > 0
+
+
+def test_unquantised_tail_streams(xkv):
+    """attn_packed_causal_tail against the oracle's full_precision_tail reading: the tiny stream
+    (first frame = all tail, eviction from frame 4), ragged frame sizes with small heads (tail start
+    anywhere inside a key tile), token-major layout, a single-token frame, and a budget below
+    first + current (cache = first frame + tail).  The packed state stays bit-exact throughout."""
+    run_stream(xkv, xkv.Params(budget=1024, max_frame_tokens=261), 261, 8, seed=1, tail=True)
+    run_stream(xkv, xkv.Params(n_heads=3, budget=500, max_frame_tokens=150, pool_g=7, n_special=2),
+               [129, 64, 150, 5, 77, 150, 33, 128], 8, seed=5, tail=True)
+    run_stream(xkv, xkv.Params(budget=700, max_frame_tokens=261), 261, 5, seed=6, token_major=True, tail=True)
+    run_stream(xkv, xkv.Params(n_heads=2, budget=256, max_frame_tokens=128, n_special=1, pool_g=16),
+               [128, 128, 1, 128, 64], 5, seed=6, tail=True)
+    run_stream(xkv, xkv.Params(n_heads=4, budget=300, max_frame_tokens=200), 200, 4, seed=9, tail=True)
+
+
+def test_unquantised_tail_on_16bit_cache_is_the_packed_result(xkv):
+    import torch
+    H, n, d = 4, 150, 64
+    p = xkv.Params(n_heads=H, budget=400, max_frame_tokens=n, kv_bits=16)
+    cache = xkv.Cache(p)
+    for t in range(5):
+        q, k, v = (to_device_bf16(x) for x in synth.gen_frame(31, 0, t, H, n, d))
+        cache.kv_append(k, v); cache.kv_score_evict(q); cache.kv_quant_pack()
+        a = cache.attn_packed_causal(q)
+        cache.xkv_debug_rewind_attention()
+        b = cache.attn_packed_causal_tail(q, k, v)
+        torch.cuda.synchronize()
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16)), t
+    # argument check: the tail has to be the frame appended last
+    q, k, v = (to_device_bf16(x) for x in synth.gen_frame(31, 0, 9, H, n, d))
+    cache.kv_append(k, v); cache.kv_score_evict(q); cache.kv_quant_pack()
+    o = torch.empty_like(q)
+    with pytest.raises(xkv.XkvError):
+        cache.attn_packed_causal_tail(q[:, :100], k[:, :100], v[:, :100], o[:, :100])
+    cache.attn_packed_causal_tail(q, k, v)

@@ -53,7 +53,8 @@ def check_attention(got: np.ndarray, ref: np.ndarray, tag: str = "") -> None:
     assert maxabs <= ATTN_MAXABS and rell2 <= ATTN_RELL2, f"{tag}: max-abs {maxabs:.3e}, rel-L2 {rell2:.3e}"
 
 
-def run_stream(xkv, p, n_tokens, n_frames, seed, impl=0, layer=0, token_major=False, check_attn_every=1):
+def run_stream(xkv, p, n_tokens, n_frames, seed, impl=0, layer=0, token_major=False, check_attn_every=1,
+               tail=False):
     """Stream n_frames through one GPU cache and one oracle layer, comparing after every call."""
     import torch
     cache = xkv.Cache(p)
@@ -84,9 +85,12 @@ def run_stream(xkv, p, n_tokens, n_frames, seed, impl=0, layer=0, token_major=Fa
         ora.quant_pack()
         compare_state(cache.export(), ora.export(), f"frame {t}")
         out = torch.empty_like(q)
-        cache.attn_packed_causal(q, out, impl=impl)
+        if tail:      # the frame's own K, V unquantised (attn_packed_causal_tail)
+            cache.attn_packed_causal_tail(q, k, v, out)
+        else:
+            cache.attn_packed_causal(q, out, impl=impl)
         if t % check_attn_every == 0 or t == len(n_list) - 1:
-            ref = ora.attend(qf)                                   # [n][H][d]
+            ref = ora.attend(qf, full_precision_tail=tail)         # [n][H][d]
             got = bf16_tensor_to_f32(out).transpose(1, 0, 2)
             check_attention(got, ref, f"frame {t}")
             e = attn_errors(got, ref)

@@ -201,6 +201,9 @@ def run_xkv(args) -> None:
     p = xkv.Params(n_heads=H, head_dim=d, n_special=w["n_special"], pool_g=w["pool_g"], quant_group=w["quant_group"],
                    kv_bits=w["kv_bits"], budget=w["budget"], max_frame_tokens=n)
     caches = [xkv.Cache(p, device=f"cuda:{local}") for _ in range(L)]
+    if args.tail:
+        for c in caches:
+            c.xkv_set_unquantised_tail(True)
     K, W = args.steps, args.warmup
     fill = -(-w["budget"] // n)                     # 12 frames until every layer's cache is full
     pool = min(fill + W + K, 40)                    # distinct resident frames, cycled afterwards
@@ -296,6 +299,7 @@ def run_xkv(args) -> None:
                     data="synthetic",
                     config=dict(workload=w["name"], layers=L, heads=H, head_dim=d, tokens_per_frame=n,
                                 budget=w["budget"], kv_bits=w["kv_bits"], prefill_frames=fill, resident_frames=pool,
+                                attention="unquantised_tail" if args.tail else "packed",
                                 l2="inputs exceed L2 (about 1.2 GB touched per step)", replicas=world),
                     clocks=clocks.summary(),
                     e2e=dict(value=world * Ke / e2e_s, unit=UNIT, h2d_bytes_per_step=3 * frame_bytes,
@@ -351,6 +355,8 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="xkv", choices=["xkv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tail", action="store_true",
+                    help="variant: every frame attends to its own K, V unquantised (attn_packed_causal_tail)")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: run a reduced stack of the same workload (default: all 24 layers)")
     args = ap.parse_args()

@@ -222,6 +222,11 @@ XKV_API int attn_packed_causal_static(xkv_cache* cache, const void* q, void* out
                               int64_t tok_stride, int64_t head_stride, float softmax_scale,
                               xkv_stream stream);
 
+/* Chooses the attention that xkv_stream_step and xkv_stream_step_host run for this
+ * cache: 0 (default) attn_packed_causal, 1 attn_packed_causal_tail with the K, V
+ * of the step.  The per-call entry points are not affected. */
+XKV_API int xkv_set_unquantised_tail(xkv_cache* cache, int32_t on);
+
 /* One frame through a stack of layers: for each layer in order, the four calls
  * above with softmax_scale = 1/sqrt(head_dim).  q, k, v, out are HOST arrays of
  * n_layers DEVICE pointers.  Stops at the first error and returns it.

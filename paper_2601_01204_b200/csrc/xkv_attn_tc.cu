@@ -673,6 +673,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
         const uint32_t kbuf = g % kNK, ku = g / kNK;
         const uint32_t vbuf = g % kNV, vu = g / kNV;
         const uint8_t* raw = sgen + kOffRaw + rs * C::kRawStage;
+        // rows of the unquantised newest frame: requested first, used after the waits below
+        uint4 tk[TAIL ? 8 : 1], tv[TAIL ? 8 : 1];
+        if (TAIL && tail_tile) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int slot = slot0 + 16 * i;
+            tk[i] = tv[i] = make_uint4(0, 0, 0, 0);
+            if (slot >= a.tail_lo && slot < a.t_phys) {
+              const int64_t off = tail_off + (int64_t)(slot - a.tail_lo) * a.tail_ts;
+              tk[i] = *reinterpret_cast<const uint4*>(a.k_tail + off);
+              tv[i] = *reinterpret_cast<const uint4*>(a.v_tail + off);
+            }
+          }
+        }
         mbar_wait<256>(b_rfull + 8 * rs, ru & 1, wc);
         if (BITS == 4) {
           // ---- fp16 parameter tables of this tile (one (group, channel) and one key per thread) ----
@@ -706,8 +720,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
               uint4 o = dequant_word_h(wd[4 * grp + i], s2, zo);
               if (TAIL && tail_tile) {
                 const int slot = slot0 + 16 * (4 * grp + i);
-                if (slot >= a.tail_lo && slot < a.t_phys)
-                  o = bf16x8_to_h8(*reinterpret_cast<const uint4*>(a.k_tail + tail_off + (int64_t)(slot - a.tail_lo) * a.tail_ts));
+                if (slot >= a.tail_lo && slot < a.t_phys) o = bf16x8_to_h8(tk[TAIL ? 4 * grp + i : 0]);
               }
               *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (4 * grp + i) * 2048) = o;
             }
@@ -725,8 +738,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
             uint4 o = dequant_word_h(wd[i], s2, zo);
             if (TAIL && tail_tile) {
               const int slot = slot0 + 16 * i;
-              if (slot >= a.tail_lo && slot < a.t_phys)
-                o = bf16x8_to_h8(*reinterpret_cast<const uint4*>(a.v_tail + tail_off + (int64_t)(slot - a.tail_lo) * a.tail_ts));
+              if (slot >= a.tail_lo && slot < a.t_phys) o = bf16x8_to_h8(tv[TAIL ? i : 0]);
             }
             *reinterpret_cast<uint4*>(sgen + kOffV + vbuf * 16384 + row_off + i * 2048) = o;
           }

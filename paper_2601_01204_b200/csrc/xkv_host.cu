@@ -263,6 +263,12 @@ int attn_packed_causal_tail(xkv_cache* c, const void* q, const void* k_t, const 
   return XKV_OK;
 }
 
+int xkv_set_unquantised_tail(xkv_cache* c, int32_t on) {
+  if (!c || (on != 0 && on != 1)) return XKV_E_INVALID;
+  c->tail_mode = on;
+  return XKV_OK;
+}
+
 int attn_packed_causal_static(xkv_cache* c, const void* q, void* out, int32_t n, int64_t ts, int64_t hs,
                               float softmax_scale, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;
@@ -336,7 +342,9 @@ int run_layer(HostStepPipe* pipe, xkv_cache* c, const void* q, const void* k, co
   if (!ok) return XKV_E_CUDA;
   rc = kv_quant_pack(c, stream);
   if (rc != XKV_OK) return rc;
-  return attn_packed_causal(c, q, out, n, ts, hs, 1.0f / sqrtf((float)c->p.head_dim), 0, stream);
+  const float scale = 1.0f / sqrtf((float)c->p.head_dim);
+  if (c->tail_mode) return attn_packed_causal_tail(c, q, k, v, out, n, ts, hs, scale, stream);
+  return attn_packed_causal(c, q, out, n, ts, hs, scale, 0, stream);
 }
 
 }  // namespace

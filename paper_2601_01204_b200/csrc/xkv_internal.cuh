@@ -63,6 +63,7 @@ struct xkv_cache {
   int last_evicted, last_kept, last_prunable;
   long long launches;
   int force_plain;         // 1: kernels take the plain (conversion-based) arithmetic forms everywhere
+  int tail_mode;           // 1: the stream-step calls attend with the step's K, V unquantised
   xkv::Profiler* prof;
 };
 

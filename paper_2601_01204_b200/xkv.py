@@ -33,7 +33,7 @@ EXPORTED = [
     "kv_quant_pack", "attn_packed_causal", "xkv_stream_step", "xkv_stream_step_host_bytes",
     "xkv_stream_step_host", "xkv_get_info", "xkv_debug_export", "xkv_poll_status", "xkv_strerror",
     "xkv_synth_fill", "xkv_profile_enable", "xkv_profile_read", "attn_packed_causal_static",
-    "xkv_debug_rewind_attention", "attn_packed_causal_tail",
+    "xkv_debug_rewind_attention", "attn_packed_causal_tail", "xkv_set_unquantised_tail",
 ]
 PROF_NAMES = ["append", "pool_q", "score", "select", "regroup_k", "gather", "attn", "attn_combine"]
 
@@ -74,6 +74,8 @@ lib.kv_quant_pack.restype = C.c_int
 lib.kv_quant_pack.argtypes = [_vp, _vp]
 lib.attn_packed_causal.restype = C.c_int
 lib.attn_packed_causal.argtypes = [_vp, _vp, _vp, _i32, _i64, _i64, C.c_float, _i32, _vp]
+lib.xkv_set_unquantised_tail.restype = C.c_int
+lib.xkv_set_unquantised_tail.argtypes = [_vp, _i32]
 lib.attn_packed_causal_tail.restype = C.c_int
 lib.attn_packed_causal_tail.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _i64, C.c_float, _vp]
 lib.attn_packed_causal_static.restype = C.c_int
@@ -196,6 +198,9 @@ class Cache:
         _check(lib.attn_packed_causal(self.handle, q.data_ptr(), out.data_ptr(), q.shape[1], ts, hs,
                                       C.c_float(scale), impl, _stream()), "attn_packed_causal")
         return out
+
+    def xkv_set_unquantised_tail(self, on: bool) -> None:
+        _check(lib.xkv_set_unquantised_tail(self.handle, 1 if on else 0), "xkv_set_unquantised_tail")
 
     def attn_packed_causal_tail(self, q, k_t, v_t, out=None, scale: float | None = None):
         """attn_packed_causal with the newest frame's keys and values taken unquantised from k_t, v_t

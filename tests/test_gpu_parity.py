@@ -161,6 +161,28 @@ def test_synth_kernel_matches_numpy_generator(xkv):
         assert np.array_equal(got, synth.gen_tensor_bits(9, 2, 5, tensor, H, n, d))
 
 
+def test_stream_step_with_unquantised_tail_option(xkv):
+    """xkv_set_unquantised_tail(1): the stream step gives what the per-call sequence with
+    attn_packed_causal_tail gives, bit for bit."""
+    import torch
+    L, H, n, d = 2, 4, 180, 64
+    p = xkv.Params(n_heads=H, budget=500, max_frame_tokens=n, kv_bits=4)
+    step_caches = [xkv.Cache(p) for _ in range(L)]
+    call_caches = [xkv.Cache(p) for _ in range(L)]
+    for c in step_caches:
+        c.xkv_set_unquantised_tail(True)
+    for t in range(5):
+        frames = [synth.gen_frame(41, l, t, H, n, d) for l in range(L)]
+        q, k, v = ([to_device_bf16(f[i]) for f in frames] for i in range(3))
+        out = [torch.empty_like(x) for x in q]
+        xkv.xkv_stream_step(step_caches, q, k, v, out)
+        for l, c in enumerate(call_caches):
+            c.kv_append(k[l], v[l]); c.kv_score_evict(q[l]); c.kv_quant_pack()
+            ref = c.attn_packed_causal_tail(q[l], k[l], v[l])
+            torch.cuda.synchronize()
+            assert torch.equal(out[l].view(torch.int16), ref.view(torch.int16)), (t, l)
+
+
 def test_host_buffer_step_equals_device_step(xkv):
     """xkv_stream_step_host (inputs and outputs in pinned host memory, copies overlapped with the
     kernels on the library's own copy streams) gives the bits of xkv_stream_step on device

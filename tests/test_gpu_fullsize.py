@@ -120,3 +120,56 @@ def test_workspace_is_the_only_memory_and_stays_flat(xkv):
     assert free1 == free0
     info = cache.xkv_get_info()
     assert info.T == 4096 and info.workspace_bytes == xkv.xkv_workspace_bytes(p)
+
+
+def test_long_stream_1000_frames_24_layers(xkv):
+    """The long-stream workload at its full length: 24 layers, 1004 tokens per frame, 1000 frames,
+    budget 16384, INT4, through xkv_stream_step.  The oracle cannot follow that far (seconds per
+    layer-step); checked here: device memory in use does not move after the caches are created,
+    every cache sits at the budget, no kernel reported an error, the outputs are finite, and the
+    survivors of every layer are the whole first frame, an increasing selection of later frames and
+    the whole last frame, in arrival order.  An uncompressed bf16 cache would hold
+    1000 x 1004 x 16 x 64 x 2 x 2 B x 24 layers = 98.7 GB by then."""
+    import torch
+    L, H, n, d, frames = 24, 16, 1004, 64, 1000
+    p = xkv.Params(n_heads=H, budget=16384, max_frame_tokens=n, kv_bits=4)
+    caches = [xkv.Cache(p) for _ in range(L)]
+    q = [torch.empty(H, n, d, dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+    k = [torch.empty_like(x) for x in q]
+    v = [torch.empty_like(x) for x in q]
+    out = [torch.empty_like(x) for x in q]
+    pool = 6          # distinct frames per layer, generated once and cycled (their content is arbitrary here)
+    bank = []
+    for f in range(pool):
+        fr = []
+        for l in range(L):
+            t3 = [torch.empty(H, n, d, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+            for x, which in zip(t3, (synth.TENSOR_Q, synth.TENSOR_K, synth.TENSOR_V)):
+                xkv.xkv_synth_fill(x, 4 + l, l, f, which)
+            fr.append(t3)
+        bank.append(fr)
+    xkv.xkv_stream_step(caches, [b[0] for b in bank[0]], [b[1] for b in bank[0]], [b[2] for b in bank[0]], out)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    held = sum(xkv.xkv_workspace_bytes(p) for _ in range(L))
+    for t in range(1, frames):
+        fr = bank[t % pool]
+        xkv.xkv_stream_step(caches, [b[0] for b in fr], [b[1] for b in fr], [b[2] for b in fr], out)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert held < 2.5e9 < 98.7e9                      # about 1.9 GB of workspaces for the whole stack
+    for l, c in enumerate(caches):
+        info = c.xkv_get_info()
+        assert info.T == 16384 and info.frames == frames and c.xkv_poll_status() == 0, l
+        assert bool(torch.isfinite(out[l].float()).all()), l
+    for l in (0, 11, 23):
+        info = caches[l].xkv_get_info()
+        org = caches[l].xkv_debug_export(xkv.BUF_ORIGIN, info.capacity * 4).view(np.int32)
+        sl = np.concatenate([np.arange(info.T_first), info.rest_base + np.arange(info.T - info.T_first)])
+        org = org[sl].astype(np.int64)
+        assert np.all(np.diff(org) > 0), l                                   # arrival order, no duplicates
+        assert np.array_equal(org[:n], (1 << 16) | np.arange(n)), l          # the first frame, whole
+        assert np.array_equal(org[-n:], (frames << 16) | np.arange(n)), l    # the newest frame, whole
+        mid = org[n:-n] >> 16
+        assert mid.min() >= 2 and mid.max() <= frames - 1, l

@@ -173,3 +173,10 @@ def test_long_stream_1000_frames_24_layers(xkv):
         assert np.array_equal(org[-n:], (frames << 16) | np.arange(n)), l    # the newest frame, whole
         mid = org[n:-n] >> 16
         assert mid.min() >= 2 and mid.max() <= frames - 1, l
+
+
+def test_ablation_budget_32768_int4(xkv):
+    """The largest budget of the ablation sweep: 1374 tokens per frame, budget 32768 (257 key tiles,
+    every item of the attention is cut into three or four pieces), first evicting frame 24."""
+    cache, evicting = _stream(xkv, 1374, 32768, 26, seed=5, attn_from=24)
+    assert cache.xkv_get_info().T == 32768 and evicting >= 2

@@ -197,6 +197,11 @@ def run_xkv(args) -> None:
     if args.layers > 0:
         w["layers"] = args.layers
         w["name"] += f"_reduced_to_{args.layers}_layers"
+    if args.budget > 0 or args.bits > 0 or args.tokens > 0:      # the ablation sweep and the long-stream shape
+        w["budget"] = args.budget or w["budget"]
+        w["kv_bits"] = args.bits or w["kv_bits"]
+        w["n_tokens"] = args.tokens or w["n_tokens"]
+        w["name"] = f"stack_{w['layers']}L_{w['n_tokens']}tok_budget{w['budget']}_{'int4' if w['kv_bits'] == 4 else 'bf16'}"
     L, H, d, n = w["layers"], w["n_heads"], w["head_dim"], w["n_tokens"]
     p = xkv.Params(n_heads=H, head_dim=d, n_special=w["n_special"], pool_g=w["pool_g"], quant_group=w["quant_group"],
                    kv_bits=w["kv_bits"], budget=w["budget"], max_frame_tokens=n)
@@ -309,7 +314,8 @@ def run_xkv(args) -> None:
                                   peak=peaks["tflops_sustained"], unit="TFLOP/s",
                                   frac=achieved / peaks["tflops_sustained"], peak_source=peaks["source"] + " (sustained)",
                                   frac_of_burst=achieved / peaks["tflops_burst"], flops_per_launch=flops,
-                                  avg_launch_ms=attn_avg_s * 1e3, traffic=ATTN_DRAM_TRAFFIC_BYTES),
+                                  avg_launch_ms=attn_avg_s * 1e3,
+                                  traffic=ATTN_DRAM_TRAFFIC_BYTES if w["name"] == WORKLOAD["name"] else None),
                     kernels={k_: dict(ms_per_step=v_[0] / K, launches_per_step=v_[1] / K,
                                       share=v_[0] / prof_total if prof_total else 0.0) for k_, v_ in prof.items()
                              if v_[1]})
@@ -326,6 +332,61 @@ def run_xkv(args) -> None:
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def run_uncompressed(args) -> None:
+    """The growing-cache baseline of the ablation list: 16-bit storage and a budget that is never
+    reached, i.e. no pruning and no quantisation, streamed from an empty cache.  The stream stops
+    at --uncompressed-frames; the frame at which this layout would fill 90 % of the free device
+    memory is computed, never provoked.  Prints one JSON line with the time of every 8th frame."""
+    import torch
+    import paper_2601_01204_b200.xkv as xkv
+    from paper_2601_01204_b200 import synth
+    if not torch.cuda.is_available():
+        sys.exit("bench.py needs a CUDA device")
+    w = dict(WORKLOAD)
+    L, H, d, n, F = w["layers"], w["n_heads"], w["head_dim"], w["n_tokens"], args.uncompressed_frames
+    p = xkv.Params(n_heads=H, head_dim=d, n_special=w["n_special"], pool_g=w["pool_g"], quant_group=w["quant_group"],
+                   kv_bits=16, budget=F * n, max_frame_tokens=n)
+    need = L * xkv.xkv_workspace_bytes(p)
+    free, _ = torch.cuda.mem_get_info()
+    per_frame = (L * xkv.xkv_workspace_bytes(xkv.Params(n_heads=H, head_dim=d, kv_bits=16, budget=2 * F * n,
+                                                        max_frame_tokens=n)) - need) / F
+    stop_frame = int((0.9 * free - (need - per_frame * F)) / per_frame)
+    if need > 0.5 * free:
+        sys.exit(f"refusing to hold {need / 1e9:.1f} GB of {free / 1e9:.1f} GB free: lower --uncompressed-frames")
+    caches = [xkv.Cache(p) for _ in range(L)]
+    pool = 4
+    frames = []
+    for f in range(pool):
+        q = torch.empty(L, H, n, d, dtype=torch.bfloat16, device="cuda")
+        k, v = torch.empty_like(q), torch.empty_like(q)
+        for l in range(L):
+            xkv.xkv_synth_fill(q[l], w["seed"] + l, l, f, synth.TENSOR_Q)
+            xkv.xkv_synth_fill(k[l], w["seed"] + l, l, f, synth.TENSOR_K)
+            xkv.xkv_synth_fill(v[l], w["seed"] + l, l, f, synth.TENSOR_V)
+        frames.append(tuple([x[l] for l in range(L)] for x in (q, k, v)))
+    out = torch.empty(L, H, n, d, dtype=torch.bfloat16, device="cuda")
+    outs = [out[l] for l in range(L)]
+    marks = []
+    for t in range(F):
+        q, k, v = frames[t % pool]
+        if t % 8 == 7 or t == F - 1:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            xkv.xkv_stream_step(caches, q, k, v, outs)
+            e1.record()
+            marks.append((t + 1, e0, e1))
+        else:
+            xkv.xkv_stream_step(caches, q, k, v, outs)
+    torch.cuda.synchronize()
+    assert all(c.xkv_get_info().T == F * n and c.xkv_poll_status() == 0 for c in caches)
+    print(json.dumps(dict(
+        workload=f"uncompressed_bf16_growing_{L}L_{n}tok", frames=F, workspace_gb=need / 1e9,
+        bytes_per_frame=per_frame, stop_frame_at_90pct_of_free_memory=stop_frame, free_gb=free / 1e9,
+        ms_per_frame={str(t): round(a.elapsed_time(b), 3) for t, a, b in marks},
+        note="this library keeps two buffer sets, so a frame costs twice the 135 MB of a single bf16 cache")),
+        flush=True)
 
 
 def maintenance_bytes(H: int, n: int, d: int, budget: int, bits: int) -> dict:
@@ -355,12 +416,19 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="xkv", choices=["xkv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--budget", type=int, default=0, help="variant of the workload: token budget (ablation sweep)")
+    ap.add_argument("--bits", type=int, default=0, choices=[0, 4, 16], help="variant: 4 or 16 (prune only)")
+    ap.add_argument("--tokens", type=int, default=0, help="variant: tokens per frame (1004 = long-stream shape)")
+    ap.add_argument("--uncompressed-frames", type=int, default=0,
+                    help="instead of the benchmark: stream this many frames through 16-bit caches that never prune")
     ap.add_argument("--tail", action="store_true",
                     help="variant: every frame attends to its own K, V unquantised (attn_packed_causal_tail)")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: run a reduced stack of the same workload (default: all 24 layers)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.uncompressed_frames > 0:
+        run_uncompressed(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_xkv(args)

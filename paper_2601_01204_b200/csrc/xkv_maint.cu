@@ -295,7 +295,8 @@ cudaError_t launch_pool_q(xkv_cache* c, const void* q, int n, int64_t ts, int64_
 // word of every head in order (Eq. 10), accumulate the head sum sequentially,
 // scale by 1/H (Eq. 4), multiply by the query vector, and add the 64 products
 // with a balanced tree: three levels inside the lane, three by xor-shuffle.
-// The words of four heads are fetched ahead of their (ordered) use.
+// The words of sixteen heads (4-bit; four 16-byte pieces for 16-bit storage) are fetched ahead of
+// their (ordered) use.
 // ---------------------------------------------------------------------------
 // Unsigned key whose order is the total order of fp32 bit patterns (so that -0 < +0).
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -362,27 +363,27 @@ score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* 
   float acc[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-  for (int h0 = 0; h0 < H; h0 += 4) {
-    uint32_t word[4];
-    uint4 wide[4];
+  constexpr int kHB = (BITS == 4) ? 16 : 4;     // heads whose words are in flight together
+  for (int h0 = 0; h0 < H; h0 += kHB) {
+    uint32_t word[BITS == 4 ? kHB : 1];
+    uint4 wide[BITS == 4 ? 1 : kHB];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kHB; ++u) {
       const int h = h0 + u;
-      word[u] = 0u;
-      wide[u] = make_uint4(0, 0, 0, 0);
+      if (BITS == 4) word[u] = 0u; else wide[u] = make_uint4(0, 0, 0, 0);
       if (valid && h < H) {
         if (BITS == 4) word[u] = *reinterpret_cast<const uint32_t*>(cur.k + ((size_t)h * cap + slot) * 32 + 4 * w);
         else wide[u] = *reinterpret_cast<const uint4*>(cur.k + ((size_t)h * cap + slot) * 128 + 16 * w);
       }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kHB; ++u) {
       const int h = h0 + u;
       if (h < H) {
         float x[8];
         if (BITS == 4) {
           if (plain) {
-            dequant8_plain(word[u], s_par + h * 64 + 8 * w, x);
+            dequant8_plain(word[BITS == 4 ? u : 0], s_par + h * 64 + 8 * w, x);
           } else {
             float2 par[8];
             const float4* pp = reinterpret_cast<const float4*>(s_par) + h * 32 + w;
@@ -392,10 +393,10 @@ score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* 
               par[2 * v] = make_float2(t.x, t.y);
               par[2 * v + 1] = make_float2(t.z, t.w);
             }
-            dequant8_magic(word[u], par, x);
+            dequant8_magic(word[BITS == 4 ? u : 0], par, x);
           }
         } else {
-          bf16x8_to_float(wide[u], x);
+          bf16x8_to_float(wide[BITS == 4 ? 0 : u], x);
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[j] = (h == 0) ? x[j] : __fadd_rn(acc[j], x[j]);

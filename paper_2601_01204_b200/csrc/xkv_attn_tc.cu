@@ -331,6 +331,26 @@ __device__ __forceinline__ uint4 bf16x8_to_h8(const uint4& u) {
   return make_uint4(h[0], h[1], h[2], h[3]);
 }
 
+// Rows of the unquantised newest frame over the dequantised rows of a K~ or V~ tile: keys
+// slot0 + 16 i of the tile that lie in [tail_lo, t_phys) are replaced by the caller's bf16 rows
+// (src already points at this thread's head and 8-channel chunk).  A real call, so that the
+// producers' loop carries none of this code.
+__device__ __noinline__ void tail_rows_over(uint8_t* tile_row, const __nv_bfloat16* src, int64_t ts, int slot0,
+                                            int tail_lo, int t_phys) {
+  uint4 u[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int slot = slot0 + 16 * i;
+    u[i] = make_uint4(0, 0, 0, 0);
+    if (slot >= tail_lo && slot < t_phys) u[i] = *reinterpret_cast<const uint4*>(src + (int64_t)(slot - tail_lo) * ts);
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int slot = slot0 + 16 * i;
+    if (slot >= tail_lo && slot < t_phys) *reinterpret_cast<uint4*>(tile_row + i * 2048) = bf16x8_to_h8(u[i]);
+  }
+}
+
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
@@ -673,20 +693,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
         const uint32_t kbuf = g % kNK, ku = g / kNK;
         const uint32_t vbuf = g % kNV, vu = g / kNV;
         const uint8_t* raw = sgen + kOffRaw + rs * C::kRawStage;
-        // rows of the unquantised newest frame: requested first, used after the waits below
-        uint4 tk[TAIL ? 8 : 1], tv[TAIL ? 8 : 1];
-        if (TAIL && tail_tile) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int slot = slot0 + 16 * i;
-            tk[i] = tv[i] = make_uint4(0, 0, 0, 0);
-            if (slot >= a.tail_lo && slot < a.t_phys) {
-              const int64_t off = tail_off + (int64_t)(slot - a.tail_lo) * a.tail_ts;
-              tk[i] = *reinterpret_cast<const uint4*>(a.k_tail + off);
-              tv[i] = *reinterpret_cast<const uint4*>(a.v_tail + off);
-            }
-          }
-        }
         mbar_wait<256>(b_rfull + 8 * rs, ru & 1, wc);
         if (BITS == 4) {
           // ---- fp16 parameter tables of this tile (one (group, channel) and one key per thread) ----
@@ -717,14 +723,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
             const uint32_t s2[4] = {sv.x, sv.y, sv.z, sv.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              uint4 o = dequant_word_h(wd[4 * grp + i], s2, zo);
-              if (TAIL && tail_tile) {
-                const int slot = slot0 + 16 * (4 * grp + i);
-                if (slot >= a.tail_lo && slot < a.t_phys) o = bf16x8_to_h8(tk[TAIL ? 4 * grp + i : 0]);
-              }
+              const uint4 o = dequant_word_h(wd[4 * grp + i], s2, zo);
               *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (4 * grp + i) * 2048) = o;
             }
           }
+          if (TAIL && tail_tile)
+            tail_rows_over(sgen + kOffK + kbuf * 16384 + row_off, a.k_tail + tail_off, a.tail_ts, slot0, a.tail_lo, a.t_phys);
           fence_proxy_async();
           mbar_arrive(b_kfull + 8 * kbuf);
           // ---- values ----
@@ -735,13 +739,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           for (int i = 0; i < 8; ++i) {
             const uint4 pv = *reinterpret_cast<const uint4*>(tab + 512 + 16 * (kb + 16 * i));
             const uint32_t s2[4] = {pv.x, pv.x, pv.x, pv.x}, zo[4] = {pv.y, pv.z, pv.y, pv.z};
-            uint4 o = dequant_word_h(wd[i], s2, zo);
-            if (TAIL && tail_tile) {
-              const int slot = slot0 + 16 * i;
-              if (slot >= a.tail_lo && slot < a.t_phys) o = bf16x8_to_h8(tv[TAIL ? i : 0]);
-            }
+            const uint4 o = dequant_word_h(wd[i], s2, zo);
             *reinterpret_cast<uint4*>(sgen + kOffV + vbuf * 16384 + row_off + i * 2048) = o;
           }
+          if (TAIL && tail_tile)
+            tail_rows_over(sgen + kOffV + vbuf * 16384 + row_off, a.v_tail + tail_off, a.tail_ts, slot0, a.tail_lo, a.t_phys);
           fence_proxy_async();
           mbar_arrive(b_vfull + 8 * vbuf);
           // The raw stage is released only here, after the words read from it have been used and

@@ -233,7 +233,9 @@ XKV_API int xkv_set_unquantised_tail(xkv_cache* cache, int32_t on);
  * Within a layer kv_append runs on a stream of the library's own (created on
  * first use, one per device) beside kv_score_evict, which does not depend on it;
  * both are ordered after everything already in `stream` and before the layer's
- * kv_quant_pack, and a layer starts only after the previous layer's attention. */
+ * kv_quant_pack, and a layer starts only after the previous layer's attention.
+ * The library's stream and its events are shared by every cache on the device:
+ * call the stream-step functions of one device from one host thread at a time. */
 XKV_API int xkv_stream_step(xkv_cache* const* layers, int32_t n_layers,
                     const void* const* q, const void* const* k, const void* const* v,
                     void* const* out, int32_t n, int64_t tok_stride, int64_t head_stride,

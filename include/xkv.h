@@ -234,6 +234,10 @@ XKV_API int xkv_set_unquantised_tail(xkv_cache* cache, int32_t on);
  * first use, one per device) beside kv_score_evict, which does not depend on it;
  * both are ordered after everything already in `stream` and before the layer's
  * kv_quant_pack, and a layer starts only after the previous layer's attention.
+ * After kv_quant_pack the step also computes, on that stream and beside the
+ * attention, the head means of the cached keys (Eq. 4) into the cache's workspace;
+ * the next frame's scoring of the same cache starts from them (same bits as
+ * kv_score_evict computes).  `stream` waits for these kernels at the end of the call.
  * The library's stream and its events are shared by every cache on the device:
  * call the stream-step functions of one device from one host thread at a time. */
 XKV_API int xkv_stream_step(xkv_cache* const* layers, int32_t n_layers,
@@ -284,7 +288,8 @@ XKV_API const char* xkv_strerror(int status);
  * *out and clears them. */
 enum { XKV_PROF_APPEND = 0, XKV_PROF_POOL = 1, XKV_PROF_SCORE = 2, XKV_PROF_SELECT = 3,
        XKV_PROF_REGROUP = 4, XKV_PROF_GATHER = 5, XKV_PROF_ATTN = 6, XKV_PROF_COMBINE = 7,
-       XKV_PROF_CATEGORIES = 8 };
+       XKV_PROF_KBAR = 8,   /* head means of the keys, computed by the stream step beside the attention */
+       XKV_PROF_CATEGORIES = 9 };
 typedef struct {
   double  ms[XKV_PROF_CATEGORIES];        /* summed device time per category, milliseconds */
   int64_t launches[XKV_PROF_CATEGORIES];  /* launches per category                         */

@@ -18,7 +18,7 @@ constexpr size_t kAlign = 256;
 struct Layout {
   int cap, row_bytes;
   size_t off_k[2], off_kpar[2], off_v[2], off_vpar[2], off_origin[2];
-  size_t off_kstage, off_qbar, off_qvec, off_scores, off_kept, off_counters, off_status, off_attn, off_hist;
+  size_t off_kstage, off_qbar, off_qvec, off_scores, off_kept, off_counters, off_status, off_attn, off_hist, off_kbar;
   size_t attn_bytes;
   size_t total;
 };
@@ -62,6 +62,7 @@ Layout make_layout(const xkv_params* p) {
   L.off_qvec = take(64 * sizeof(float));
   L.off_scores = take((size_t)L.cap * sizeof(float));
   L.off_kept = take((size_t)L.cap * sizeof(int32_t));
+  L.off_kbar = take((size_t)L.cap * 64 * sizeof(float));
   L.attn_bytes = attn_tc_scratch_bytes(p);
   L.off_attn = take(L.attn_bytes);
   L.total = off;
@@ -79,6 +80,7 @@ void reset_host_state(xkv_cache* c) {
   c->frames = c->T = c->T_first = c->rest_base = c->cur = c->stage = 0;
   c->n_pending = c->kk_pending = c->rold_pending = c->evict_pending = c->first_pending = 0;
   c->last_evicted = c->last_kept = c->last_prunable = 0;
+  c->kbar_T = c->kbar_cur = c->kbar_frames = -1;
 }
 
 }  // namespace
@@ -125,6 +127,7 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
   c->kept = reinterpret_cast<int32_t*>(c->ws + L.off_kept);
   c->counters = reinterpret_cast<unsigned int*>(c->ws + L.off_counters);
   c->sel_hist = reinterpret_cast<unsigned int*>(c->ws + L.off_hist);
+  c->kbar = reinterpret_cast<float*>(c->ws + L.off_kbar);
   c->status = reinterpret_cast<int*>(c->ws + L.off_status);
   c->attn_part = reinterpret_cast<float*>(c->ws + L.off_attn);
   c->attn_part_bytes = L.attn_bytes;
@@ -137,14 +140,18 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
   }
   c->prof = new (std::nothrow) Profiler;
   if (!c->prof) { delete c; return XKV_E_NOMEM; }
+  if (cudaEventCreateWithFlags(&c->kbar_done, cudaEventDisableTiming) != cudaSuccess) {
+    delete c->prof; delete c; return XKV_E_CUDA;
+  }
   const int rc = zero_workspace(c, reinterpret_cast<cudaStream_t>(stream));
-  if (rc != XKV_OK) { delete c->prof; delete c; return rc; }
+  if (rc != XKV_OK) { cudaEventDestroy(c->kbar_done); delete c->prof; delete c; return rc; }
   *out = c;
   return XKV_OK;
 }
 
 int xkv_reset(xkv_cache* c, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;
+  if (c->kbar_done) cudaEventSynchronize(c->kbar_done);      // a head-mean kernel of the last stream step
   reset_host_state(c);
   return zero_workspace(c, reinterpret_cast<cudaStream_t>(stream));
 }
@@ -156,6 +163,7 @@ int xkv_destroy(xkv_cache* c) {
     for (auto& e : c->prof->pool) cudaEventDestroy(e);
     delete c->prof;
   }
+  if (c->kbar_done) { cudaEventSynchronize(c->kbar_done); cudaEventDestroy(c->kbar_done); }
   delete c;
   return XKV_OK;
 }
@@ -186,7 +194,10 @@ int kv_append(xkv_cache* c, const void* k, const void* v, int32_t n, int64_t ts,
   return XKV_OK;
 }
 
-int kv_score_evict(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t hs, xkv_stream stream) {
+// use_kbar: the stream step has computed the head means of the current cache beside the previous
+// attention (and made `stream` wait for them); the scoring then starts from those.
+static int score_evict_on(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t hs, xkv_stream stream,
+                          bool use_kbar) {
   if (!c) return XKV_E_INVALID;
   if (c->stage != 1) return XKV_E_STATE;
   if (n != c->n_pending || !aligned16(q) || !strides_ok(ts, hs)) return XKV_E_INVALID;
@@ -199,12 +210,18 @@ int kv_score_evict(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t h
     c->last_evicted = r_old - kk;
     if (kk > 0 && kk < r_old) {
       if (launch_pool_q(c, q, n, ts, hs, st) != cudaSuccess) return XKV_E_CUDA;
-      if (launch_score(c, r_old, st) != cudaSuccess) return XKV_E_CUDA;
+      const bool from_kbar = use_kbar && c->kbar_T == c->T && c->kbar_cur == c->cur && c->kbar_frames == c->frames &&
+                             r_old == c->T - c->T_first;
+      if (launch_score(c, r_old, st, from_kbar) != cudaSuccess) return XKV_E_CUDA;
       if (launch_select(c, r_old, kk, st) != cudaSuccess) return XKV_E_CUDA;
     }
   }
   c->stage = 2;
   return XKV_OK;
+}
+
+int kv_score_evict(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t hs, xkv_stream stream) {
+  return score_evict_on(c, q, n, ts, hs, stream, false);
 }
 
 int kv_quant_pack(xkv_cache* c, xkv_stream stream) {
@@ -335,16 +352,42 @@ int run_layer(HostStepPipe* pipe, xkv_cache* c, const void* q, const void* k, co
   if (!ok) return XKV_E_CUDA;
   int rc = kv_append(c, k, v, n, ts, hs, reinterpret_cast<xkv_stream>(pipe->side));
   ok = cudaEventRecord(pipe->join, pipe->side) == cudaSuccess;
-  if (rc == XKV_OK && ok) rc = kv_score_evict(c, q, n, ts, hs, stream);
+  if (rc == XKV_OK && ok) {
+    const bool have_kbar = c->kbar_frames == c->frames && c->kbar_T == c->T && c->kbar_cur == c->cur;
+    if (have_kbar && cudaStreamWaitEvent(st, c->kbar_done, 0) != cudaSuccess) ok = false;
+    if (ok) rc = score_evict_on(c, q, n, ts, hs, stream, have_kbar);
+  }
   // the join is made also after an error, so that the side stream is never left behind
   ok = ok && cudaStreamWaitEvent(st, pipe->join, 0) == cudaSuccess;
   if (rc != XKV_OK) return rc;
   if (!ok) return XKV_E_CUDA;
   rc = kv_quant_pack(c, stream);
   if (rc != XKV_OK) return rc;
+  // Head means of the keys of the cache just built (Eq. 4), for the next frame's scoring: on the
+  // side stream, beside the attention.  Not for the first frame (nothing after it yet).
+  if (c->T > c->T_first) {
+    ok = cudaEventRecord(pipe->fork, st) == cudaSuccess && cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess;
+    if (!ok) return XKV_E_CUDA;
+    const bool launched = launch_kbar(c, pipe->side) == cudaSuccess;
+    ok = cudaEventRecord(c->kbar_done, pipe->side) == cudaSuccess;
+    // (the caller's stream waits for it at the end of the stream-step call, and at the next
+    // frame's scoring)
+    if (!launched || !ok) return XKV_E_CUDA;
+    c->kbar_T = c->T; c->kbar_cur = c->cur; c->kbar_frames = c->frames;
+  }
   const float scale = 1.0f / sqrtf((float)c->p.head_dim);
-  if (c->tail_mode) return attn_packed_causal_tail(c, q, k, v, out, n, ts, hs, scale, stream);
-  return attn_packed_causal(c, q, out, n, ts, hs, scale, 0, stream);
+  return c->tail_mode ? attn_packed_causal_tail(c, q, k, v, out, n, ts, hs, scale, stream)
+                      : attn_packed_causal(c, q, out, n, ts, hs, scale, 0, stream);
+}
+
+// Everything a stream-step call started on the side stream is ordered before what the caller
+// enqueues next: the caller's stream waits for the head-mean kernels of all layers.
+bool join_side_work(xkv_cache* const* layers, int n_layers, cudaStream_t st) {
+  bool ok = true;
+  for (int l = 0; l < n_layers; ++l)
+    if (layers[l] && layers[l]->kbar_frames == layers[l]->frames && layers[l]->kbar_frames > 0)
+      ok = cudaStreamWaitEvent(st, layers[l]->kbar_done, 0) == cudaSuccess && ok;
+  return ok;
 }
 
 }  // namespace
@@ -359,9 +402,9 @@ int xkv_stream_step(xkv_cache* const* layers, int32_t n_layers, const void* cons
     xkv_cache* c = layers[l];
     if (!c) return XKV_E_INVALID;
     const int rc = run_layer(pipe, c, q[l], k[l], v[l], out[l], n, ts, hs, reinterpret_cast<cudaStream_t>(stream));
-    if (rc != XKV_OK) return rc;
+    if (rc != XKV_OK) { join_side_work(layers, l + 1, reinterpret_cast<cudaStream_t>(stream)); return rc; }
   }
-  return XKV_OK;
+  return join_side_work(layers, n_layers, reinterpret_cast<cudaStream_t>(stream)) ? XKV_OK : XKV_E_CUDA;
 }
 
 size_t xkv_stream_step_host_bytes(const xkv_params* params, int32_t n) {
@@ -424,6 +467,7 @@ int xkv_stream_step_host(xkv_cache* const* layers, int32_t n_layers, const void*
     ck(cudaEventRecord(pipe->down_done[sl], pipe->down));
   }
   // everything started above ends before the call returns, also after an error
+  if (!join_side_work(layers, n_layers, st)) cuda_ok = false;
   ck(cudaStreamSynchronize(pipe->up));
   ck(cudaStreamSynchronize(st));
   ck(cudaStreamSynchronize(pipe->down));

@@ -64,6 +64,11 @@ struct xkv_cache {
   long long launches;
   int force_plain;         // 1: kernels take the plain (conversion-based) arithmetic forms everywhere
   int tail_mode;           // 1: the stream-step calls attend with the step's K, V unquantised
+  // head means of the keys after the first frame (Eq. 4), filled by the stream step beside the
+  // attention and used by the next step's scoring when the cache has not changed since
+  float* kbar;             // [cap][64]
+  cudaEvent_t kbar_done;
+  int kbar_T, kbar_cur, kbar_frames;   // state of the cache the array was computed from (-1: none)
   xkv::Profiler* prof;
 };
 
@@ -96,7 +101,8 @@ struct LaunchScope {
 cudaError_t launch_append(xkv_cache* c, const void* k, const void* v, int n, int64_t ts, int64_t hs,
                           int dst_slot, bool first, cudaStream_t st);
 cudaError_t launch_pool_q(xkv_cache* c, const void* q, int n, int64_t ts, int64_t hs, cudaStream_t st);
-cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st);
+cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st, bool from_kbar = false);
+cudaError_t launch_kbar(xkv_cache* c, cudaStream_t st);
 cudaError_t launch_select(xkv_cache* c, int r_old, int k, cudaStream_t st);
 cudaError_t launch_pack(xkv_cache* c, int n, int kk, bool identity, bool first, cudaStream_t st);
 cudaError_t launch_attn_simple(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,

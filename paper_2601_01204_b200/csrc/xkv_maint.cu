@@ -306,10 +306,15 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 
 constexpr int kSelBins = 4096;          // histogram of the top 12 key bits, filled by the score kernel
 
-template <int BITS>
+// MODE 0: the whole computation.  MODE 1: only Eq. 4, the head means K-bar[i][c] (fp32, exactly the
+// value MODE 0 holds at that point) stored to `kbar` -- run beside the attention of the step that
+// built the cache.  MODE 2: only Eq. 5-6 from a stored K-bar -- the next step's scoring.  1 + 2
+// perform the operations of 0 in the same order, so the scores are the same bits.
+template <int BITS, int MODE>
 __global__ void __launch_bounds__(512)
 score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* __restrict__ qvec,
-             float* __restrict__ scores, unsigned int* __restrict__ hist, int force_plain) {
+             float* __restrict__ scores, unsigned int* __restrict__ hist, int force_plain,
+             float* __restrict__ kbar) {
   // Parameters of the CTA's key group.  Fast path: float4 [H][4][8] = (s, magic + z) of channels
   // 8w + 2v and 8w + 2v + 1 at [h][v][w], so that the eight lanes of a quarter-warp read
   // consecutive 16-byte chunks.  Plain path: float2 (s, z) [H][64].
@@ -322,7 +327,7 @@ score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* 
   const int slot = rest_base + i;
   const int grp = (rest_base >> 6) + blockIdx.x;
   bool plain = false;
-  if (BITS == 4) {
+  if (BITS == 4 && MODE != 2) {
     int big = force_plain;
     float2 mine[4];                              // H <= 64: at most 8 elements per thread, 4 at a time
     for (int e0 = 0; e0 < H * 64; e0 += 2048) {
@@ -357,14 +362,14 @@ score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* 
       }
     }
   }
-  if (tid < 64) s_w[tid] = qvec[tid];
+  if (MODE != 1 && tid < 64) s_w[tid] = qvec[tid];
   __syncthreads();
   const bool valid = i < r_old;
   float acc[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) acc[j] = 0.f;
   constexpr int kHB = (BITS == 4) ? 16 : 4;     // heads whose words are in flight together
-  for (int h0 = 0; h0 < H; h0 += kHB) {
+  for (int h0 = 0; MODE != 2 && h0 < H; h0 += kHB) {
     uint32_t word[BITS == 4 ? kHB : 1];
     uint4 wide[BITS == 4 ? 1 : kHB];
 #pragma unroll
@@ -404,9 +409,26 @@ score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* 
     }
   }
   const float inv_h = __fdiv_rn(1.f, (float)H);
+  float kb[8];
+  if (MODE == 2) {
+    const float4* src = reinterpret_cast<const float4*>(kbar + (size_t)(valid ? i : 0) * 64 + 8 * w);
+    const float4 x = src[0], y = src[1];
+    kb[0] = x.x; kb[1] = x.y; kb[2] = x.z; kb[3] = x.w; kb[4] = y.x; kb[5] = y.y; kb[6] = y.z; kb[7] = y.w;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) kb[j] = __fmul_rn(acc[j], inv_h);
+  }
+  if (MODE == 1) {
+    if (valid) {
+      float4* dst = reinterpret_cast<float4*>(kbar + (size_t)i * 64 + 8 * w);
+      dst[0] = make_float4(kb[0], kb[1], kb[2], kb[3]);
+      dst[1] = make_float4(kb[4], kb[5], kb[6], kb[7]);
+    }
+    return;
+  }
   float p[8];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) p[j] = __fmul_rn(__fmul_rn(acc[j], inv_h), s_w[8 * w + j]);
+  for (int j = 0; j < 8; ++j) p[j] = __fmul_rn(kb[j], s_w[8 * w + j]);
   float t0 = __fadd_rn(p[0], p[1]), t1 = __fadd_rn(p[2], p[3]);
   float t2 = __fadd_rn(p[4], p[5]), t3 = __fadd_rn(p[6], p[7]);
   t0 = __fadd_rn(t0, t1);
@@ -420,16 +442,43 @@ score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* 
   }
 }
 
-cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st) {
+cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st, bool from_kbar) {
   const int blocks = (r_old + 63) / 64;
   const size_t smem = (size_t)c->p.n_heads * 64 * sizeof(float2);
   LaunchScope ls(c, XKV_PROF_SCORE, st);
+  const BufSet& b = c->buf[c->cur];
+  const int H = c->p.n_heads;
+  if (from_kbar) {
+    if (c->p.kv_bits == 16)
+      score_kernel<16, 2><<<blocks, 512, smem, st>>>(b, H, c->cap, c->rest_base, r_old, c->qvec, c->scores, c->sel_hist,
+                                                     c->force_plain, c->kbar);
+    else
+      score_kernel<4, 2><<<blocks, 512, smem, st>>>(b, H, c->cap, c->rest_base, r_old, c->qvec, c->scores, c->sel_hist,
+                                                    c->force_plain, c->kbar);
+  } else if (c->p.kv_bits == 16) {
+    score_kernel<16, 0><<<blocks, 512, smem, st>>>(b, H, c->cap, c->rest_base, r_old, c->qvec, c->scores, c->sel_hist,
+                                                   c->force_plain, nullptr);
+  } else {
+    score_kernel<4, 0><<<blocks, 512, smem, st>>>(b, H, c->cap, c->rest_base, r_old, c->qvec, c->scores, c->sel_hist,
+                                                  c->force_plain, nullptr);
+  }
+  return cudaGetLastError();
+}
+
+// Head means of the keys after the first frame, of the cache as it stands (after kv_quant_pack).
+cudaError_t launch_kbar(xkv_cache* c, cudaStream_t st) {
+  const int r = c->T - c->T_first;
+  if (r <= 0) return cudaSuccess;
+  const int blocks = (r + 63) / 64;
+  const size_t smem = (size_t)c->p.n_heads * 64 * sizeof(float2);
+  LaunchScope ls(c, XKV_PROF_KBAR, st);
+  const BufSet& b = c->buf[c->cur];
   if (c->p.kv_bits == 16)
-    score_kernel<16><<<blocks, 512, smem, st>>>(c->buf[c->cur], c->p.n_heads, c->cap, c->rest_base, r_old,
-                                                c->qvec, c->scores, c->sel_hist, c->force_plain);
+    score_kernel<16, 1><<<blocks, 512, smem, st>>>(b, c->p.n_heads, c->cap, c->rest_base, r, nullptr, nullptr, nullptr,
+                                                   c->force_plain, c->kbar);
   else
-    score_kernel<4><<<blocks, 512, smem, st>>>(c->buf[c->cur], c->p.n_heads, c->cap, c->rest_base, r_old,
-                                               c->qvec, c->scores, c->sel_hist, c->force_plain);
+    score_kernel<4, 1><<<blocks, 512, smem, st>>>(b, c->p.n_heads, c->cap, c->rest_base, r, nullptr, nullptr, nullptr,
+                                                  c->force_plain, c->kbar);
   return cudaGetLastError();
 }
 

@@ -35,7 +35,7 @@ EXPORTED = [
     "xkv_synth_fill", "xkv_profile_enable", "xkv_profile_read", "attn_packed_causal_static",
     "xkv_debug_rewind_attention", "attn_packed_causal_tail", "xkv_set_unquantised_tail",
 ]
-PROF_NAMES = ["append", "pool_q", "score", "select", "regroup_k", "gather", "attn", "attn_combine"]
+PROF_NAMES = ["append", "pool_q", "score", "select", "regroup_k", "gather", "attn", "attn_combine", "kbar"]
 
 
 class xkv_params(C.Structure):
@@ -50,7 +50,7 @@ class xkv_info(C.Structure):
 
 
 class xkv_profile(C.Structure):
-    _fields_ = [("ms", C.c_double * 8), ("launches", C.c_int64 * 8)]
+    _fields_ = [("ms", C.c_double * 9), ("launches", C.c_int64 * 9)]
 
 
 _vp, _i32, _i64, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t

@@ -161,6 +161,40 @@ def test_synth_kernel_matches_numpy_generator(xkv):
         assert np.array_equal(got, synth.gen_tensor_bits(9, 2, 5, tensor, H, n, d))
 
 
+@pytest.mark.parametrize("bits", [4, 16])
+def test_stream_step_scoring_from_stored_head_means(xkv, bits):
+    """The stream step computes the head means of the keys (Eq. 4) beside the attention and the next
+    frame's scoring starts from them; the per-call sequence computes them inside the scoring.  Both
+    must give the same bits: scores, kept indices, the whole packed state and the outputs, frame
+    after frame, also across a reset."""
+    import torch
+    L, H, n, d = 2, 4, 150, 64
+    p = xkv.Params(n_heads=H, budget=400, max_frame_tokens=n, kv_bits=bits)
+    step_caches = [xkv.Cache(p) for _ in range(L)]
+    call_caches = [xkv.Cache(p) for _ in range(L)]
+    for rnd in range(2):
+        for t in range(6):
+            frames = [synth.gen_frame(51 + rnd, l, t, H, n, d) for l in range(L)]
+            q, k, v = ([to_device_bf16(f[i]) for f in frames] for i in range(3))
+            out = [torch.empty_like(x) for x in q]
+            xkv.xkv_stream_step(step_caches, q, k, v, out)
+            for l, c in enumerate(call_caches):
+                c.kv_append(k[l], v[l]); c.kv_score_evict(q[l]); c.kv_quant_pack()
+                ref = c.attn_packed_causal(q[l])
+                torch.cuda.synchronize()
+                assert torch.equal(out[l].view(torch.int16), ref.view(torch.int16)), (rnd, t, l)
+                ia, ib = step_caches[l].xkv_get_info(), c.xkv_get_info()
+                assert (ia.T, ia.last_kept, ia.last_evicted) == (ib.T, ib.last_kept, ib.last_evicted)
+                if ib.last_evicted > 0:
+                    for buf, nb in ((xkv.BUF_SCORES, ib.last_prunable * 4), (xkv.BUF_KEPT, ib.last_kept * 4)):
+                        assert np.array_equal(step_caches[l].xkv_debug_export(buf, nb), c.xkv_debug_export(buf, nb)), (rnd, t, l)
+                ea, eb = step_caches[l].export(), c.export()
+                assert all(np.array_equal(np.asarray(ea[key]), np.asarray(eb[key])) for key in eb), (rnd, t, l)
+        assert step_caches[0].xkv_get_info().last_evicted > 0
+        for c in step_caches + call_caches:
+            c.xkv_reset()
+
+
 def test_stream_step_with_unquantised_tail_option(xkv):
     """xkv_set_unquantised_tail(1): the stream step gives what the per-call sequence with
     attn_packed_causal_tail gives, bit for bit."""

@@ -50,7 +50,14 @@ Pins (tests/test_oracle_*.py): worked quantiser example derived from Eq. 7-8,
 error bound s/2, brute-force top-k, GEMV special case of the score, linearity,
 streaming == one-shot frame-causal attention when nothing is pruned or
 quantised, library softmax-attention on CPU, T = 1 and uniform-key closed
-forms, pack/unpack vectors.  The reading "re-quantise changed groups" is a
+forms, pack/unpack vectors.  The stateful composition under pruning
+(OracleLayer.score_evict, OracleLayer.quant_pack) is pinned in
+tests/test_oracle_eviction_pins.py: survivors' value codes equal the
+quantisation of the raw rows their origins name, cached keys stay within the
+accumulated s/2 bound of those raw rows, scores equal the literal Eq. 2-6 on
+the cache as it stood before the step, the regroup rule on crafted steps; the
+same file plants a dozen bookkeeping mistakes in copies of this source and
+requires each to fail a pin.  The reading "re-quantise changed groups" is a
 choice, not something the paper fixes: parity unpinned for that reading only.
 """
 from __future__ import annotations

@@ -20,7 +20,7 @@
  *     the rest its patch tokens in raster order (Sec. 3.1).
  *   - Calls are stream-ordered and never synchronise, allocate device memory or
  *     read device data on the host (exceptions: xkv_debug_export,
- *     xkv_poll_status, xkv_stream_step_host).  All cache lengths are functions
+ *     xkv_poll_status, xkv_profile_read, xkv_stream_step_host).  All cache lengths are functions
  *     of the frame sizes seen so far and the budget, so they are tracked on the
  *     host.
  *   - The caller owns the workspace; the library never frees it.  Memory use of
@@ -56,7 +56,9 @@ typedef enum {
   XKV_E_UNSUPPORTED = -4,   /* parameter combination not implemented                   */
   XKV_E_CUDA        = -5,   /* a CUDA runtime/driver call failed                       */
   XKV_E_TIMEOUT     = -6,   /* a bounded device-side wait ran out (see xkv_poll_status)*/
-  XKV_E_LIMIT       = -7    /* the call needs more than a fixed built-in limit allows   */
+  XKV_E_LIMIT       = -7,   /* the call needs more than a fixed built-in limit allows   */
+  XKV_E_RANGE       = -8    /* a value left the range of the 16-bit tensor-core operands */
+                            /* (see attn_packed_causal and xkv_poll_status)             */
 } xkv_status;
 
 /* Method parameters.  Defaults of the paper: n_special = 5 (1 camera + 4
@@ -121,7 +123,9 @@ XKV_API size_t xkv_workspace_bytes(const xkv_params* params);
 XKV_API int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes,
                xkv_stream stream, xkv_cache** out);
 
-/* Back to the empty state on the same workspace (stream-ordered zero-fill). */
+/* Back to the empty state on the same workspace (stream-ordered zero-fill, which also clears the
+ * device status word).  `stream` is made to wait for any kernel that a stream step of this cache
+ * still has in flight on the library's own stream; the host does not wait. */
 XKV_API int xkv_reset(xkv_cache* cache, xkv_stream stream);
 
 /* Free the host handle.  The workspace stays with the caller. */
@@ -160,8 +164,21 @@ XKV_API int kv_quant_pack(xkv_cache* cache, xkv_stream stream);
  * softmax_scale) V~ per head over all T cached tokens (all of them belong to
  * frames <= t, so the frame-causal mask hides nothing).  out has the strides of
  * q.  impl: 0 = default (tensor-core kernel), 1 = the simple CUDA-core kernel
- * kept as a cross-check.  Errors: XKV_E_STATE unless kv_quant_pack was the
- * previous call (the cache returns to idle); XKV_E_INVALID as above. */
+ * kept as a cross-check (fp32 throughout).  Errors: XKV_E_STATE unless kv_quant_pack was the
+ * previous call (the cache returns to idle); XKV_E_INVALID as above.
+ *
+ * Operand range of the tensor-core kernel.  A 4-bit cache is multiplied in fp16 with fp32
+ * accumulation: q, the dequantised keys and values x~ = s*q_code + (-s*z) (Eq. 10, the constant
+ * formed in fp32 per group and channel resp. per token) and the softmax weights are rounded to
+ * fp16, i.e. to 11 significant bits, with fp16's floor of 6e-8 on the absolute resolution.  Any
+ * integer zero-point and any scale are accepted.  What fp16 cannot hold is a magnitude above
+ * 65504: if a query element, a dequantised key or value, or (tail variant) a raw key or value
+ * of the newest frame exceeds it, the kernel records XKV_E_RANGE in the cache's status word
+ * (xkv_poll_status) and the output of that call is unspecified; impl = 1 has no such limit.
+ * A 16-bit cache is multiplied in bf16 and has no range limit.  Keys whose spread within a
+ * 64-token group is far below the resolution of a 16-bit number at their magnitude (a large
+ * common offset, a tiny range) lose that spread in any 16-bit operand: the result then
+ * carries the error of rounding x~ to 11 bits, no more. */
 XKV_API int attn_packed_causal(xkv_cache* cache, const void* q, void* out, int32_t n,
                        int64_t tok_stride, int64_t head_stride, float softmax_scale,
                        int32_t impl, xkv_stream stream);
@@ -202,13 +219,13 @@ XKV_API int attn_packed_causal_tail(xkv_cache* cache, const void* q, const void*
  *   - Same arguments, state requirements and result as attn_packed_causal with
  *     impl = 0; q and out are still the caller's.
  *   - The need does not grow with the frame or the cache: each thread block
- *     leaves at most two partial slots of 135 168 bytes, and the kernel runs one
- *     block per multiprocessor.  The array holds XKV_STATIC_SCRATCH_BYTES /
- *     135 168 = 248 slots; on a GPU with more than 124 multiprocessors the
- *     variant launches 124 blocks instead of one per multiprocessor (slower,
- *     same result).  If not even one block's slots fit, the call returns
- *     XKV_E_LIMIT before anything is enqueued and the cache stays in the packed
- *     state, so attn_packed_causal can still take the frame.
+ *     leaves at most two partial slots of 67 584 bytes (two query tiles of 128 rows, 64
+ *     accumulators plus running max and sum each), and the kernel runs one block per
+ *     multiprocessor.  The array holds XKV_STATIC_SCRATCH_BYTES / 67 584 = 496 slots, enough
+ *     for 248 blocks; a GPU with more multiprocessors than that would run 248 blocks (each
+ *     item of work cut into fewer, longer pieces: slower, same result).  A B200 has 148.
+ *     XKV_E_LIMIT is returned, before anything is enqueued and with the cache left in the
+ *     packed state, only if not even one block's slots fit.
  *   - The first call on a device looks up the array's device address (once per
  *     device, with that device current).  Make that first call outside any
  *     stream capture.
@@ -229,7 +246,8 @@ XKV_API int xkv_set_unquantised_tail(xkv_cache* cache, int32_t on);
 
 /* One frame through a stack of layers: for each layer in order, the four calls
  * above with softmax_scale = 1/sqrt(head_dim).  q, k, v, out are HOST arrays of
- * n_layers DEVICE pointers.  Stops at the first error and returns it.
+ * n_layers DEVICE pointers.  Stops at the first error and returns it; the layer that failed
+ * may then be left between two of its four calls, and the only way on is xkv_reset.
  * Within a layer kv_append runs on a stream of the library's own (created on
  * first use, one per device) beside kv_score_evict, which does not depend on it;
  * both are ordered after everything already in `stream` and before the layer's
@@ -274,11 +292,31 @@ XKV_API int64_t xkv_debug_export(const xkv_cache* cache, int32_t which, void* ho
  * cache contents (with the same or other queries).  XKV_E_STATE otherwise. */
 XKV_API int xkv_debug_rewind_attention(xkv_cache* cache);
 
-/* Synchronises `stream` and returns the device status word of the cache:
- * XKV_OK, or XKV_E_TIMEOUT if a bounded wait inside a kernel ran out. */
+/* Synchronises `stream` and returns the device status word of the cache: XKV_OK,
+ * XKV_E_TIMEOUT if a bounded wait inside a kernel ran out (the kernel still ended in order: it
+ * drained its copies and freed its tensor memory; results of that call are void), or
+ * XKV_E_RANGE (see attn_packed_causal).  The word is sticky until xkv_reset. */
 XKV_API int xkv_poll_status(const xkv_cache* cache, xkv_stream stream);
 
 XKV_API const char* xkv_strerror(int status);
+
+/* ---- test hooks (per cache; no environment variables, no process-wide switches) ---------- */
+
+/* Tests only.  The maintenance kernels evaluate Eq. 7 and Eq. 10 in conversion-free forms when
+ * the zero-points and scaled values of a group are small enough, and in the plain forms
+ * otherwise; on = 1 makes every kernel of this cache take the plain forms everywhere. */
+XKV_API int xkv_debug_force_plain(xkv_cache* cache, int32_t on);
+
+/* Tests only.  Caps the number of thread blocks of the tensor-core attention of this cache
+ * (0 = no cap: one block per multiprocessor).  With fewer blocks every item of work is cut into
+ * fewer, longer pieces and a block may cover several items; the result does not change. */
+XKV_API int xkv_debug_limit_attention_blocks(xkv_cache* cache, int32_t max_blocks);
+
+/* Tests only.  Launches one small thread block that waits, with the attention kernel's bounded
+ * wait, on a barrier that nothing will ever complete.  The wait gives up after its iteration
+ * limit (a fraction of a second), the kernel ends normally and the cache's status word reads
+ * XKV_E_TIMEOUT at the next xkv_poll_status; xkv_reset clears it.  Nothing faults or hangs. */
+XKV_API int xkv_debug_timeout_probe(xkv_cache* cache, xkv_stream stream);
 
 /* Optional per-kernel timing for benchmarks.  While enabled, every kernel the
  * library launches for this cache is bracketed by a pair of CUDA events on the

@@ -37,6 +37,11 @@ Readings taken where the paper is silent (each also listed in the design notes):
     carried over verbatim when it is complete and holds exactly the same
     tokens, in place, as before; every other rest group is re-quantised from
     the fp32 dequantised survivors and the fp32 new keys.
+  - key_mode = "once" is the other reading of Sec. 3.3 / Sec. 4.1 (the quantiser the paper
+    names quantises a group once): a frame's keys are quantised on arrival in groups of G
+    consecutive tokens of that frame (the last group of a frame may be partial), codes and
+    group parameters are never rewritten, a survivor carries a reference to its group's
+    parameters, and a group's parameters are dropped when its last token is evicted.
   - values are quantised once per (head, token) over the d channels.
   - rounding is to nearest, ties to even; x/s is evaluated as x * (1/s).
   - max == min in a group gives s = 1.
@@ -81,6 +86,11 @@ class OracleParams:
     quant_group: int = 64    # G, tokens per key group (Sec. 4.1)
     kv_bits: int = 4         # b; 16 = keep bf16 values (prune only)
     budget: int = 2048       # L_max
+    # how the per-channel key groups (Eq. 9) live with eviction:
+    #   "regroup": groups are runs of G cache positions; a group that changed is re-quantised
+    #   "once":    groups are runs of G arrival positions of one frame, quantised once when the
+    #              frame arrives (KIVI-style); a survivor keeps its codes and its group's (s, z)
+    key_mode: str = "regroup"
 
 
 # --------------------------------------------------------------------------
@@ -358,6 +368,10 @@ class OracleLayer:
         self.k_val = np.zeros((H, 0, d), dtype=F32)
         self.v_val = np.zeros((H, 0, d), dtype=F32)
         self.origin = np.zeros(0, dtype=np.int32)      # (frame << 16) | token
+        # key_mode "once": group id (frame << 16 | group within the frame) of every cached token and
+        # the parameter table {group id: (s [H][d], z [H][d])} of the groups that still have a token
+        self.k_gid = np.zeros(0, dtype=np.int64)
+        self.k_table = {}
         # pending (appended, not yet quantised) frame
         self._new_k = None
         self._new_v = None
@@ -385,10 +399,22 @@ class OracleLayer:
         p = self.p
         if p.kv_bits == 16:
             return self.k_val
+        if p.key_mode == "once":
+            s, z = self.key_params_per_token()
+            return dequantize(self.k_codes, s, z)
         Tf = self.T_first
         first = dequantize_keys(self.k_codes[:, :Tf], self.k_s_first, self.k_z_first, p.quant_group)
         rest = dequantize_keys(self.k_codes[:, Tf:], self.k_s_rest, self.k_z_rest, p.quant_group)
         return np.concatenate([first, rest], axis=1)
+
+    def key_params_per_token(self):
+        """key_mode "once": (s, z) fp32 [H][T][d], every token looked up through its group id."""
+        H, d = self.p.n_heads, self.p.head_dim
+        s = np.zeros((H, self.T, d), dtype=F32)
+        z = np.zeros((H, self.T, d), dtype=F32)
+        for i, g in enumerate(self.k_gid.tolist()):
+            s[:, i], z[:, i] = self.k_table[g]
+        return s, z
 
     def values_dequantized(self) -> np.ndarray:
         if self.p.kv_bits == 16:
@@ -445,6 +471,9 @@ class OracleLayer:
             self.origin = frame_origin
             if p.kv_bits == 16:
                 self.k_val, self.v_val = K_new, V_new
+            elif p.key_mode == "once":
+                self.k_codes = self._quantise_frame_keys_once(K_new)
+                self.v_codes, self.v_s, self.v_z = quantize_values(V_new, p.kv_bits)
             else:
                 self.k_codes, self.k_s_first, self.k_z_first = quantize_keys(K_new, G, p.kv_bits)
                 self.v_codes, self.v_s, self.v_z = quantize_values(V_new, p.kv_bits)
@@ -469,6 +498,19 @@ class OracleLayer:
         self.v_s = np.concatenate([self.v_s[:, keep_abs], vs], axis=1)
         self.v_z = np.concatenate([self.v_z[:, keep_abs], vz], axis=1)
 
+        if p.key_mode == "once":
+            # keys: survivors keep codes and group; the frame is quantised on its own; groups
+            # without a token left give their parameters back
+            gid_kept = self.k_gid[keep_abs]
+            codes_kept = self.k_codes[:, keep_abs]
+            self.k_gid = gid_kept
+            new_codes = self._quantise_frame_keys_once(K_new)
+            self.k_codes = np.concatenate([codes_kept, new_codes], axis=1)
+            live = set(self.k_gid.tolist())
+            self.k_table = {g: v for g, v in self.k_table.items() if g in live}
+            self._new_k = self._new_v = None
+            return
+
         # keys: regroup the rest segment
         old_codes = self.k_codes[:, Tf:]
         old_deq = dequantize_keys(old_codes, self.k_s_rest, self.k_z_rest, G)
@@ -492,6 +534,18 @@ class OracleLayer:
         self.k_codes = np.concatenate([self.k_codes[:, :Tf], new_codes], axis=1)
         self.k_s_rest, self.k_z_rest = new_s, new_z
         self._new_k = self._new_v = None
+
+    def _quantise_frame_keys_once(self, K_new: np.ndarray) -> np.ndarray:
+        """key_mode "once": Eq. 7-9 on the frame alone, groups of G tokens from its first token;
+        registers the groups' parameters and appends the tokens' group ids.  Returns the codes."""
+        p = self.p
+        n = K_new.shape[1]
+        codes, s, z = quantize_keys(K_new, p.quant_group, p.kv_bits)
+        base = np.int64(self.frames) << 16
+        for g in range(s.shape[1]):
+            self.k_table[int(base | g)] = (s[:, g].copy(), z[:, g].copy())
+        self.k_gid = np.concatenate([self.k_gid, base | (np.arange(n, dtype=np.int64) // p.quant_group)])
+        return codes
 
     # ---- step 5: attention over the packed cache ---------------------------
     def attend(self, Q: np.ndarray, scale: float | None = None, full_precision_tail: bool = False) -> np.ndarray:
@@ -533,7 +587,11 @@ class OracleLayer:
         else:
             out["k_packed"] = pack_nibbles(self.k_codes)
             out["v_packed"] = pack_nibbles(self.v_codes)
-            out["k_s_first"], out["k_z_first"] = self.k_s_first.copy(), self.k_z_first.copy()
-            out["k_s_rest"], out["k_z_rest"] = self.k_s_rest.copy(), self.k_z_rest.copy()
+            if p.key_mode == "once":
+                out["k_s_tok"], out["k_z_tok"] = self.key_params_per_token()
+                out["k_groups_live"] = len(self.k_table)
+            else:
+                out["k_s_first"], out["k_z_first"] = self.k_s_first.copy(), self.k_z_first.copy()
+                out["k_s_rest"], out["k_z_rest"] = self.k_s_rest.copy(), self.k_z_rest.copy()
             out["v_s"], out["v_z"] = self.v_s.copy(), self.v_z.copy()
         return out

@@ -73,8 +73,8 @@ template <> struct Cfg<16> {
 constexpr int kOffQ = 0;                          // 2 x 16 KB  Q tiles, K-major, SW128
 constexpr int kOffK = 32768;                      // kNK x 16 KB  K~ tiles
 constexpr int kOffV = kOffK + kNK * 16384;        // kNV x 16 KB  V~ tiles
-constexpr int kOffTab = kOffV + kNV * 16384;      // 2 x (K table 512 B + V table 2048 B) fp16 parameters
-constexpr int kTabBytes = 512 + 2048;
+constexpr int kOffTab = kOffV + kNV * 16384;      // 2 x (K table 768 B + V table 2048 B) fp16 parameters
+constexpr int kTabBytes = 768 + 2048;
 constexpr int kOffBar = kOffTab + 2 * kTabBytes;  // barriers, tmem base, abort flag
 constexpr int kBarBytes = 512;
 constexpr int kOffRaw = kOffBar + kBarBytes;      // raw stages (16-byte aligned)
@@ -296,31 +296,52 @@ __device__ __forceinline__ uint32_t h2_sub(uint32_t a, uint32_t b) {
   return r;
 }
 
-__device__ __forceinline__ uint32_t h2_mul(uint32_t a, uint32_t b) {
+
+__device__ __forceinline__ uint32_t h2_fma(uint32_t a, uint32_t b, uint32_t c) {
   uint32_t r;
-  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
   return r;
 }
 
-// Eight 4-bit codes of one packed word -> four fp16 pairs s * (q - z)  (Eq. 10).
-// (w & 0x000F000F) | 0x6400 is the fp16 number 1024 + q and (w & 0x00F000F0) | 0x5400 is 64 + q,
-// so one subtraction of (1024 + z) resp. (64 + z) gives q - z exactly (z is an integer), and one
-// multiplication by the fp16 scale follows.  zlo/zhi hold those two constants per channel pair:
-// pairs 0 and 2 of a word use the 1024 offset, pairs 1 and 3 the 64 offset.
-__device__ __forceinline__ uint4 dequant_word_h(uint32_t w, const uint32_t (&s2)[4], const uint32_t (&zo)[4]) {
+// Eight 4-bit codes of one packed word -> four fp16 pairs of s * (q - z)  (Eq. 10).
+// (w & 0x000F000F) | 0x6400 is the fp16 number 1024 + q and (w & 0x00F000F0) | 0x5400 is 64 + q.
+// Every pair is formed as  fma(biased - zo, s, c)  with constants chosen per group (dequant_consts):
+//   zo = bias + z, c = 0       when bias + z is an integer fp16 holds exactly (|bias + z| <= 2048):
+//                              the difference is q - z exactly and the product is rounded once;
+//   zo = bias,     c = -s z    otherwise (c formed in fp32): s q + c, valid for any zero-point.
+// Pairs 0 and 2 of a word carry the bias 1024, pairs 1 and 3 the bias 64.
+__device__ __forceinline__ uint4 dequant_word_h(uint32_t w, const uint32_t (&s2)[4], const uint32_t (&zo)[4],
+                                                const uint32_t (&c2)[4]) {
   const uint32_t t = w >> 8;
   const uint32_t a0 = (w & 0x000F000Fu) | 0x64006400u;
   const uint32_t a1 = (w & 0x00F000F0u) | 0x54005400u;
   const uint32_t a2 = (t & 0x000F000Fu) | 0x64006400u;
   const uint32_t a3 = (t & 0x00F000F0u) | 0x54005400u;
   uint4 r;
-  r.x = h2_mul(h2_sub(a0, zo[0]), s2[0]);
-  r.y = h2_mul(h2_sub(a1, zo[1]), s2[1]);
-  r.z = h2_mul(h2_sub(a2, zo[2]), s2[2]);
-  r.w = h2_mul(h2_sub(a3, zo[3]), s2[3]);
+  r.x = h2_fma(h2_sub(a0, zo[0]), s2[0], c2[0]);
+  r.y = h2_fma(h2_sub(a1, zo[1]), s2[1], c2[1]);
+  r.z = h2_fma(h2_sub(a2, zo[2]), s2[2], c2[2]);
+  r.w = h2_fma(h2_sub(a3, zo[3]), s2[3], c2[3]);
   return r;
 }
 
+// The constants of dequant_word_h for one (scale, zero-point): both biases must be exact for the
+// first form.  z is an integer-valued float (Eq. 8).
+__device__ __forceinline__ void dequant_consts(float s, float z, float& zo_1024, float& zo_64, float& c) {
+  const bool exact = fabsf(1024.f + z) <= 2048.f && fabsf(64.f + z) <= 2048.f;
+  zo_1024 = exact ? 1024.f + z : 1024.f;
+  zo_64 = exact ? 64.f + z : 64.f;
+  c = exact ? 0.f : -s * z;
+}
+
+// fp16 can hold magnitudes up to 65504; anything beyond (or not a number) is reported.
+__device__ __forceinline__ bool beyond_fp16(float x) { return !(fabsf(x) <= 65504.f); }
+__device__ __noinline__ void report_range(int* status) { atomicCAS(status, 0, (int)XKV_E_RANGE); }
+
+// true when one of the two fp16 numbers is an infinity or a NaN (all exponent bits set)
+__device__ __forceinline__ bool h2_not_finite(uint32_t h) {
+  return (h & 0x7C00u) == 0x7C00u || (h & 0x7C000000u) == 0x7C000000u;
+}
 
 // Eight bf16 values -> eight fp16 values (exact whenever the value is in fp16's range).
 __device__ __forceinline__ uint4 bf16x8_to_h8(const uint4& u) {
@@ -336,7 +357,7 @@ __device__ __forceinline__ uint4 bf16x8_to_h8(const uint4& u) {
 // (src already points at this thread's head and 8-channel chunk).  A real call, so that the
 // producers' loop carries none of this code.
 __device__ __noinline__ void tail_rows_over(uint8_t* tile_row, const __nv_bfloat16* src, int64_t ts, int slot0,
-                                            int tail_lo, int t_phys) {
+                                            int tail_lo, int t_phys, int* status) {
   uint4 u[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
@@ -347,7 +368,11 @@ __device__ __noinline__ void tail_rows_over(uint8_t* tile_row, const __nv_bfloat
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int slot = slot0 + 16 * i;
-    if (slot >= tail_lo && slot < t_phys) *reinterpret_cast<uint4*>(tile_row + i * 2048) = bf16x8_to_h8(u[i]);
+    if (slot >= tail_lo && slot < t_phys) {
+      const uint4 hv = bf16x8_to_h8(u[i]);
+      *reinterpret_cast<uint4*>(tile_row + i * 2048) = hv;
+      if (h2_not_finite(hv.x) || h2_not_finite(hv.y) || h2_not_finite(hv.z) || h2_not_finite(hv.w)) report_range(status);
+    }
   }
 }
 
@@ -407,7 +432,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
   const long long step_hi = piece_start(a.total, gridDim.x, blockIdx.x + 1);
 
   if (tid == 0) {
-    *abort_flag = (*reinterpret_cast<volatile int*>(a.status) != 0) ? 1 : 0;   // an earlier CTA already gave up
+    *abort_flag = (*reinterpret_cast<volatile int*>(a.status) == (int)XKV_E_TIMEOUT) ? 1 : 0;   // an earlier CTA already gave up
     for (int i = 0; i < kNK; ++i) { mbar_init(b_kfull + 8 * i, 128); mbar_init(b_kfree + 8 * i, 2); }
     for (int i = 0; i < kNV; ++i) { mbar_init(b_vfull + 8 * i, 128); mbar_init(b_vfree + 8 * i, 2); }
     for (int i = 0; i < C::kNR; ++i) { mbar_init(b_rfull + 8 * i, 1); mbar_init(b_rfree + 8 * i, 128); }
@@ -459,6 +484,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
 #pragma unroll
           for (int c = 0; c < 8; ++c) u[c] = make_uint4(0, 0, 0, 0);
         }
+        bool q_bad = false;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           uint4 o = u[c];
@@ -466,12 +492,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
             const uint32_t rr[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
             uint32_t hh[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < 4; ++i) {
               hh[i] = pack_h2(__uint_as_float(rr[i] << 16), __uint_as_float(rr[i] & 0xFFFF0000u));
+              q_bad |= h2_not_finite(hh[i]);
+            }
             o = make_uint4(hh[0], hh[1], hh[2], hh[3]);
           }
           *reinterpret_cast<uint4*>(sgen + kOffQ + t * 16384 + swz_off(r, c)) = o;
         }
+        if (q_bad) report_range(a.status);
         fence_proxy_async();
         mbar_arrive(b_qfull + 8 * t);
       }
@@ -699,16 +728,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           uint8_t* tab = sgen + kOffTab + (g & 1) * kTabBytes;
           {
             const float2 kp = *reinterpret_cast<const float2*>(raw + C::kRawK + C::kRawV + 8 * t);  // (group t>>6, channel t&63)
-            const int c = t & 63;
-            const float off = (((c & 7) >> 1) & 1) ? 64.f : 1024.f;
-            __half* ks = reinterpret_cast<__half*>(tab);              // [2][64] scales, then [2][64] offsets
+            float zl, zh, kc;
+            dequant_consts(kp.x, kp.y, zl, zh, kc);
+            __half* ks = reinterpret_cast<__half*>(tab);              // [2][64] scales, [2][64] offsets, [2][64] constants
             ks[t] = __float2half_rn(kp.x);
-            ks[128 + t] = __float2half_rn(off + kp.y);
+            ks[128 + t] = __float2half_rn((((t & 7) >> 1) & 1) ? zh : zl);
+            ks[256 + t] = __float2half_rn(kc);
             const float2 vp = *reinterpret_cast<const float2*>(raw + C::kRawK + C::kRawV + C::kRawKP + 8 * t);   // key t
-            const uint32_t s1 = pack_h2(vp.x, vp.x);
-            const uint32_t zl = pack_h2(1024.f + vp.y, 1024.f + vp.y);
-            const uint32_t zh = pack_h2(64.f + vp.y, 64.f + vp.y);
-            *reinterpret_cast<uint4*>(tab + 512 + 16 * t) = make_uint4(s1, zl, zh, 0u);
+            float vl, vh, vc;
+            dequant_consts(vp.x, vp.y, vl, vh, vc);
+            *reinterpret_cast<uint4*>(tab + 768 + 16 * t) =
+                make_uint4(pack_h2(vp.x, vp.x), pack_h2(vl, vl), pack_h2(vh, vh), pack_h2(vc, vc));
+            // largest magnitude a code of this group / token can dequantise to
+            if (beyond_fp16(fabsf(kp.x) * (fabsf(kp.y) + 15.f)) || beyond_fp16(fabsf(vp.x) * (fabsf(vp.y) + 15.f)))
+              report_range(a.status);
           }
           producer_sync();
           // ---- keys ----
@@ -720,15 +753,17 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           for (int grp = 0; grp < 2; ++grp) {
             const uint4 sv = *reinterpret_cast<const uint4*>(tab + grp * 128 + 16 * w);
             const uint4 zv = *reinterpret_cast<const uint4*>(tab + 256 + grp * 128 + 16 * w);
+            const uint4 cv = *reinterpret_cast<const uint4*>(tab + 512 + grp * 128 + 16 * w);
             const uint32_t s2[4] = {sv.x, sv.y, sv.z, sv.w}, zo[4] = {zv.x, zv.y, zv.z, zv.w};
+            const uint32_t c2[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              const uint4 o = dequant_word_h(wd[4 * grp + i], s2, zo);
+              const uint4 o = dequant_word_h(wd[4 * grp + i], s2, zo, c2);
               *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (4 * grp + i) * 2048) = o;
             }
           }
           if (TAIL && tail_tile)
-            tail_rows_over(sgen + kOffK + kbuf * 16384 + row_off, a.k_tail + tail_off, a.tail_ts, slot0, a.tail_lo, a.t_phys);
+            tail_rows_over(sgen + kOffK + kbuf * 16384 + row_off, a.k_tail + tail_off, a.tail_ts, slot0, a.tail_lo, a.t_phys, a.status);
           fence_proxy_async();
           mbar_arrive(b_kfull + 8 * kbuf);
           // ---- values ----
@@ -737,13 +772,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           mbar_wait<256>(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const uint4 pv = *reinterpret_cast<const uint4*>(tab + 512 + 16 * (kb + 16 * i));
+            const uint4 pv = *reinterpret_cast<const uint4*>(tab + 768 + 16 * (kb + 16 * i));
             const uint32_t s2[4] = {pv.x, pv.x, pv.x, pv.x}, zo[4] = {pv.y, pv.z, pv.y, pv.z};
-            const uint4 o = dequant_word_h(wd[i], s2, zo);
+            const uint32_t c2[4] = {pv.w, pv.w, pv.w, pv.w};
+            const uint4 o = dequant_word_h(wd[i], s2, zo, c2);
             *reinterpret_cast<uint4*>(sgen + kOffV + vbuf * 16384 + row_off + i * 2048) = o;
           }
           if (TAIL && tail_tile)
-            tail_rows_over(sgen + kOffV + vbuf * 16384 + row_off, a.v_tail + tail_off, a.tail_ts, slot0, a.tail_lo, a.t_phys);
+            tail_rows_over(sgen + kOffV + vbuf * 16384 + row_off, a.v_tail + tail_off, a.tail_ts, slot0, a.tail_lo, a.t_phys, a.status);
           fence_proxy_async();
           mbar_arrive(b_vfull + 8 * vbuf);
           // The raw stage is released only here, after the words read from it have been used and
@@ -951,16 +987,20 @@ size_t attn_tc_scratch_bytes(const xkv_params*) { return (size_t)2 * kMaxGrid * 
 // available (two per CTA) and by the number of steps.
 struct TailArgs { const void* k; const void* v; int64_t ts, hs; };
 
-static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
-                                     float scale, float* part, size_t part_bytes, cudaStream_t st,
-                                     const TailArgs* tail = nullptr) {
-  static int sm_count = 0;
-  static bool attr_set = false;
-  if (!attr_set) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+// Per device, on first use with that device current: the SM count, and the opt-in to more than
+// 48 KB of dynamic shared memory for the attention kernels (a per-device function attribute).
+static std::mutex g_setup_mutex;
+static int g_sm_count[kMaxDevices] = {0};       // 0: not set up yet
+
+static cudaError_t attn_device_setup(int* sm_count) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
+  if (g_sm_count[dev] == 0) {
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
     if (e != cudaSuccess) return e;
@@ -968,7 +1008,19 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    g_sm_count[dev] = sms;
+  }
+  *sm_count = g_sm_count[dev];
+  return cudaSuccess;
+}
+
+static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
+                                     float scale, float* part, size_t part_bytes, cudaStream_t st,
+                                     const TailArgs* tail = nullptr) {
+  int sm_count = 0;
+  {
+    const cudaError_t e = attn_device_setup(&sm_count);
+    if (e != cudaSuccess) return e;
   }
   Args a;
   a.q = reinterpret_cast<const __nv_bfloat16*>(q);
@@ -988,6 +1040,7 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
   const size_t slots = part_bytes / kSlotBytes;
   long long grid = sm_count;
   if (grid > (long long)(slots / 2)) grid = (long long)(slots / 2);
+  if (c->attn_max_blocks > 0 && grid > c->attn_max_blocks) grid = c->attn_max_blocks;
   if (grid > a.total) grid = a.total;
   if (grid < 1) return cudaErrorMemoryAllocation;
   a.part_o = part;
@@ -1067,6 +1120,30 @@ cudaError_t launch_attn_tc_static(xkv_cache* c, const void* q, void* out, int n,
   }
   return launch_attn_tc_on(c, q, out, n, ts, hs, scale, reinterpret_cast<float*>(addr),
                            (size_t)XKV_STATIC_SCRATCH_BYTES, st);
+}
+
+// ---------------------------------------------------------------------------
+// Test hook: the bounded wait of the attention kernel on a barrier that nothing completes.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(32) timeout_probe_kernel(int* status) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const WaitCtx wc{status, &abort_flag};
+  if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0, wc);     // phase 0 never completes: runs into the limit
+  __syncthreads();
+  mbar_wait(smem_u32(&bar), 0, wc);                           // the flag is up: every later wait returns at once
+}
+
+cudaError_t launch_timeout_probe(xkv_cache* c, cudaStream_t st) {
+  timeout_probe_kernel<<<1, 32, 0, st>>>(c->status);
+  c->launches++;
+  return cudaGetLastError();
 }
 
 }  // namespace xkv

@@ -132,12 +132,6 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
   c->attn_part = reinterpret_cast<float*>(c->ws + L.off_attn);
   c->attn_part_bytes = L.attn_bytes;
   reset_host_state(c);
-  {
-    // test hook: the maintenance kernels have conversion-free fast forms of Eq. 7 and Eq. 10 with a
-    // plain fallback; XKV_FORCE_PLAIN=1 makes every kernel of this cache take the fallback
-    const char* fp = getenv("XKV_FORCE_PLAIN");
-    c->force_plain = (fp && fp[0] == '1') ? 1 : 0;
-  }
   c->prof = new (std::nothrow) Profiler;
   if (!c->prof) { delete c; return XKV_E_NOMEM; }
   if (cudaEventCreateWithFlags(&c->kbar_done, cudaEventDisableTiming) != cudaSuccess) {
@@ -151,7 +145,9 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
 
 int xkv_reset(xkv_cache* c, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;
-  if (c->kbar_done) cudaEventSynchronize(c->kbar_done);      // a head-mean kernel of the last stream step
+  // a head-mean kernel of the last stream step may still run on the library's stream
+  if (c->kbar_done && cudaStreamWaitEvent(reinterpret_cast<cudaStream_t>(stream), c->kbar_done, 0) != cudaSuccess)
+    return XKV_E_CUDA;
   reset_host_state(c);
   return zero_workspace(c, reinterpret_cast<cudaStream_t>(stream));
 }
@@ -530,7 +526,25 @@ int xkv_poll_status(const xkv_cache* c, xkv_stream stream) {
   if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
   int word = 0;
   if (cudaMemcpy(&word, c->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return XKV_E_CUDA;
-  return word == 0 ? XKV_OK : XKV_E_TIMEOUT;
+  if (word == 0) return XKV_OK;
+  return word == (int)XKV_E_RANGE ? XKV_E_RANGE : XKV_E_TIMEOUT;
+}
+
+int xkv_debug_force_plain(xkv_cache* c, int32_t on) {
+  if (!c || (on != 0 && on != 1)) return XKV_E_INVALID;
+  c->force_plain = on;
+  return XKV_OK;
+}
+
+int xkv_debug_limit_attention_blocks(xkv_cache* c, int32_t max_blocks) {
+  if (!c || max_blocks < 0) return XKV_E_INVALID;
+  c->attn_max_blocks = max_blocks;
+  return XKV_OK;
+}
+
+int xkv_debug_timeout_probe(xkv_cache* c, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  return launch_timeout_probe(c, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? XKV_OK : XKV_E_CUDA;
 }
 
 int xkv_profile_enable(xkv_cache* c, int enable) {
@@ -572,6 +586,7 @@ const char* xkv_strerror(int status) {
     case XKV_E_CUDA: return "CUDA call failed";
     case XKV_E_TIMEOUT: return "bounded device-side wait ran out";
     case XKV_E_LIMIT: return "request exceeds a fixed built-in limit (static scratch size)";
+    case XKV_E_RANGE: return "a value exceeds the range of the 16-bit tensor-core operands";
     default: return "unknown status";
   }
 }

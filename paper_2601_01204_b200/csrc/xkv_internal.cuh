@@ -64,6 +64,7 @@ struct xkv_cache {
   long long launches;
   int force_plain;         // 1: kernels take the plain (conversion-based) arithmetic forms everywhere
   int tail_mode;           // 1: the stream-step calls attend with the step's K, V unquantised
+  int attn_max_blocks;     // test hook: cap on the thread blocks of the tensor-core attention (0: none)
   // head means of the keys after the first frame (Eq. 4), filled by the stream step beside the
   // attention and used by the next step's scoring when the cache has not changed since
   float* kbar;             // [cap][64]
@@ -119,5 +120,7 @@ cudaError_t launch_attn_tc_tail(xkv_cache* c, const void* q, const void* k_t, co
 cudaError_t launch_attn_tc_static(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
                                   float scale, cudaStream_t st);
 size_t attn_tc_scratch_bytes(const xkv_params* p);
+// One small block running the attention kernel's bounded wait on a barrier nobody completes.
+cudaError_t launch_timeout_probe(xkv_cache* c, cudaStream_t st);
 
 }  // namespace xkv

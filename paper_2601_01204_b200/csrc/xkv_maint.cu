@@ -5,6 +5,8 @@
 // codes) that must be reproducible bit for bit.
 #include <stdlib.h>
 
+#include <mutex>
+
 #include "xkv_internal.cuh"
 
 namespace xkv {
@@ -672,15 +674,24 @@ select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restri
 }
 
 cudaError_t launch_select(xkv_cache* c, int r_old, int k, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(select_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kSelSmemKeys * (int)sizeof(uint32_t));
+  {
+    // opt-in to large dynamic shared memory: a per-device function attribute, set once per device
+    static std::mutex mu;
+    static bool attr_set[64] = {false};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(select_kernel<true, 17>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kSelSmemKeys * (int)sizeof(uint32_t));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!attr_set[dev]) {
+      e = cudaFuncSetAttribute(select_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               kSelSmemKeys * (int)sizeof(uint32_t));
+      if (e != cudaSuccess) return e;
+      e = cudaFuncSetAttribute(select_kernel<true, 17>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               kSelSmemKeys * (int)sizeof(uint32_t));
+      if (e != cudaSuccess) return e;
+      attr_set[dev] = true;
+    }
   }
   LaunchScope ls(c, XKV_PROF_SELECT, st);
   const size_t smem = (size_t)r_old * sizeof(uint32_t);

@@ -25,6 +25,7 @@ lib = C.CDLL(LIB_PATH)
 
 XKV_OK, XKV_E_INVALID, XKV_E_STATE, XKV_E_NOMEM, XKV_E_UNSUPPORTED, XKV_E_CUDA, XKV_E_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 XKV_E_LIMIT = -7
+XKV_E_RANGE = -8
 STATIC_SCRATCH_BYTES = 32 << 20
 BUF_K_CODES, BUF_K_PARAMS, BUF_V_CODES, BUF_V_PARAMS, BUF_ORIGIN, BUF_SCORES, BUF_KEPT, BUF_QVEC = range(8)
 
@@ -34,6 +35,7 @@ EXPORTED = [
     "xkv_stream_step_host", "xkv_get_info", "xkv_debug_export", "xkv_poll_status", "xkv_strerror",
     "xkv_synth_fill", "xkv_profile_enable", "xkv_profile_read", "attn_packed_causal_static",
     "xkv_debug_rewind_attention", "attn_packed_causal_tail", "xkv_set_unquantised_tail",
+    "xkv_debug_force_plain", "xkv_debug_limit_attention_blocks", "xkv_debug_timeout_probe",
 ]
 PROF_NAMES = ["append", "pool_q", "score", "select", "regroup_k", "gather", "attn", "attn_combine", "kbar"]
 
@@ -94,6 +96,12 @@ lib.xkv_debug_export.restype = _i64
 lib.xkv_debug_export.argtypes = [_vp, _i32, _vp, _sz, _vp]
 lib.xkv_debug_rewind_attention.restype = C.c_int
 lib.xkv_debug_rewind_attention.argtypes = [_vp]
+lib.xkv_debug_force_plain.restype = C.c_int
+lib.xkv_debug_force_plain.argtypes = [_vp, _i32]
+lib.xkv_debug_limit_attention_blocks.restype = C.c_int
+lib.xkv_debug_limit_attention_blocks.argtypes = [_vp, _i32]
+lib.xkv_debug_timeout_probe.restype = C.c_int
+lib.xkv_debug_timeout_probe.argtypes = [_vp, _vp]
 lib.xkv_poll_status.restype = C.c_int
 lib.xkv_poll_status.argtypes = [_vp, _vp]
 lib.xkv_strerror.restype = C.c_char_p
@@ -253,6 +261,15 @@ class Cache:
 
     def xkv_debug_rewind_attention(self) -> None:
         _check(lib.xkv_debug_rewind_attention(self.handle), "xkv_debug_rewind_attention")
+
+    def xkv_debug_force_plain(self, on: bool) -> None:
+        _check(lib.xkv_debug_force_plain(self.handle, 1 if on else 0), "xkv_debug_force_plain")
+
+    def xkv_debug_limit_attention_blocks(self, max_blocks: int) -> None:
+        _check(lib.xkv_debug_limit_attention_blocks(self.handle, max_blocks), "xkv_debug_limit_attention_blocks")
+
+    def xkv_debug_timeout_probe(self) -> None:
+        _check(lib.xkv_debug_timeout_probe(self.handle, _stream()), "xkv_debug_timeout_probe")
 
     def xkv_poll_status(self) -> int:
         return int(lib.xkv_poll_status(self.handle, _stream()))

@@ -49,6 +49,6 @@ def test_workspace_bytes_and_param_validation(xkv):
 
 def test_strerror(xkv):
     assert xkv.lib.xkv_strerror(0) == b"ok"
-    for code in range(-6, 0):
+    for code in range(-8, 0):
         assert len(xkv.lib.xkv_strerror(code)) > 3
     assert b"unknown" in xkv.lib.xkv_strerror(-99)

@@ -26,7 +26,10 @@ def xkv():
     return m
 
 
-def _stream(xkv, n, budget, frames, seed, attn_from, bits=4):
+def _stream(xkv, n, budget, frames, seed, attn_from, bits=4, layer=0, via_stream_step=False):
+    """One layer's cache against the oracle.  via_stream_step: the frame goes through
+    xkv_stream_step (scores and kept indices are read back after the step) instead of the four
+    per-layer calls."""
     import torch
     H, d = 16, 64
     p = xkv.Params(n_heads=H, head_dim=d, budget=budget, max_frame_tokens=n, kv_bits=bits)
@@ -35,13 +38,17 @@ def _stream(xkv, n, budget, frames, seed, attn_from, bits=4):
     rng = np.random.default_rng(seed)
     evicting = 0
     for t in range(frames):
-        qb, kb, vb = synth.gen_frame(seed, 0, t, H, n, d)
+        qb, kb, vb = synth.gen_frame(seed, layer, t, H, n, d)
         qf, kf, vf = (synth.bf16_bits_to_f32(x) for x in (qb, kb, vb))
         q, k, v = (to_device_bf16(x) for x in (qb, kb, vb))
-        cache.kv_append(k, v)
-        cache.kv_score_evict(q)
+        out = torch.empty_like(q)
         ora.append(kf, vf)
         ora.score_evict(qf)
+        if via_stream_step:
+            xkv.xkv_stream_step([cache], [q], [k], [v], [out])
+        else:
+            cache.kv_append(k, v)
+            cache.kv_score_evict(q)
         info = cache.xkv_get_info()
         if ora.last_scores is not None and info.last_kept > 0:
             evicting += 1
@@ -49,11 +56,12 @@ def _stream(xkv, n, budget, frames, seed, attn_from, bits=4):
             assert np.array_equal(s.view(np.uint32), ora.last_scores.view(np.uint32)), f"frame {t}: scores"
             kept = cache.xkv_debug_export(xkv.BUF_KEPT, info.last_kept * 4).view(np.int32)
             assert np.array_equal(kept, ora.last_kept_mid), f"frame {t}: kept indices"
-        cache.kv_quant_pack()
+        if not via_stream_step:
+            cache.kv_quant_pack()
         ora.quant_pack()
         compare_state(cache.export(), ora.export(), f"frame {t}")
-        out = torch.empty_like(q)
-        cache.attn_packed_causal(q, out)
+        if not via_stream_step:
+            cache.attn_packed_causal(q, out)
         if t >= attn_from:
             rows = np.sort(rng.choice(n, size=24, replace=False))
             rows[0], rows[-1] = 0, n - 1                      # first row of the first tile, last row of the ragged tile
@@ -90,9 +98,33 @@ def test_long_stream_layer_1004_tokens_budget_16384(xkv):
     assert cache.xkv_get_info().T == 16384 and evicting >= 1
 
 
-def test_single_layer_1374_tokens_budget_8192(xkv):
-    cache, evicting = _stream(xkv, 1374, 8192, 8, seed=2, attn_from=5)
+def test_full_stack_last_layer_through_stream_step(xkv):
+    """The full-stack workload seeds every layer on its own (seed 3 + layer, the layer's own
+    outlier channels): layer 23, through xkv_stream_step."""
+    cache, evicting = _stream(xkv, 1374, 16384, 14, seed=3 + 23, attn_from=12, layer=23, via_stream_step=True)
+    info = cache.xkv_get_info()
+    assert info.T == 16384 and evicting >= 2 and info.last_evicted == 1374
+
+
+def test_single_layer_1374_tokens_budget_8192_all_32_frames(xkv):
+    """The single-layer workload at its full length: 32 frames, 27 of them evicting."""
+    cache, evicting = _stream(xkv, 1374, 8192, 32, seed=2, attn_from=29)
+    assert cache.xkv_get_info().T == 8192 and evicting >= 26
+
+
+def test_ablation_budget_4096_int4(xkv):
+    cache, evicting = _stream(xkv, 1374, 4096, 6, seed=5, attn_from=3)
+    assert cache.xkv_get_info().T == 4096 and evicting >= 3
+
+
+def test_prune_only_16bit_budget_8192(xkv):
+    cache, evicting = _stream(xkv, 1374, 8192, 8, seed=5, attn_from=6, bits=16)
     assert cache.xkv_get_info().T == 8192 and evicting >= 2
+
+
+def test_prune_only_16bit_budget_16384(xkv):
+    cache, evicting = _stream(xkv, 1374, 16384, 14, seed=5, attn_from=12, bits=16)
+    assert cache.xkv_get_info().T == 16384 and evicting >= 2
 
 
 def test_prune_only_16bit_budget_4096(xkv):

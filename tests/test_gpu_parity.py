@@ -31,20 +31,21 @@ def test_tiny_stream_4bit(xkv, impl):
     print("tiny 4-bit impl", impl, "worst (max-abs, rel-L2)", worst)
 
 
-def test_tiny_stream_4bit_plain_arithmetic_forms(xkv, monkeypatch):
+def test_tiny_stream_4bit_plain_arithmetic_forms(xkv):
     """The maintenance kernels dequantise and quantise without conversion instructions when the
     zero-points and scaled values are small enough, and fall back to the plain forms otherwise.
-    XKV_FORCE_PLAIN=1 (read when a cache is created) sends every kernel down the fallback:
-    both must give the oracle's bits."""
-    monkeypatch.setenv("XKV_FORCE_PLAIN", "1")
+    xkv_debug_force_plain sends every kernel of the cache down the fallback: both must give the
+    oracle's bits."""
     p = xkv.Params(budget=1024, max_frame_tokens=261, kv_bits=4)
-    cache, ora, worst = run_stream(xkv, p, 261, 7, seed=11)
+    cache, ora, worst = run_stream(xkv, p, 261, 7, seed=11, force_plain=True)
     assert cache.xkv_get_info().T == 1024
 
 
 def test_large_offset_keys(xkv):
-    """Keys with a large common offset: zero-points of a few thousand and |x / s| far from 0."""
-    import torch
+    """Keys with a large common offset on every channel: zero-points of a few thousand and |x / s|
+    far from 0.  The packed state must be bit-exact.  Keys near 100 with a spread of 0.05 lose that
+    spread in any 16-bit operand (spacing 0.06), so the attention check of this case uses the fp32
+    CUDA-core kernel."""
     from xkv_testlib import compare_state, oracle_params, bf16_tensor_to_f32, check_attention
     from oracle import xkv_oracle as xo
     p = xkv.Params(n_heads=4, budget=400, max_frame_tokens=128, kv_bits=4)
@@ -59,11 +60,110 @@ def test_large_offset_keys(xkv):
         cache.kv_append(k, v); cache.kv_score_evict(q); cache.kv_quant_pack()
         ora.append(kf, vf); ora.score_evict(qf); ora.quant_pack()
         compare_state(cache.export(), ora.export(), f"frame {t}")
-        # keys near 100 with a spread of 0.05 cannot be held in 16-bit operands (spacing 0.06), so the
-        # attention check uses the fp32 CUDA-core kernel; the point here is the bit-exact state above
         out = cache.attn_packed_causal(q, impl=1)
         check_attention(bf16_tensor_to_f32(out).transpose(1, 0, 2), ora.attend(qf), f"frame {t}")
     assert cache.xkv_get_info().T == 400
+
+
+def _offset_channel_frame(t, H, n, d):
+    """Ordinary keys except four channels per head that sit at +254 / -255 and move by one step:
+    the channel-wise key outliers of Fig. 3 in their hardest form for Eq. 8, zero-points of -3810
+    and +3825.  Every seventh token has a value row of range 1e-4 (scale 7e-6)."""
+    qb, kb, vb = synth.gen_frame(12, 0, t, H, n, d)
+    kf, vf = synth.bf16_bits_to_f32(kb).copy(), synth.bf16_bits_to_f32(vb).copy()
+    bit = (synth.gen_tensor_bits(99, 0, t, synth.TENSOR_Q, H, n, d) & 1).astype(np.float32)
+    for c, base in ((3, 254.0), (17, 254.0), (40, -255.0), (63, -255.0)):
+        kf[:, :, c] = base + bit[:, :, c]
+    vf[:, ::7, :] *= np.float32(1e-5)
+    return qb, synth.f32_to_bf16_bits(kf), synth.f32_to_bf16_bits(vf)
+
+
+@pytest.mark.parametrize("tail", [False, True])
+def test_offset_channels_through_the_tensor_core_kernel(xkv, tail):
+    """Zero-points in the thousands and tiny value scales through impl = 0: the fp16 operand path
+    forms s * q + (-s z) with the constant taken in fp32, which holds for any integer zero-point
+    (Eq. 10).  State bit-exact, attention within the usual tolerance, no status raised."""
+    from xkv_testlib import compare_state, oracle_params, bf16_tensor_to_f32, check_attention
+    from oracle import xkv_oracle as xo
+    H, n, d = 4, 128, 64
+    p = xkv.Params(n_heads=H, budget=400, max_frame_tokens=n, kv_bits=4)
+    cache, ora = xkv.Cache(p), xo.OracleLayer(oracle_params(p))
+    zmax = 0.0
+    for t in range(6):
+        qb, kb, vb = _offset_channel_frame(t, H, n, d)
+        qf, kf, vf = (synth.bf16_bits_to_f32(x) for x in (qb, kb, vb))
+        q, k, v = (to_device_bf16(x) for x in (qb, kb, vb))
+        cache.kv_append(k, v); cache.kv_score_evict(q); cache.kv_quant_pack()
+        ora.append(kf, vf); ora.score_evict(qf); ora.quant_pack()
+        compare_state(cache.export(), ora.export(), f"frame {t}")
+        out = cache.attn_packed_causal_tail(q, k, v) if tail else cache.attn_packed_causal(q, impl=0)
+        check_attention(bf16_tensor_to_f32(out).transpose(1, 0, 2), ora.attend(qf, full_precision_tail=tail), f"frame {t}")
+        assert cache.xkv_poll_status() == 0
+        zmax = max(zmax, float(np.abs(ora.k_z_first).max()), float(np.abs(ora.k_z_rest).max()) if ora.T > n else 0.0)
+    assert zmax > 3000 and float(ora.v_s.min()) < 2e-5
+
+
+def test_values_beyond_fp16_are_reported_not_silent(xkv):
+    """Magnitudes above 65504 cannot be tensor-core operands of a 4-bit cache: the call records
+    XKV_E_RANGE in the status word (queries, dequantised keys, raw tail rows), the fp32 kernel and a
+    16-bit cache take the same inputs without complaint, and xkv_reset clears the word."""
+    import torch
+    H, n, d = 2, 64, 64
+    qb, kb, vb = synth.gen_frame(14, 0, 0, H, n, d)
+    q, k, v = (to_device_bf16(x) for x in (qb, kb, vb))
+    big_k = k.clone(); big_k[1, 5, 9] = 1.0e5
+    big_q = q.clone(); big_q[0, 3, 2] = -7.0e4
+    p = xkv.Params(n_heads=H, budget=256, max_frame_tokens=n, kv_bits=4)
+    cache = xkv.Cache(p)
+    for qq, kk, use_tail, want in ((q, k, False, 0), (q, big_k, False, xkv.XKV_E_RANGE), (big_q, k, False, xkv.XKV_E_RANGE),
+                                   (q, big_k, True, xkv.XKV_E_RANGE)):
+        cache.xkv_reset()
+        cache.kv_append(kk, v); cache.kv_score_evict(qq); cache.kv_quant_pack()
+        if use_tail:
+            cache.attn_packed_causal_tail(qq, kk, v)
+        else:
+            cache.attn_packed_causal(qq, impl=0)
+        assert cache.xkv_poll_status() == want
+    # the fp32 kernel has no such limit
+    cache.xkv_reset()
+    cache.kv_append(big_k, v); cache.kv_score_evict(q); cache.kv_quant_pack()
+    out = cache.attn_packed_causal(q, impl=1)
+    assert cache.xkv_poll_status() == 0 and bool(torch.isfinite(out.float()).all())
+    # a 16-bit cache multiplies in bf16
+    c16 = xkv.Cache(xkv.Params(n_heads=H, budget=256, max_frame_tokens=n, kv_bits=16))
+    c16.kv_append(big_k, v); c16.kv_score_evict(big_q); c16.kv_quant_pack()
+    out = c16.attn_packed_causal(big_q, impl=0)
+    assert c16.xkv_poll_status() == 0 and bool(torch.isfinite(out.float()).all())
+
+
+def test_bounded_wait_reports_timeout_and_the_context_survives(xkv):
+    """Every wait inside the attention kernel is bounded.  The probe runs that wait on a barrier
+    nothing completes: it gives up at its limit, the kernel ends, the status word reads
+    XKV_E_TIMEOUT, and after xkv_reset the same cache streams a frame normally."""
+    import torch
+    H, n, d = 2, 64, 64
+    p = xkv.Params(n_heads=H, budget=256, max_frame_tokens=n, kv_bits=4)
+    cache = xkv.Cache(p)
+    assert cache.xkv_poll_status() == 0
+    cache.xkv_debug_timeout_probe()
+    assert cache.xkv_poll_status() == xkv.XKV_E_TIMEOUT
+    assert xkv.lib.xkv_strerror(xkv.XKV_E_TIMEOUT) == b"bounded device-side wait ran out"
+    cache.xkv_reset()
+    assert cache.xkv_poll_status() == 0
+    cache2, ora, _ = run_stream(xkv, p, n, 3, seed=8)
+    q, k, v = (to_device_bf16(x) for x in synth.gen_frame(8, 0, 0, H, n, d))
+    out = cache.step(q, k, v)
+    assert cache.xkv_poll_status() == 0 and bool(torch.isfinite(out.float()).all())
+
+
+@pytest.mark.parametrize("blocks", [1, 5, 20])
+def test_attention_with_fewer_blocks_than_multiprocessors(xkv, blocks):
+    """The attention cuts its line of (item, key tile) steps into one piece per thread block.  With
+    the block count capped a piece spans several items and an item few pieces: same result."""
+    p = xkv.Params(n_heads=6, budget=900, max_frame_tokens=300, kv_bits=4)
+    run_stream(xkv, p, 300, 5, seed=16, max_blocks=blocks)
+    p = xkv.Params(n_heads=3, budget=600, max_frame_tokens=200, kv_bits=16)
+    run_stream(xkv, p, 200, 4, seed=17, max_blocks=blocks, tail=False)
 
 
 @pytest.mark.parametrize("impl", [0, 1])

@@ -17,6 +17,11 @@ eviction belongs to the tokens its origins name:
   P4  the regroup rule on crafted steps: a complete key group whose tokens all survive in
       place is carried over verbatim; a group that lost a token is the quantiser applied to
       the hand-assembled dequantised survivors and raw new keys.
+  P5  key_mode "once" (keys quantised once, on arrival, in groups of G tokens of their frame):
+      at every later frame a survivor's codes and dequantised key are exactly those of
+      quantising its own frame alone, found through its origin; the parameter table holds
+      exactly the groups that still have a token (bounded by the cache length, reclaimed);
+      without pruning the stream equals quantise-each-frame-then-attend.
 
 Each pin is a function of the oracle module, so that test_planted_mistakes_are_caught can
 run the same pins against copies of the oracle with one plausible mistake planted in each
@@ -45,9 +50,12 @@ def _origin_to_pos(org, n):
 
 
 # ---------------------------------------------------------------------------- P1 + P2 + P3
-def pin_survivor_data_follows_origins(xo, bits, seed=23, frames=10):
+def pin_survivor_data_follows_origins(xo, bits, seed=23, frames=10, key_mode="regroup"):
     H, n, d, G = 4, 37, 16, 8
-    p = xo.OracleParams(n_heads=H, head_dim=d, n_special=5, pool_g=4, quant_group=G, kv_bits=bits, budget=150)
+    p = xo.OracleParams(n_heads=H, head_dim=d, n_special=5, pool_g=4, quant_group=G, kv_bits=bits, budget=150,
+                        key_mode=key_mode)
+    arrival = []                               # key_mode "once": each frame quantised alone, (codes, dequantised)
+    peak_groups = 0
     L = xo.OracleLayer(p)
     raw = []                                   # (K, V) of every frame
     kbound = {}                                # origin -> accumulated Eq. 7-8 bound per (head, channel)
@@ -91,6 +99,23 @@ def pin_survivor_data_follows_origins(xo, bits, seed=23, frames=10):
         assert np.array_equal(L.v_z.view(np.uint32), vz.view(np.uint32)), f"frame {t}: value zero-points"
         assert np.array_equal(L.values_dequantized(), xo_real.dequantize_values(vc, vs, vz))
 
+        # ---- P5: keys quantised once ----
+        if key_mode == "once":
+            kc, ks, kz = xo_real.quantize_keys(k, G, bits)
+            arrival.append((kc, xo_real.dequantize_keys(kc, ks, kz, G), ks))
+            want_codes = np.stack([arrival[f][0][:, tok] for f, tok in zip(fi, ti)], axis=1)
+            want_deq = np.stack([arrival[f][1][:, tok] for f, tok in zip(fi, ti)], axis=1)
+            assert np.array_equal(L.k_codes, want_codes), f"frame {t}: key codes"
+            Kd = L.keys_dequantized()
+            assert np.array_equal(Kd.view(np.uint32), want_deq.view(np.uint32)), f"frame {t}: dequantised keys"
+            s_tok = np.stack([arrival[f][2][:, tok // G] for f, tok in zip(fi, ti)], axis=1)
+            assert np.all(np.abs(Kd.astype(np.float64) - Kraw) <= 0.5 * s_tok * (1 + 1e-4) + 1e-6)   # one quantisation only
+            live = {(int(f), int(tok) // G) for f, tok in zip(fi, ti)}
+            assert len(L.k_table) == len(live) <= L.T, f"frame {t}: parameter table holds {len(L.k_table)} groups, {len(live)} live"
+            assert L.export()["k_groups_live"] == len(live)
+            peak_groups = max(peak_groups, len(live))
+            continue
+
         # ---- P2: keys ----
         Kd = L.keys_dequantized()
         Tf = L.T_first
@@ -114,6 +139,29 @@ def pin_survivor_data_follows_origins(xo, bits, seed=23, frames=10):
         err = np.abs(Kd.astype(np.float64) - Kraw)
         assert np.all(err <= bound * (1 + 1e-4) + 1e-6), f"frame {t}: key error {float((err - bound).max())} over the bound"
     assert evicting >= 5
+    if key_mode == "once":      # groups did die and were given back: the table is smaller than "every group ever made"
+        assert peak_groups < frames * -(-n // G)
+
+
+def pin_quantise_once_without_pruning_is_framewise_quantisation(xo):
+    """key_mode "once", budget never reached, ragged frame sizes: the stream's attention equals
+    attention over the frames quantised one by one (Eq. 7-10), bit for bit in the cache and to
+    rounding in the output."""
+    H, d, G = 2, 16, 16
+    p = xo.OracleParams(n_heads=H, head_dim=d, n_special=5, pool_g=4, quant_group=G, kv_bits=4, budget=10 ** 6,
+                        key_mode="once")
+    L = xo.OracleLayer(p)
+    Kd, Vd = [], []
+    for t, n in enumerate([40, 23, 64, 7]):
+        q, k, v = _frame(31, t, H, n, d)
+        out = L.step(q, k, v)
+        kc, ks, kz = xo_real.quantize_keys(k, G, 4)
+        vc, vs, vz = xo_real.quantize_values(v, 4)
+        Kd.append(xo_real.dequantize_keys(kc, ks, kz, G)), Vd.append(xo_real.dequantize_values(vc, vs, vz))
+        ref = xo_real.attention(q, np.concatenate(Kd, 1), np.concatenate(Vd, 1), 1 / np.sqrt(d))
+        np.testing.assert_allclose(out.transpose(1, 0, 2), ref, rtol=1e-6, atol=1e-7)
+        assert np.array_equal(L.keys_dequantized(), np.concatenate(Kd, 1))
+    assert len(L.k_table) == 3 + 2 + 4 + 1
 
 
 # ---------------------------------------------------------------------------- P4
@@ -180,6 +228,9 @@ PINS = [
     ("survivors-8bit", lambda xo: pin_survivor_data_follows_origins(xo, 8, seed=24)),
     ("survivors-16bit", lambda xo: pin_survivor_data_follows_origins(xo, 16, seed=25)),
     ("regroup-rule", pin_regroup_rule_on_crafted_steps),
+    ("once-4bit", lambda xo: pin_survivor_data_follows_origins(xo, 4, seed=26, key_mode="once")),
+    ("once-8bit", lambda xo: pin_survivor_data_follows_origins(xo, 8, seed=27, key_mode="once")),
+    ("once-no-pruning", pin_quantise_once_without_pruning_is_framewise_quantisation),
 ]
 
 
@@ -231,6 +282,19 @@ MUTATIONS = [
     ("survivors re-quantised from their codes, not their values",
      "old_deq = dequantize_keys(old_codes, self.k_s_rest, self.k_z_rest, G)",
      "old_deq = old_codes.astype(F32)"),
+    ("once: key codes not gathered",
+     "codes_kept = self.k_codes[:, keep_abs]",
+     "codes_kept = self.k_codes[:, :len(keep_abs)]"),
+    ("once: group references not gathered",
+     "gid_kept = self.k_gid[keep_abs]",
+     "gid_kept = self.k_gid[:len(keep_abs)]"),
+    ("once: parameter table never reclaimed",
+     "self.k_table = {g: v for g, v in self.k_table.items() if g in live}",
+     "self.k_table = dict(self.k_table)"),
+    ("once: a frame's groups counted from the cache position, not from the frame's first token",
+     "codes, s, z = quantize_keys(K_new, p.quant_group, p.kv_bits)\n        base",
+     "codes, s, z = quantize_keys(np.concatenate([K_new[:, :self.T % p.quant_group], K_new], 1), p.quant_group, p.kv_bits)\n"
+     "        codes = codes[:, self.T % p.quant_group:]\n        base"),
     ("first frame re-quantised with the rest",
      "self.k_codes = np.concatenate([self.k_codes[:, :Tf], new_codes], axis=1)",
      "self.k_codes = np.concatenate([self.k_codes[:, :Tf] * 0, new_codes], axis=1)"),

@@ -4,9 +4,12 @@ Some users of the library run where cudaMalloc is forbidden (a host that bans
 allocation after start-up, a plug-in without its own allocator).  For them the
 library offers attention with the split-KV partials in a fixed device array
 that belongs to the library image.  This file checks, through the C ABI, that
-the variant returns what attn_packed_causal returns, on several frames in a row
-(the array is shared and keeps the previous call's contents), also when it has
-to run with fewer thread blocks than the GPU has multiprocessors.
+the variant returns what attn_packed_causal returns and what the CPU oracle
+computes, on several frames in a row (the array is shared and keeps the previous
+call's contents), also with fewer thread blocks than the GPU has multiprocessors
+(the array holds 496 partial slots of 67 584 bytes, two per block: a GPU with more
+than 248 multiprocessors would run capped; a B200 has 148, so the test caps the
+block count through the library's test hook to walk that path).
 
 The file name sorts last on purpose: a run that stops at the first failure has
 then already executed every other test.
@@ -14,8 +17,10 @@ then already executed every other test.
 import numpy as np
 import pytest
 
+from oracle import xkv_oracle as xo
 from paper_2601_01204_b200 import synth
-from xkv_testlib import ATTN_MAXABS, ATTN_RELL2, attn_errors, bf16_tensor_to_f32, to_device_bf16
+from xkv_testlib import (ATTN_MAXABS, ATTN_RELL2, attn_errors, bf16_tensor_to_f32, check_attention, oracle_params,
+                         to_device_bf16)
 
 pytestmark = pytest.mark.gpu
 
@@ -61,13 +66,19 @@ def test_static_scratch_attention_matches_workspace_attention(xkv):
     assert checked >= 2 and sta_cache.xkv_get_info().T == 1024
 
 
-def test_static_scratch_attention_larger_frames(xkv):
+@pytest.mark.parametrize("max_blocks", [0, 24])
+def test_static_scratch_attention_larger_frames(xkv, max_blocks):
     """Frames of several query-tile pairs and many heads: the fixed array must still do (its size
-    does not depend on the frame), with fewer thread blocks than the workspace variant may use."""
+    does not depend on the frame).  max_blocks = 24 runs both variants with fewer thread blocks
+    than multiprocessors, as the static variant would on a GPU too large for its array.  Checked
+    against attn_packed_causal and against the oracle."""
     import torch
     H, n, d = 24, 700, 64
     p = xkv.Params(n_heads=H, budget=2048, max_frame_tokens=n, kv_bits=4)
     ref_cache, sta_cache = xkv.Cache(p), xkv.Cache(p)
+    ora = xo.OracleLayer(oracle_params(p))
+    for c in (ref_cache, sta_cache):
+        c.xkv_debug_limit_attention_blocks(max_blocks)
     for t, (qb, kb, vb) in enumerate(_frames(32, 4, H, n, d)):
         q, k, v = (to_device_bf16(x) for x in (qb, kb, vb))
         outs = []
@@ -84,3 +95,5 @@ def test_static_scratch_attention_larger_frames(xkv):
             outs.append(bf16_tensor_to_f32(out))
         maxabs, rell2 = attn_errors(outs[1], outs[0])
         assert maxabs <= ATTN_MAXABS and rell2 <= ATTN_RELL2, (t, maxabs, rell2)
+        qf, kf, vf = (synth.bf16_bits_to_f32(x) for x in (qb, kb, vb))
+        check_attention(outs[1].transpose(1, 0, 2), ora.step(qf, kf, vf), f"frame {t} against the oracle")

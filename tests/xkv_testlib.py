@@ -54,10 +54,14 @@ def check_attention(got: np.ndarray, ref: np.ndarray, tag: str = "") -> None:
 
 
 def run_stream(xkv, p, n_tokens, n_frames, seed, impl=0, layer=0, token_major=False, check_attn_every=1,
-               tail=False):
+               tail=False, force_plain=False, max_blocks=0):
     """Stream n_frames through one GPU cache and one oracle layer, comparing after every call."""
     import torch
     cache = xkv.Cache(p)
+    if force_plain:
+        cache.xkv_debug_force_plain(True)
+    if max_blocks:
+        cache.xkv_debug_limit_attention_blocks(max_blocks)
     ora = xo.OracleLayer(oracle_params(p))
     n_list = n_tokens if isinstance(n_tokens, (list, tuple)) else [n_tokens] * n_frames
     H, d = p.n_heads, p.head_dim

@@ -140,8 +140,8 @@ def run_reference(args) -> None:
     times = _oracle_layer_steps(w, steps, warm)
     per_layer = float(np.mean(times))
     value = 1.0 / (per_layer * w["layers"])
-    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
-                warmup=args.warmup, ms_per_step=per_layer * w["layers"] * 1e3, higher_is_better=True, scaling="weak",
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=steps,
+                warmup=warm, steps_requested=args.steps, warmup_requested=args.warmup, ms_per_step=per_layer * w["layers"] * 1e3, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f32/f64", data="synthetic",
                 config=dict(workload=w["name"], layers=w["layers"], tokens_per_frame=w["n_tokens"],
                             budget=w["budget"], kv_bits=w["kv_bits"],
@@ -255,15 +255,32 @@ def run_xkv(args) -> None:
     assert all(c.xkv_poll_status() == 0 for c in caches)
 
     # per-kernel device time over the same K steps, events on the launching stream
+    def read_profiles() -> dict:
+        acc = {}
+        for c in caches:
+            for name, (ms, cnt) in c.xkv_profile_read().items():
+                a = acc.setdefault(name, [0.0, 0])
+                a[0] += ms; a[1] += cnt
+        return acc
+
     for c in caches:
         c.xkv_profile_enable(True)
     for _ in range(K):
         step(t); t += 1
-    prof = {}
+    prof = read_profiles()
+    # the same frames through the per-call entry points (one launch per call, nothing overlapped),
+    # and the head-mean kernel alone: the stream step runs it beside the attention, where an
+    # event pair around it also spans the time it waits for multiprocessors
+    Kc = max(1, min(K, 5))
+    for _ in range(Kc):
+        q, k, v = frames[t % pool]; t += 1
+        for l, c in enumerate(caches):
+            c.kv_append(k[l], v[l]); c.kv_score_evict(q[l]); c.kv_quant_pack(); c.attn_packed_causal(q[l], outs[l])
+    calls = read_profiles()
     for c in caches:
-        for name, (ms, cnt) in c.xkv_profile_read().items():
-            a = prof.setdefault(name, [0.0, 0])
-            a[0] += ms; a[1] += cnt
+        c.xkv_debug_head_means()
+    kbar_alone = read_profiles()["kbar"]
+    for c in caches:
         c.xkv_profile_enable(False)
 
     # end to end: host tensors in pinned memory, copies inside the timed region
@@ -298,10 +315,31 @@ def run_xkv(args) -> None:
         flops = 4.0 * n * w["budget"] * d * H                     # useful FLOPs of one attention launch
         attn_avg_s = (attn_ms / max(attn_cnt, 1)) * 1e-3
         achieved = flops / attn_avg_s / 1e12 if attn_avg_s > 0 else 0.0
-        # kernels that the stream step runs on its side stream beside others; their event times
-        # include waiting for multiprocessors, so they are listed but not counted in the shares
+        # the head means run on the library's side stream beside the attention: their event span in
+        # the stream step is not a duration and is left out of the shares
         overlapped = ("kbar",)
         prof_total = sum(v[0] for k_, v in prof.items() if k_ not in overlapped)
+        nbytes = maintenance_bytes(H, n, d, w["budget"], w["kv_bits"])
+
+        def entry(ms: float, cnt: int, per: int, key: str | None, **extra) -> dict:
+            e = dict(ms_per_step=ms / per, launches_per_step=cnt / per, avg_launch_us=ms / max(cnt, 1) * 1e3, **extra)
+            if key in nbytes and ms > 0:
+                sec = ms / cnt * 1e-3
+                e.update(bytes_per_launch=nbytes[key], gb_per_s=nbytes[key] / sec / 1e9,
+                         hbm_frac=nbytes[key] / sec / 1e9 / peaks["hbm_gbs"])
+            return e
+
+        kernels = {}
+        for k_, v_ in prof.items():
+            if not v_[1]:
+                continue
+            if k_ in overlapped:
+                kernels[k_] = dict(launches_per_step=v_[1] / K, overlapped=True,
+                                   note="event span beside the attention; see kernels_per_call.kbar for its duration")
+            else:
+                kernels[k_] = entry(v_[0], v_[1], K, k_, share=v_[0] / prof_total if prof_total else 0.0)
+        per_call = {k_: entry(v_[0], v_[1], Kc, k_) for k_, v_ in calls.items() if v_[1] and k_ in ("append", "score_evict", "pack")}
+        per_call["kbar"] = entry(kbar_alone[0], kbar_alone[1], 1, "kbar")
         line = dict(metric=METRIC, value=aggregate_frames_per_s(world, K, ms_total), unit=UNIT, n_gpus=world, steps=K, warmup=W,
                     ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f16",
                     data="synthetic",
@@ -319,18 +357,7 @@ def run_xkv(args) -> None:
                                   frac_of_burst=achieved / peaks["tflops_burst"], flops_per_launch=flops,
                                   avg_launch_ms=attn_avg_s * 1e3,
                                   traffic=ATTN_DRAM_TRAFFIC_BYTES if w["name"] == WORKLOAD["name"] else None),
-                    kernels={k_: (dict(ms_per_step=v_[0] / K, launches_per_step=v_[1] / K, overlapped=True)
-                                  if k_ in overlapped else
-                                  dict(ms_per_step=v_[0] / K, launches_per_step=v_[1] / K,
-                                       share=v_[0] / prof_total if prof_total else 0.0))
-                             for k_, v_ in prof.items() if v_[1]})
-        # cache-maintenance kernels against the HBM roofline: algorithmic bytes of one launch in
-        # steady state (cache full, n tokens evicted per step) over its measured duration
-        for k_, nbytes in maintenance_bytes(H, n, d, w["budget"], w["kv_bits"]).items():
-            if k_ in line["kernels"] and prof[k_][0] > 0:
-                sec = prof[k_][0] / prof[k_][1] * 1e-3
-                line["kernels"][k_].update(bytes_per_launch=nbytes, gb_per_s=nbytes / sec / 1e9,
-                                           hbm_frac=nbytes / sec / 1e9 / peaks["hbm_gbs"])
+                    kernels=kernels, kernels_per_call=per_call)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w)
         print(json.dumps(line), flush=True)
@@ -395,23 +422,26 @@ def run_uncompressed(args) -> None:
 
 
 def maintenance_bytes(H: int, n: int, d: int, budget: int, bits: int) -> dict:
-    """Bytes that one steady-state launch of each cache-maintenance kernel has to move (4-bit cache):
+    """Bytes that one steady-state launch of each cache-maintenance launch has to move (4-bit cache):
     what it reads plus what it writes, every array once.  prunable = budget - n middle tokens are
-    scored, k = budget - 2 n of them survive, n new tokens arrive."""
+    scored, k = budget - 2 n of them survive, n new tokens arrive.  Keys are the profile categories:
+    the per-call launches (append, score_evict, pack), the head means (kbar) and the stream step's
+    single launch (maint = append + pooled query + scores + selection + pack)."""
     if bits != 4:
         return {}
     row, code, par = d * 2, d // 2, 8                      # bf16 row, packed row, one (scale, zero) pair
     prunable, k = budget - n, max(0, budget - 2 * n)
     grp = lambda tokens: (tokens + 63) // 64 * d * par     # key parameters of the 64-token groups
-    return {
-        "append": H * n * (2 * row) + H * n * (row + code + par),          # K, V in; staged K, V codes + params out
-        "pool_q": H * n * row,
-        "score": H * (prunable * code + grp(prunable)) + 4 * prunable,
-        "select": 4 * prunable + 4 * k,
-        # keys regrouped (survivors' codes and parameters, new bf16 keys in; codes and parameters
-        # out) and the survivors' value rows and parameters moved
-        "regroup_k": H * (k * code + grp(k) + n * row + (k + n) * code + grp(k + n)) + 2 * H * k * (code + par),
-    }
+    append = H * n * (2 * row) + H * n * (row + code + par)                 # K, V in; staged K, V codes + params out
+    pool = H * n * row                                                     # Q in
+    score = prunable * (4 * d + 4)                                         # stored head means in, scores out
+    select = 2 * 4 * prunable + 4 * k                                      # scores read by both passes, kept out
+    kbar = H * (prunable * code + grp(prunable)) + prunable * 4 * d        # codes + parameters in, head means out
+    # keys regrouped (survivors' codes and parameters, new bf16 keys in; codes and parameters
+    # out) and the survivors' value rows and parameters moved
+    pack = H * (k * code + grp(k) + n * row + (k + n) * code + grp(k + n)) + 2 * H * k * (code + par)
+    return {"append": append, "score_evict": pool + kbar + score + select, "pack": pack, "kbar": kbar,
+            "maint": append + pool + score + select + pack}
 
 
 def main() -> None:

@@ -312,6 +312,12 @@ XKV_API int xkv_debug_force_plain(xkv_cache* cache, int32_t on);
  * fewer, longer pieces and a block may cover several items; the result does not change. */
 XKV_API int xkv_debug_limit_attention_blocks(xkv_cache* cache, int32_t max_blocks);
 
+/* Tests and benchmarks only.  Recomputes, on `stream`, the head means of the keys after the first
+ * frame (Eq. 4) that the stream step keeps for the next frame's scoring, from the cache as it
+ * stands (idle cache; same values, nothing else changes).  Lets a benchmark time that kernel by
+ * itself: inside the stream step it runs beside the attention. */
+XKV_API int xkv_debug_head_means(xkv_cache* cache, xkv_stream stream);
+
 /* Tests only.  Launches one small thread block that waits, with the attention kernel's bounded
  * wait, on a barrier that nothing will ever complete.  The wait gives up after its iteration
  * limit (a fraction of a second), the kernel ends normally and the cache's status word reads
@@ -324,10 +330,13 @@ XKV_API int xkv_debug_timeout_probe(xkv_cache* cache, xkv_stream stream);
  * xkv_profile_read synchronises `stream`, adds the elapsed time of all launches
  * recorded since the last read to the per-category totals, copies the totals to
  * *out and clears them. */
-enum { XKV_PROF_APPEND = 0, XKV_PROF_POOL = 1, XKV_PROF_SCORE = 2, XKV_PROF_SELECT = 3,
-       XKV_PROF_REGROUP = 4, XKV_PROF_GATHER = 5, XKV_PROF_ATTN = 6, XKV_PROF_COMBINE = 7,
-       XKV_PROF_KBAR = 8,   /* head means of the keys, computed by the stream step beside the attention */
-       XKV_PROF_CATEGORIES = 9 };
+enum { XKV_PROF_APPEND = 0,       /* kv_append                                                       */
+       XKV_PROF_SCORE_EVICT = 1,  /* kv_score_evict: pooled query, scores, selection                 */
+       XKV_PROF_PACK = 2,         /* kv_quant_pack: key regroup / survivor gather                    */
+       XKV_PROF_KBAR = 3,         /* head means of the keys, by the stream step beside the attention */
+       XKV_PROF_MAINT = 4,        /* the three calls above as one launch (stream step)               */
+       XKV_PROF_ATTN = 5, XKV_PROF_COMBINE = 6,
+       XKV_PROF_CATEGORIES = 7 };
 typedef struct {
   double  ms[XKV_PROF_CATEGORIES];        /* summed device time per category, milliseconds */
   int64_t launches[XKV_PROF_CATEGORIES];  /* launches per category                         */

@@ -17,8 +17,9 @@ constexpr size_t kAlign = 256;
 
 struct Layout {
   int cap, row_bytes;
-  size_t off_k[2], off_kpar[2], off_v[2], off_vpar[2], off_origin[2];
-  size_t off_kstage, off_qbar, off_qvec, off_scores, off_kept, off_counters, off_status, off_attn, off_hist, off_kbar;
+  size_t off_k[2], off_kpar[2], off_v[2], off_vpar[2], off_origin[2], off_kbar[2];
+  size_t off_kstage, off_qbar, off_qvec, off_scores, off_kept, off_counters, off_status, off_attn, off_hist;
+  size_t off_run_hi, off_cand;
   size_t attn_bytes;
   size_t total;
 };
@@ -47,14 +48,15 @@ Layout make_layout(const xkv_params* p) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + kAlign - 1) / kAlign * kAlign; return o; };
   L.off_status = take(256);
-  L.off_counters = take(256);
-  L.off_hist = take(4096 * sizeof(unsigned int));
+  L.off_counters = take(576 * sizeof(unsigned int));
+  L.off_hist = take(4 * 4096 * sizeof(unsigned int));
   for (int b = 0; b < 2; ++b) {
     L.off_k[b] = take(H * L.cap * L.row_bytes);
     L.off_kpar[b] = take(H * (L.cap / 64) * 64 * sizeof(float2));
     L.off_v[b] = take(H * L.cap * L.row_bytes);
     L.off_vpar[b] = take(H * L.cap * sizeof(float2));
     L.off_origin[b] = take((size_t)L.cap * sizeof(int32_t));
+    L.off_kbar[b] = take((size_t)L.cap * 64 * sizeof(float));
   }
   L.off_kstage = take(H * max_n * 64 * sizeof(__nv_bfloat16));
   const int np_max = max_n;  // upper bound of N_pooled
@@ -62,7 +64,8 @@ Layout make_layout(const xkv_params* p) {
   L.off_qvec = take(64 * sizeof(float));
   L.off_scores = take((size_t)L.cap * sizeof(float));
   L.off_kept = take((size_t)L.cap * sizeof(int32_t));
-  L.off_kbar = take((size_t)L.cap * 64 * sizeof(float));
+  L.off_run_hi = take((size_t)(L.cap / 64) * sizeof(unsigned int));
+  L.off_cand = take((size_t)L.cap * sizeof(unsigned long long));
   L.attn_bytes = attn_tc_scratch_bytes(p);
   L.off_attn = take(L.attn_bytes);
   L.total = off;
@@ -81,6 +84,8 @@ void reset_host_state(xkv_cache* c) {
   c->n_pending = c->kk_pending = c->rold_pending = c->evict_pending = c->first_pending = 0;
   c->last_evicted = c->last_kept = c->last_prunable = 0;
   c->kbar_T = c->kbar_cur = c->kbar_frames = -1;
+  c->bar_base = 0;
+  c->sel_parity = 0;
 }
 
 }  // namespace
@@ -119,6 +124,8 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
     c->buf[b].v = c->ws + L.off_v[b];
     c->buf[b].vpar = reinterpret_cast<float2*>(c->ws + L.off_vpar[b]);
     c->buf[b].origin = reinterpret_cast<int32_t*>(c->ws + L.off_origin[b]);
+    c->buf[b].kbar = reinterpret_cast<float*>(c->ws + L.off_kbar[b]);
+    c->buf[b].kslot = nullptr;
   }
   c->kstage = reinterpret_cast<__nv_bfloat16*>(c->ws + L.off_kstage);
   c->qbar = reinterpret_cast<float*>(c->ws + L.off_qbar);
@@ -127,7 +134,8 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
   c->kept = reinterpret_cast<int32_t*>(c->ws + L.off_kept);
   c->counters = reinterpret_cast<unsigned int*>(c->ws + L.off_counters);
   c->sel_hist = reinterpret_cast<unsigned int*>(c->ws + L.off_hist);
-  c->kbar = reinterpret_cast<float*>(c->ws + L.off_kbar);
+  c->run_hi = reinterpret_cast<unsigned int*>(c->ws + L.off_run_hi);
+  c->cand = reinterpret_cast<unsigned long long*>(c->ws + L.off_cand);
   c->status = reinterpret_cast<int*>(c->ws + L.off_status);
   c->attn_part = reinterpret_cast<float*>(c->ws + L.off_attn);
   c->attn_part_bytes = L.attn_bytes;
@@ -164,79 +172,144 @@ int xkv_destroy(xkv_cache* c) {
   return XKV_OK;
 }
 
+}  // extern "C"
+
+namespace {
+
+// What the cache will look like once the frame of n tokens is in: a pure function of the sizes
+// seen so far and the budget (Sec. 3.2), so no device data is needed.
+struct FramePlan { int first, r_old, kk, evict, dst_slot; };
+
+int plan_frame(const xkv_cache* c, int n, FramePlan* p) {
+  p->first = (c->frames == 0) ? 1 : 0;
+  p->r_old = p->kk = p->evict = p->dst_slot = 0;
+  if (!p->first) {
+    p->r_old = c->T - c->T_first;
+    p->evict = (c->T + n > c->p.budget) ? 1 : 0;               // pruning is triggered when T > L_max
+    p->kk = p->evict ? (c->p.budget - c->T_first - n) : p->r_old;   // k = max(0, L_max - T_first - T_current)
+    if (p->kk < 0) p->kk = 0;
+    p->dst_slot = c->rest_base + p->kk;
+    if (p->dst_slot + n > c->cap) return XKV_E_NOMEM;
+  }
+  return XKV_OK;
+}
+
+// Everything of MaintArgs that describes the cache and the pending frame.
+void maint_args(const xkv_cache* c, MaintArgs* a) {
+  memset(a, 0, sizeof(*a));
+  a->H = c->p.n_heads; a->cap = c->cap; a->max_n = c->p.max_frame_tokens;
+  a->frame = c->frames + 1;
+  a->first = c->first_pending;
+  a->cur = c->buf[c->cur]; a->oth = c->buf[c->cur ^ 1];
+  a->n = c->n_pending;
+  a->rest_base = c->rest_base; a->r_old = c->rold_pending; a->kk = c->kk_pending;
+  a->r_new = c->kk_pending + c->n_pending;
+  a->dst_slot = c->first_pending ? 0 : c->rest_base + c->kk_pending;
+  a->identity = !(c->evict_pending && c->kk_pending > 0 && c->kk_pending < c->rold_pending);
+  a->n_special = c->p.n_special < c->n_pending ? c->p.n_special : c->n_pending;
+  a->pool_g = c->p.pool_g;
+  a->n_pooled = a->n_special + (c->n_pending - a->n_special + c->p.pool_g - 1) / c->p.pool_g;
+  a->kstage = c->kstage; a->qbar = c->qbar; a->qvec = c->qvec; a->scores = c->scores; a->kept = c->kept;
+  a->hist = c->sel_hist; a->run_hi = c->run_hi; a->cand = c->cand;
+  a->force_plain = c->force_plain;
+}
+
+void set_pending(xkv_cache* c, int n, const FramePlan& p) {
+  c->n_pending = n;
+  c->kk_pending = p.kk;
+  c->rold_pending = p.r_old;
+  c->evict_pending = p.evict;
+  c->first_pending = p.first;
+}
+
+bool selecting(const xkv_cache* c) {
+  return c->evict_pending && c->kk_pending > 0 && c->kk_pending < c->rold_pending;
+}
+
+bool kbar_fresh(const xkv_cache* c) {
+  return c->kbar_T == c->T && c->kbar_cur == c->cur && c->kbar_frames == c->frames;
+}
+
+void note_scored(xkv_cache* c) {
+  c->last_evicted = 0;
+  if (c->evict_pending) {
+    c->last_prunable = c->rold_pending;
+    c->last_kept = c->kk_pending;
+    c->last_evicted = c->rold_pending - c->kk_pending;
+  }
+}
+
+void note_packed(xkv_cache* c) {
+  const int n = c->n_pending;
+  if (c->first_pending) {
+    c->T_first = n;
+    c->rest_base = round_up(n, kTile);
+    c->T = n;
+  } else {
+    c->T = c->T_first + c->kk_pending + n;
+    c->cur ^= 1;
+  }
+  c->frames += 1;
+}
+
+}  // namespace
+
+extern "C" {
+
 int kv_append(xkv_cache* c, const void* k, const void* v, int32_t n, int64_t ts, int64_t hs, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;
   if (c->stage != 0) return XKV_E_STATE;
   if (n < 1 || n > c->p.max_frame_tokens || !aligned16(k) || !aligned16(v) || !strides_ok(ts, hs))
     return XKV_E_INVALID;
-  const bool first = (c->frames == 0);
-  int r_old = 0, kk = 0, evict = 0, dst_slot = 0;
-  if (!first) {
-    r_old = c->T - c->T_first;
-    evict = (c->T + n > c->p.budget) ? 1 : 0;               // pruning is triggered when T > L_max (Sec. 3.2)
-    kk = evict ? (c->p.budget - c->T_first - n) : r_old;    // k = max(0, L_max - T_first - T_current)
-    if (kk < 0) kk = 0;
-    dst_slot = c->rest_base + kk;
-    if (dst_slot + n > c->cap) return XKV_E_NOMEM;
-  }
-  const cudaError_t e = launch_append(c, k, v, n, ts, hs, dst_slot, first, reinterpret_cast<cudaStream_t>(stream));
-  if (e != cudaSuccess) return XKV_E_CUDA;
-  c->n_pending = n;
-  c->kk_pending = kk;
-  c->rold_pending = r_old;
-  c->evict_pending = evict;
-  c->first_pending = first ? 1 : 0;
+  FramePlan plan;
+  const int rc = plan_frame(c, n, &plan);
+  if (rc != XKV_OK) return rc;
+  set_pending(c, n, plan);
+  MaintArgs a;
+  maint_args(c, &a);
+  a.phases = kPhAppend;
+  a.k = reinterpret_cast<const __nv_bfloat16*>(k);
+  a.v = reinterpret_cast<const __nv_bfloat16*>(v);
+  a.ts_kv = ts; a.hs_kv = hs;
+  if (launch_maint(c, a, XKV_PROF_APPEND, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
   c->stage = 1;
   return XKV_OK;
 }
 
-// use_kbar: the stream step has computed the head means of the current cache beside the previous
-// attention (and made `stream` wait for them); the scoring then starts from those.
-static int score_evict_on(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t hs, xkv_stream stream,
-                          bool use_kbar) {
+int kv_score_evict(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t hs, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;
   if (c->stage != 1) return XKV_E_STATE;
   if (n != c->n_pending || !aligned16(q) || !strides_ok(ts, hs)) return XKV_E_INVALID;
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  c->last_evicted = 0;
-  if (c->evict_pending) {
-    const int r_old = c->rold_pending, kk = c->kk_pending;
-    c->last_prunable = r_old;
-    c->last_kept = kk;
-    c->last_evicted = r_old - kk;
-    if (kk > 0 && kk < r_old) {
-      if (launch_pool_q(c, q, n, ts, hs, st) != cudaSuccess) return XKV_E_CUDA;
-      const bool from_kbar = use_kbar && c->kbar_T == c->T && c->kbar_cur == c->cur && c->kbar_frames == c->frames &&
-                             r_old == c->T - c->T_first;
-      if (launch_score(c, r_old, st, from_kbar) != cudaSuccess) return XKV_E_CUDA;
-      if (launch_select(c, r_old, kk, st) != cudaSuccess) return XKV_E_CUDA;
+  note_scored(c);
+  if (selecting(c)) {
+    MaintArgs a;
+    maint_args(c, &a);
+    a.phases = kPhPool | kPhScore | kPhSel;
+    if (!kbar_fresh(c)) {          // head means of the keys (Eq. 4) of the cache as it stands
+      a.phases |= kPhKbar;
+      a.kbar_on_other = 0; a.kbar_lo = 0; a.kbar_hi = c->rold_pending;
     }
+    a.q = reinterpret_cast<const __nv_bfloat16*>(q);
+    a.ts_q = ts; a.hs_q = hs;
+    if (launch_maint(c, a, XKV_PROF_SCORE_EVICT, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
+    c->kbar_T = c->T; c->kbar_cur = c->cur; c->kbar_frames = c->frames;
   }
   c->stage = 2;
   return XKV_OK;
 }
 
-int kv_score_evict(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t hs, xkv_stream stream) {
-  return score_evict_on(c, q, n, ts, hs, stream, false);
-}
-
 int kv_quant_pack(xkv_cache* c, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;
   if (c->stage != 2) return XKV_E_STATE;
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  const int n = c->n_pending, kk = c->kk_pending;
-  const bool first = c->first_pending != 0;
-  const bool identity = !(c->evict_pending && kk > 0 && kk < c->rold_pending);
-  if (launch_pack(c, n, kk, identity, first, st) != cudaSuccess) return XKV_E_CUDA;
-  if (first) {
-    c->T_first = n;
-    c->rest_base = round_up(n, kTile);
-    c->T = n;
-  } else {
-    c->T = c->T_first + kk + n;
-    c->cur ^= 1;
+  MaintArgs a;
+  maint_args(c, &a);
+  if (c->p.kv_bits == 4) {
+    if (launch_regroup(c, a, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
+  } else if (c->kk_pending > 0) {                   // a 16-bit cache without survivors to move has nothing to do
+    a.phases = kPhPack;
+    if (launch_maint(c, a, XKV_PROF_PACK, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
   }
-  c->frames += 1;
+  note_packed(c);
   c->stage = 3;
   return XKV_OK;
 }
@@ -335,36 +408,49 @@ HostStepPipe* host_step_pipe() {
   return &p;
 }
 
-// One layer, one frame.  kv_append (it needs K and V and writes the staging area and the other
-// buffer set) runs on the side stream while the pooled query, the scores and the selection (they
-// need Q and read the current buffer set) run on the caller's stream; the two meet before
-// kv_quant_pack.  The side stream starts where the caller's stream stands, i.e. after the previous
-// layer's attention: nothing of a layer starts before the layer before it has finished.
+// One layer, one frame: the three maintenance calls as one launch, then -- on the library's side
+// stream, beside the attention -- the head means of the keys of the cache just built (Eq. 4), from
+// which the next frame's scoring starts.
 int run_layer(HostStepPipe* pipe, xkv_cache* c, const void* q, const void* k, const void* v, void* out, int32_t n,
               int64_t ts, int64_t hs, cudaStream_t st) {
   xkv_stream stream = reinterpret_cast<xkv_stream>(st);
-  bool ok = cudaEventRecord(pipe->fork, st) == cudaSuccess &&
-            cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess;
-  if (!ok) return XKV_E_CUDA;
-  int rc = kv_append(c, k, v, n, ts, hs, reinterpret_cast<xkv_stream>(pipe->side));
-  ok = cudaEventRecord(pipe->join, pipe->side) == cudaSuccess;
-  if (rc == XKV_OK && ok) {
-    const bool have_kbar = c->kbar_frames == c->frames && c->kbar_T == c->T && c->kbar_cur == c->cur;
-    if (have_kbar && cudaStreamWaitEvent(st, c->kbar_done, 0) != cudaSuccess) ok = false;
-    if (ok) rc = score_evict_on(c, q, n, ts, hs, stream, have_kbar);
+  if (c->stage != 0) return XKV_E_STATE;
+  if (n < 1 || n > c->p.max_frame_tokens || !aligned16(k) || !aligned16(v) || !aligned16(q) || !strides_ok(ts, hs))
+    return XKV_E_INVALID;
+  FramePlan plan;
+  int rc = plan_frame(c, n, &plan);
+  if (rc != XKV_OK) return rc;
+  set_pending(c, n, plan);
+  note_scored(c);
+  MaintArgs a;
+  maint_args(c, &a);
+  a.phases = kPhAppend;
+  if (c->p.kv_bits == 16 && c->kk_pending > 0) a.phases |= kPhPack;
+  if (selecting(c)) {
+    a.phases |= kPhPool | kPhScore | kPhSel;
+    if (kbar_fresh(c)) {
+      if (cudaStreamWaitEvent(st, c->kbar_done, 0) != cudaSuccess) return XKV_E_CUDA;
+    } else {
+      a.phases |= kPhKbar;
+      a.kbar_on_other = 0; a.kbar_lo = 0; a.kbar_hi = c->rold_pending;
+    }
   }
-  // the join is made also after an error, so that the side stream is never left behind
-  ok = ok && cudaStreamWaitEvent(st, pipe->join, 0) == cudaSuccess;
-  if (rc != XKV_OK) return rc;
-  if (!ok) return XKV_E_CUDA;
-  rc = kv_quant_pack(c, stream);
-  if (rc != XKV_OK) return rc;
-  // Head means of the keys of the cache just built (Eq. 4), for the next frame's scoring: on the
-  // side stream, beside the attention.  Not for the first frame (nothing after it yet).
+  a.q = reinterpret_cast<const __nv_bfloat16*>(q);
+  a.k = reinterpret_cast<const __nv_bfloat16*>(k);
+  a.v = reinterpret_cast<const __nv_bfloat16*>(v);
+  a.ts_q = a.ts_kv = ts; a.hs_q = a.hs_kv = hs;
+  if (launch_maint(c, a, XKV_PROF_MAINT, st) != cudaSuccess) return XKV_E_CUDA;
+  if (c->p.kv_bits == 4 && launch_regroup(c, a, st) != cudaSuccess) return XKV_E_CUDA;
+  note_packed(c);
+  c->stage = 3;
   if (c->T > c->T_first) {
-    ok = cudaEventRecord(pipe->fork, st) == cudaSuccess && cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess;
+    bool ok = cudaEventRecord(pipe->fork, st) == cudaSuccess && cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess;
     if (!ok) return XKV_E_CUDA;
-    const bool launched = launch_kbar(c, pipe->side) == cudaSuccess;
+    MaintArgs b;
+    maint_args(c, &b);
+    b.phases = kPhKbar;
+    b.kbar_on_other = 0; b.kbar_lo = 0; b.kbar_hi = c->T - c->T_first;
+    const bool launched = launch_maint(c, b, XKV_PROF_KBAR, pipe->side) == cudaSuccess;
     ok = cudaEventRecord(c->kbar_done, pipe->side) == cudaSuccess;
     // (the caller's stream waits for it at the end of the stream-step call, and at the next
     // frame's scoring)
@@ -539,6 +625,22 @@ int xkv_debug_force_plain(xkv_cache* c, int32_t on) {
 int xkv_debug_limit_attention_blocks(xkv_cache* c, int32_t max_blocks) {
   if (!c || max_blocks < 0) return XKV_E_INVALID;
   c->attn_max_blocks = max_blocks;
+  return XKV_OK;
+}
+
+int xkv_debug_head_means(xkv_cache* c, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  if (c->stage != 0) return XKV_E_STATE;
+  if (c->T <= c->T_first) return XKV_OK;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (c->kbar_done && cudaStreamWaitEvent(st, c->kbar_done, 0) != cudaSuccess) return XKV_E_CUDA;
+  MaintArgs a;
+  maint_args(c, &a);
+  a.phases = kPhKbar;
+  a.kbar_on_other = 0; a.kbar_lo = 0; a.kbar_hi = c->T - c->T_first;
+  if (launch_maint(c, a, XKV_PROF_KBAR, st) != cudaSuccess) return XKV_E_CUDA;
+  if (cudaEventRecord(c->kbar_done, st) != cudaSuccess) return XKV_E_CUDA;
+  c->kbar_T = c->T; c->kbar_cur = c->cur; c->kbar_frames = c->frames;
   return XKV_OK;
 }
 

@@ -24,6 +24,39 @@ struct BufSet {
   uint8_t* v;        // [H][cap][row_bytes]
   float2* vpar;      // [H][cap]          (scale, zero)
   int32_t* origin;   // [cap]
+  float* kbar;       // [cap][64] head means of the keys after the first frame (Eq. 4), by rest-local position
+  int32_t* kslot;    // [cap] quantise-once mode: parameter-table slot of each token's key group
+};
+
+// Phases of the maintenance kernel (bit mask) and its arguments.
+constexpr uint32_t kPhAppend = 1u, kPhPool = 2u, kPhKbar = 4u, kPhScore = 8u, kPhSel = 16u, kPhPack = 32u;
+struct MaintArgs {
+  uint32_t phases;
+  // the frame
+  const __nv_bfloat16* q; const __nv_bfloat16* k; const __nv_bfloat16* v;
+  int n;
+  int64_t ts_q, hs_q, ts_kv, hs_kv;
+  // the cache
+  int H, cap, max_n, frame, first;
+  BufSet cur, oth;                 // current buffer set (source) and the other one (destination)
+  int dst_slot;                    // physical slot of the frame's first token in the destination
+  int rest_base, r_old, kk, r_new, identity;
+  int n_special, pool_g, n_pooled;
+  int kbar_on_other, kbar_lo, kbar_hi;   // KBAR phase: buffer set and rest-local range
+  __nv_bfloat16* kstage;
+  float* qbar; float* qvec; float* scores;
+  int32_t* kept;
+  unsigned int* hist;
+  unsigned int* run_hi;            // [cap / 64] sure keeps of every 64-token run
+  unsigned long long* cand;        // [cap] candidates (key << 32 | ~position)
+  unsigned int* cand_count;        // counter of this launch
+  unsigned int* cand_count_next;   // counter of the next selecting launch (cleared by this one)
+  unsigned int* hist2;             // [256] histogram of the candidates' next 8 key bits
+  unsigned int* hist2_next;        // the next selecting launch's (cleared by this one)
+  int32_t* ref; int32_t* free_list; int* free_top;   // quantise-once mode: parameter-table bookkeeping
+  int force_plain;
+  unsigned int* bar; uint32_t bar_base;
+  int* status;
 };
 
 // Optional per-launch timing (xkv_profile_enable): one event pair per kernel launch.
@@ -52,8 +85,13 @@ struct xkv_cache {
   float* qvec;             // [64]
   float* scores;           // [cap]
   int32_t* kept;           // [cap]
-  unsigned int* counters;  // [8] device counters (self-resetting)
+  unsigned int* counters;  // device counters: [0] grid barrier (only grows), [2], [3] candidate counters,
+                           // [64..319], [320..575] the two sub-histograms of the selection
+  uint32_t bar_base;       // value of the barrier counter when the next maintenance kernel starts
+  int sel_parity;          // which candidate counter the next selecting launch uses
   unsigned int* sel_hist;  // [4096] histogram of the top 12 bits of the score keys (self-clearing)
+  unsigned int* run_hi;    // [cap / 64]
+  unsigned long long* cand;  // [cap]
   int* status;             // device status word
   float* attn_part;        // split-KV partials of the attention kernel
   size_t attn_part_bytes;
@@ -65,9 +103,8 @@ struct xkv_cache {
   int force_plain;         // 1: kernels take the plain (conversion-based) arithmetic forms everywhere
   int tail_mode;           // 1: the stream-step calls attend with the step's K, V unquantised
   int attn_max_blocks;     // test hook: cap on the thread blocks of the tensor-core attention (0: none)
-  // head means of the keys after the first frame (Eq. 4), filled by the stream step beside the
-  // attention and used by the next step's scoring when the cache has not changed since
-  float* kbar;             // [cap][64]
+  // head means of the keys after the first frame (Eq. 4; BufSet::kbar), filled by the stream step
+  // beside the attention and used by the next step's scoring when the cache has not changed since
   cudaEvent_t kbar_done;
   int kbar_T, kbar_cur, kbar_frames;   // state of the cache the array was computed from (-1: none)
   xkv::Profiler* prof;
@@ -99,13 +136,11 @@ struct LaunchScope {
 // ---- launchers implemented in the kernel translation units -------------------
 // All return cudaError_t of the launch (cudaGetLastError) and count launches.
 
-cudaError_t launch_append(xkv_cache* c, const void* k, const void* v, int n, int64_t ts, int64_t hs,
-                          int dst_slot, bool first, cudaStream_t st);
-cudaError_t launch_pool_q(xkv_cache* c, const void* q, int n, int64_t ts, int64_t hs, cudaStream_t st);
-cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st, bool from_kbar = false);
-cudaError_t launch_kbar(xkv_cache* c, cudaStream_t st);
-cudaError_t launch_select(xkv_cache* c, int r_old, int k, cudaStream_t st);
-cudaError_t launch_pack(xkv_cache* c, int n, int kk, bool identity, bool first, cudaStream_t st);
+// The maintenance kernel with the phases in a.phases (cooperative when it has a grid barrier).
+// Fills in the barrier and status fields of `a`; everything else is the caller's.
+cudaError_t launch_maint(xkv_cache* c, MaintArgs& a, int prof_cat, cudaStream_t st);
+// kv_quant_pack of a 4-bit cache: key regroup + re-quantisation fused with the survivor gather.
+cudaError_t launch_regroup(xkv_cache* c, const MaintArgs& a, cudaStream_t st);
 cudaError_t launch_attn_simple(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
                                float scale, cudaStream_t st);
 // Returns cudaErrorNotSupported when the tensor-core kernel cannot take the call.

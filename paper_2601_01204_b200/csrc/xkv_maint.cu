@@ -1,8 +1,33 @@
-// Cache-maintenance kernels: append (+ per-token value quantisation), pooled
-// query, importance scores, top-k selection, key regroup/re-quantisation and the
+// Cache maintenance: append (+ per-token value quantisation), pooled query,
+// importance scores, top-k selection, key regroup / re-quantisation and the
 // survivor gather.  All bandwidth- or latency-bound; fp32 arithmetic whose every
 // operation and order is fixed, because it decides integers (kept indices, 4-bit
 // codes) that must be reproducible bit for bit.
+//
+// One persistent kernel, launched cooperatively with two thread blocks per SM,
+// runs the phases that a call needs, separated by grid-wide barriers:
+//
+//   APPEND  values quantised per token (Eq. 7-9) into their final slot; keys staged
+//           (4-bit) or copied (16-bit)                                 [kv_append]
+//   POOL    pooled query rows, Eq. 2-3                                 [kv_score_evict]
+//   KBAR    head means of the cached keys after the first frame, Eq. 4, when the
+//           stored ones are stale
+//   ---- barrier ----
+//   SCORE   row mean of the pooled query, scores S = w . K-bar (Eq. 5-6), histogram
+//           of the top 12 bits of the score keys
+//   ---- barrier ----
+//   SEL1    every block finds the histogram bin that holds the k-th largest key;
+//           keys in higher bins are kept, keys in that bin become candidates
+//   ---- barrier ----
+//   SEL2    every block finds the k-th largest (key, position) among the candidates
+//           by bisection and writes the kept positions of its own tokens in order
+//   ---- barrier ----
+//   PACK    16-bit caches: the survivor gather                          [kv_quant_pack]
+//
+// xkv_stream_step runs all of them in one launch; the per-call entry points launch
+// the same kernel with the phases of that call.  The 4-bit kv_quant_pack (key regroup +
+// re-quantisation, Eq. 7-9, fused with the survivor gather) is a kernel of its own,
+// launched right behind.
 #include <stdlib.h>
 
 #include <mutex>
@@ -10,6 +35,12 @@
 #include "xkv_internal.cuh"
 
 namespace xkv {
+
+namespace {
+
+constexpr int kMT = 512;                 // threads per block
+constexpr int kBlocksPerSM = 2;
+constexpr uint32_t kBarSpin = 1u << 21;  // polls of a grid barrier before it gives up (about 0.1 s)
 
 // ---------------------------------------------------------------------------
 // Eq. 7-8, fixed-order fp32:  s = (max-min)/15 (1 if the range is 0),
@@ -48,112 +79,17 @@ __device__ __forceinline__ void bf16x8_to_float(const uint4& u, float (&x)[8]) {
   }
 }
 
-// Eq. 10 for the 8 channels of one packed word: x~ = s * (q - z).
-__device__ __forceinline__ void dequant8(uint32_t word, const float2* __restrict__ par, float (&x)[8]) {
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const float2 sz = par[j];
-    const float q = (float)((word >> nib_shift(j)) & 0xFu);
-    x[j] = __fmul_rn(sz.x, __fsub_rn(q, sz.y));
-  }
-}
-
-// ---------------------------------------------------------------------------
-// kv_append.  Thread = (head, token, 8-channel word).  Values: per-token
-// min/max over the 64 channels by xor-shuffle inside the 8-lane group, then
-// codes -> one 32-bit word per lane.  Keys: copied to the staging buffer (4-bit)
-// or to their final slot (16-bit).
-// ---------------------------------------------------------------------------
-template <int BITS>
-__global__ void __launch_bounds__(256)
-append_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, int n,
-              int64_t ts, int64_t hs, int H, int cap, int max_n, int dst_slot, int frame,
-              BufSet d0, BufSet d1, bool two, __nv_bfloat16* __restrict__ kstage) {
-  const long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const int w = (int)(g & 7);
-  const long long th = g >> 3;
-  const bool valid = th < (long long)H * n;
-  const int h = valid ? (int)(th / n) : 0;
-  const int tok = valid ? (int)(th % n) : 0;
-  const int64_t src = (int64_t)h * hs + (int64_t)tok * ts + 8 * w;
-  const uint4 kv = *reinterpret_cast<const uint4*>(k + src);
-  const uint4 vv = *reinterpret_cast<const uint4*>(v + src);
-  const size_t slot = (size_t)h * cap + dst_slot + tok;
-
-  if (BITS == 16) {
-    if (valid) {
-      *reinterpret_cast<uint4*>(d0.k + slot * 128 + 16 * w) = kv;
-      *reinterpret_cast<uint4*>(d0.v + slot * 128 + 16 * w) = vv;
-      if (two) {
-        *reinterpret_cast<uint4*>(d1.k + slot * 128 + 16 * w) = kv;
-        *reinterpret_cast<uint4*>(d1.v + slot * 128 + 16 * w) = vv;
-      }
-    }
-  } else {
-    float x[8];
-    bf16x8_to_float(vv, x);
-    float mn = x[0], mx = x[0];
-#pragma unroll
-    for (int j = 1; j < 8; ++j) { mn = fminf(mn, x[j]); mx = fmaxf(mx, x[j]); }
-#pragma unroll
-    for (int o = 1; o < 8; o <<= 1) {
-      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    }
-    float s, inv, z;
-    quant_params(mn, mx, s, inv, z);
-    uint32_t c[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) c[j] = quant_code(x[j], inv, z);
-    const uint32_t word = pack8(c);
-    if (valid) {
-      *reinterpret_cast<uint32_t*>(d0.v + slot * 32 + 4 * w) = word;
-      if (w == 0) d0.vpar[slot] = make_float2(s, z);
-      if (two) {
-        *reinterpret_cast<uint32_t*>(d1.v + slot * 32 + 4 * w) = word;
-        if (w == 0) d1.vpar[slot] = make_float2(s, z);
-      }
-      *reinterpret_cast<uint4*>(kstage + ((size_t)h * max_n + tok) * 64 + 8 * w) = kv;
-    }
-  }
-  if (valid && h == 0 && w == 0) {
-    const int32_t o = (frame << 16) | tok;
-    d0.origin[dst_slot + tok] = o;
-    if (two) d1.origin[dst_slot + tok] = o;
-  }
-}
-
-cudaError_t launch_append(xkv_cache* c, const void* k, const void* v, int n, int64_t ts, int64_t hs,
-                          int dst_slot, bool first, cudaStream_t st) {
-  const long long threads = (long long)c->p.n_heads * n * 8;
-  const int blocks = (int)((threads + 255) / 256);
-  const BufSet d0 = c->buf[c->cur ^ 1];
-  const BufSet d1 = c->buf[c->cur];
-  auto kk = reinterpret_cast<const __nv_bfloat16*>(k);
-  auto vv = reinterpret_cast<const __nv_bfloat16*>(v);
-  LaunchScope ls(c, XKV_PROF_APPEND, st);
-  if (c->p.kv_bits == 16)
-    append_kernel<16><<<blocks, 256, 0, st>>>(kk, vv, n, ts, hs, c->p.n_heads, c->cap,
-                                              c->p.max_frame_tokens, dst_slot, c->frames + 1, d0, d1,
-                                              first, c->kstage);
-  else
-    append_kernel<4><<<blocks, 256, 0, st>>>(kk, vv, n, ts, hs, c->p.n_heads, c->cap,
-                                             c->p.max_frame_tokens, dst_slot, c->frames + 1, d0, d1,
-                                             first, c->kstage);
-  return cudaGetLastError();
-}
-
 // ---------------------------------------------------------------------------
 // Conversion-free forms of Eq. 10 and Eq. 7.  They produce the same fp32 results
-// as dequant8 / quant_code whenever their preconditions hold (callers check them
-// and take the plain forms otherwise), but use no int<->float conversion or
-// round instruction, which issue at a quarter of the fp32 rate.
+// as the plain forms whenever their preconditions hold (callers check them and
+// take the plain forms otherwise), but use no int<->float conversion or round
+// instruction, which issue at a quarter of the fp32 rate.
 //
 // A 4-bit code q sitting at bit 4i of a word, OR-ed into the mantissa of
 // 2^(23-4i), is the float 2^(23-4i) + q.  Subtracting 2^(23-4i) + z (exact for
 // integer |z| < 2^22) gives q - z exactly, like float(q) - z.
 // ---------------------------------------------------------------------------
-constexpr float kZLimit = 4194304.f;     // 2^22
+constexpr float kZLimit = 4194304.f;       // 2^22
 constexpr float kRoundMagic = 12582912.f;  // 1.5 * 2^23: y + magic has rint(y) in its mantissa for |y| < 2^22
 
 __device__ __forceinline__ uint32_t magic_bits(int j) { return 0x4B000000u - (uint32_t)(j >> 1) * 0x02000000u; }
@@ -191,315 +127,44 @@ __device__ __forceinline__ void dequant8_plain(uint32_t word, const float2* par,
   for (int j = 0; j < 8; ++j) x[j] = dequant_one_call((word >> nib_shift(j)) & 0xFu, par[j].x, par[j].y);
 }
 
-// ---------------------------------------------------------------------------
-// Pooled query, Eq. 2-3, then the row mean that Eq. 5-6 reduce to.
-// One CTA per pooled row i; thread (c, hs) builds pooled[h][i][c] for heads
-// h = hs, hs+16, ... (sequential sum over the group's tokens, divided by the
-// group size); threads with hs == 0 add the heads in order and scale by 1/H.
-// The last CTA to finish adds the rows in order and divides by N_pooled.
-// Loads are issued in batches ahead of the (ordered) additions.
-// ---------------------------------------------------------------------------
-constexpr int kPoolRows = 128;   // pooled rows staged in shared memory at a time by the last CTA
-
-__global__ void __launch_bounds__(1024)
-pool_q_kernel(const __nv_bfloat16* __restrict__ q, int n, int64_t ts, int64_t hs, int H, int n_special,
-              int g, int n_pooled, float* __restrict__ qbar, float* __restrict__ qvec,
-              unsigned int* __restrict__ counter) {
-  extern __shared__ float s_pooled[];  // [H][64]
-  __shared__ float s_rows[kPoolRows * 64];
-  __shared__ float s_acc[64];
-  __shared__ bool s_last;
-  const int i = blockIdx.x;
-  const int c = threadIdx.x;   // 0..63
-  const int hslot = threadIdx.y;
-  int a, b;
-  if (i < n_special) { a = i; b = i + 1; }
-  else { a = n_special + (i - n_special) * g; b = min(a + g, n); }
-  for (int h = hslot; h < H; h += blockDim.y) {
-    const __nv_bfloat16* base = q + (int64_t)h * hs + c;
-    float acc = 0.f;
-    for (int t0 = a; t0 < b; t0 += 16) {
-      float x[16];
-#pragma unroll
-      for (int u = 0; u < 16; ++u) x[u] = (t0 + u < b) ? __bfloat162float(base[(int64_t)(t0 + u) * ts]) : 0.f;
-#pragma unroll
-      for (int u = 0; u < 16; ++u)
-        if (t0 + u < b) acc = (t0 + u == a) ? x[u] : __fadd_rn(acc, x[u]);
-    }
-    if (i >= n_special) acc = __fdiv_rn(acc, (float)(b - a));
-    s_pooled[h * 64 + c] = acc;
-  }
-  __syncthreads();
-  if (hslot == 0) {
-    // (reads in batches ahead of the ordered additions)
-    float acc = 0.f;
-    for (int h0 = 0; h0 < H; h0 += 16) {
-      float v[16];
-#pragma unroll
-      for (int u = 0; u < 16; ++u) v[u] = (h0 + u < H) ? s_pooled[(h0 + u) * 64 + c] : 0.f;
-#pragma unroll
-      for (int u = 0; u < 16; ++u)
-        if (h0 + u < H) acc = (h0 + u == 0) ? v[u] : __fadd_rn(acc, v[u]);
-    }
-    const float inv_h = __fdiv_rn(1.f, (float)H);
-    __stcg(&qbar[i * 64 + c], __fmul_rn(acc, inv_h));
-  }
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0 && threadIdx.y == 0) {
-    const unsigned int done = atomicAdd(counter, 1u);
-    s_last = (done == (unsigned int)n_pooled - 1u);
-  }
-  __syncthreads();
-  if (s_last) {
-    __threadfence();
-    // all threads fetch the rows (one round trip), then one thread per channel adds them in order
-    const int tid = threadIdx.y * 64 + threadIdx.x, nthr = blockDim.y * 64;
-    for (int r0 = 0; r0 < n_pooled; r0 += kPoolRows) {
-      const int rows = min(kPoolRows, n_pooled - r0);
-      __syncthreads();
-      for (int e = tid; e < rows * 64; e += nthr) s_rows[e] = __ldcg(&qbar[r0 * 64 + e]);
-      __syncthreads();
-      if (hslot == 0) {
-        float acc = (r0 == 0) ? 0.f : s_acc[c];
-        for (int q0 = 0; q0 < rows; q0 += 16) {
-          float v[16];
-#pragma unroll
-          for (int u = 0; u < 16; ++u) v[u] = (q0 + u < rows) ? s_rows[(q0 + u) * 64 + c] : 0.f;
-#pragma unroll
-          for (int u = 0; u < 16; ++u)
-            if (q0 + u < rows) acc = (r0 == 0 && q0 + u == 0) ? v[u] : __fadd_rn(acc, v[u]);
-        }
-        s_acc[c] = acc;
-      }
-    }
-    if (hslot == 0) qvec[c] = __fdiv_rn(s_acc[c], (float)n_pooled);
-    if (threadIdx.x == 0 && threadIdx.y == 0) *counter = 0u;  // re-arm for the next launch
-  }
-}
-
-cudaError_t launch_pool_q(xkv_cache* c, const void* q, int n, int64_t ts, int64_t hs, cudaStream_t st) {
-  const int H = c->p.n_heads;
-  const int nsp = min(c->p.n_special, n);
-  const int np = nsp + (n - nsp + c->p.pool_g - 1) / c->p.pool_g;
-  const dim3 block(64, H < 16 ? H : 16);
-  LaunchScope ls(c, XKV_PROF_POOL, st);
-  pool_q_kernel<<<np, block, (size_t)H * 64 * sizeof(float), st>>>(
-      reinterpret_cast<const __nv_bfloat16*>(q), n, ts, hs, H, nsp, c->p.pool_g, np, c->qbar, c->qvec,
-      c->counters);
-  return cudaGetLastError();
-}
-
-// ---------------------------------------------------------------------------
-// Scores, Eq. 4-6.  One CTA per 64-slot key group of the middle segment (the
-// rest segment starts on a 128-slot boundary, so a CTA's tokens share their
-// quantisation parameters).  Thread = (token, 8-channel word): dequantise the
-// word of every head in order (Eq. 10), accumulate the head sum sequentially,
-// scale by 1/H (Eq. 4), multiply by the query vector, and add the 64 products
-// with a balanced tree: three levels inside the lane, three by xor-shuffle.
-// The words of sixteen heads (4-bit; four 16-byte pieces for 16-bit storage) are fetched ahead of
-// their (ordered) use.
-// ---------------------------------------------------------------------------
 // Unsigned key whose order is the total order of fp32 bit patterns (so that -0 < +0).
 __device__ __forceinline__ uint32_t order_key(float f) {
   const uint32_t u = __float_as_uint(f);
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-constexpr int kSelBins = 4096;          // histogram of the top 12 key bits, filled by the score kernel
-
-// MODE 0: the whole computation.  MODE 1: only Eq. 4, the head means K-bar[i][c] (fp32, exactly the
-// value MODE 0 holds at that point) stored to `kbar` -- run beside the attention of the step that
-// built the cache.  MODE 2: only Eq. 5-6 from a stored K-bar -- the next step's scoring.  1 + 2
-// perform the operations of 0 in the same order, so the scores are the same bits.
-template <int BITS, int MODE>
-__global__ void __launch_bounds__(512)
-score_kernel(BufSet cur, int H, int cap, int rest_base, int r_old, const float* __restrict__ qvec,
-             float* __restrict__ scores, unsigned int* __restrict__ hist, int force_plain,
-             float* __restrict__ kbar) {
-  // Parameters of the CTA's key group.  Fast path: float4 [H][4][8] = (s, magic + z) of channels
-  // 8w + 2v and 8w + 2v + 1 at [h][v][w], so that the eight lanes of a quarter-warp read
-  // consecutive 16-byte chunks.  Plain path: float2 (s, z) [H][64].
-  extern __shared__ __align__(16) float2 s_par[];
-  __shared__ float s_w[64];
-  const int tid = threadIdx.x;
-  const int w = tid & 7;
-  const int tok = tid >> 3;
-  const int i = blockIdx.x * 64 + tok;          // rest-local index
-  const int slot = rest_base + i;
-  const int grp = (rest_base >> 6) + blockIdx.x;
-  bool plain = false;
-  if (BITS == 4 && MODE != 2) {
-    int big = force_plain;
-    float2 mine[4];                              // H <= 64: at most 8 elements per thread, 4 at a time
-    for (int e0 = 0; e0 < H * 64; e0 += 2048) {
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int e = e0 + u * 512 + tid;
-        mine[u] = make_float2(0.f, 0.f);
-        if (e < H * 64) mine[u] = cur.kpar[((size_t)(e >> 6) * (cap >> 6) + grp) * 64 + (e & 63)];
-        big |= !(fabsf(mine[u].y) < kZLimit);
-      }
-      // the layout depends on the path, which the whole CTA has to agree on: H * 64 <= 2048 makes
-      // this loop run once for H <= 32; for more heads the parameters are re-read below
-      if (e0 == 0 && H * 64 <= 2048) break;
-    }
-    plain = __syncthreads_or(big) != 0;
-    for (int e0 = 0; e0 < H * 64; e0 += 2048) {
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int e = e0 + u * 512 + tid;
-        if (e < H * 64) {
-          float2 sz = mine[u];
-          if (H * 64 > 2048) sz = cur.kpar[((size_t)(e >> 6) * (cap >> 6) + grp) * 64 + (e & 63)];
-          if (plain) {
-            s_par[e] = sz;
-          } else {
-            const int h = e >> 6, ch = e & 63;
-            sz.y = __fadd_rn(magic_val(ch & 7), sz.y);
-            // [h][v = (ch & 7) >> 1][w = ch >> 3], two float2 per float4
-            s_par[((h * 4 + ((ch & 7) >> 1)) * 8 + (ch >> 3)) * 2 + (ch & 1)] = sz;
-          }
-        }
-      }
-    }
-  }
-  if (MODE != 1 && tid < 64) s_w[tid] = qvec[tid];
-  __syncthreads();
-  const bool valid = i < r_old;
-  float acc[8];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-  constexpr int kHB = (BITS == 4) ? 16 : 4;     // heads whose words are in flight together
-  for (int h0 = 0; MODE != 2 && h0 < H; h0 += kHB) {
-    uint32_t word[BITS == 4 ? kHB : 1];
-    uint4 wide[BITS == 4 ? 1 : kHB];
-#pragma unroll
-    for (int u = 0; u < kHB; ++u) {
-      const int h = h0 + u;
-      if (BITS == 4) word[u] = 0u; else wide[u] = make_uint4(0, 0, 0, 0);
-      if (valid && h < H) {
-        if (BITS == 4) word[u] = *reinterpret_cast<const uint32_t*>(cur.k + ((size_t)h * cap + slot) * 32 + 4 * w);
-        else wide[u] = *reinterpret_cast<const uint4*>(cur.k + ((size_t)h * cap + slot) * 128 + 16 * w);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < kHB; ++u) {
-      const int h = h0 + u;
-      if (h < H) {
-        float x[8];
-        if (BITS == 4) {
-          if (plain) {
-            dequant8_plain(word[BITS == 4 ? u : 0], s_par + h * 64 + 8 * w, x);
-          } else {
-            float2 par[8];
-            const float4* pp = reinterpret_cast<const float4*>(s_par) + h * 32 + w;
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              const float4 t = pp[v * 8];
-              par[2 * v] = make_float2(t.x, t.y);
-              par[2 * v + 1] = make_float2(t.z, t.w);
-            }
-            dequant8_magic(word[BITS == 4 ? u : 0], par, x);
-          }
-        } else {
-          bf16x8_to_float(wide[BITS == 4 ? 0 : u], x);
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] = (h == 0) ? x[j] : __fadd_rn(acc[j], x[j]);
-      }
-    }
-  }
-  const float inv_h = __fdiv_rn(1.f, (float)H);
-  float kb[8];
-  if (MODE == 2) {
-    const float4* src = reinterpret_cast<const float4*>(kbar + (size_t)(valid ? i : 0) * 64 + 8 * w);
-    const float4 x = src[0], y = src[1];
-    kb[0] = x.x; kb[1] = x.y; kb[2] = x.z; kb[3] = x.w; kb[4] = y.x; kb[5] = y.y; kb[6] = y.z; kb[7] = y.w;
-  } else {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) kb[j] = __fmul_rn(acc[j], inv_h);
-  }
-  if (MODE == 1) {
-    if (valid) {
-      float4* dst = reinterpret_cast<float4*>(kbar + (size_t)i * 64 + 8 * w);
-      dst[0] = make_float4(kb[0], kb[1], kb[2], kb[3]);
-      dst[1] = make_float4(kb[4], kb[5], kb[6], kb[7]);
-    }
-    return;
-  }
-  float p[8];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) p[j] = __fmul_rn(kb[j], s_w[8 * w + j]);
-  float t0 = __fadd_rn(p[0], p[1]), t1 = __fadd_rn(p[2], p[3]);
-  float t2 = __fadd_rn(p[4], p[5]), t3 = __fadd_rn(p[6], p[7]);
-  t0 = __fadd_rn(t0, t1);
-  t2 = __fadd_rn(t2, t3);
-  float s = __fadd_rn(t0, t2);
-#pragma unroll
-  for (int o = 1; o < 8; o <<= 1) s = __fadd_rn(s, __shfl_xor_sync(0xffffffffu, s, o));
-  if (valid && w == 0) {
-    scores[i] = s;
-    atomicAdd(&hist[order_key(s) >> 20], 1u);      // first digit of the selection (the select kernel clears it)
-  }
+__device__ __forceinline__ uint32_t ld_acquire_u32(const unsigned int* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
 }
 
-cudaError_t launch_score(xkv_cache* c, int r_old, cudaStream_t st, bool from_kbar) {
-  const int blocks = (r_old + 63) / 64;
-  const size_t smem = (size_t)c->p.n_heads * 64 * sizeof(float2);
-  LaunchScope ls(c, XKV_PROF_SCORE, st);
-  const BufSet& b = c->buf[c->cur];
-  const int H = c->p.n_heads;
-  if (from_kbar) {
-    if (c->p.kv_bits == 16)
-      score_kernel<16, 2><<<blocks, 512, smem, st>>>(b, H, c->cap, c->rest_base, r_old, c->qvec, c->scores, c->sel_hist,
-                                                     c->force_plain, c->kbar);
-    else
-      score_kernel<4, 2><<<blocks, 512, smem, st>>>(b, H, c->cap, c->rest_base, r_old, c->qvec, c->scores, c->sel_hist,
-                                                    c->force_plain, c->kbar);
-  } else if (c->p.kv_bits == 16) {
-    score_kernel<16, 0><<<blocks, 512, smem, st>>>(b, H, c->cap, c->rest_base, r_old, c->qvec, c->scores, c->sel_hist,
-                                                   c->force_plain, nullptr);
-  } else {
-    score_kernel<4, 0><<<blocks, 512, smem, st>>>(b, H, c->cap, c->rest_base, r_old, c->qvec, c->scores, c->sel_hist,
-                                                  c->force_plain, nullptr);
-  }
-  return cudaGetLastError();
-}
+constexpr int kSelBins = 4096;       // histogram of the top 12 key bits
+constexpr int kHistCopies = 4;       // copies of the histogram (a block adds to copy blockIdx mod 4: fewer collisions)
+constexpr int kPoolRows = 120;       // pooled rows staged in shared memory at a time
+constexpr int kCandSmem = 4096;      // candidates a block holds in shared memory
+constexpr int kSubBins = 256;        // second histogram: the next 8 key bits of the candidates
+constexpr int kSubList = 512;        // candidates of one sub-bin that a block lists in shared memory
 
-// Head means of the keys after the first frame, of the cache as it stands (after kv_quant_pack).
-cudaError_t launch_kbar(xkv_cache* c, cudaStream_t st) {
-  const int r = c->T - c->T_first;
-  if (r <= 0) return cudaSuccess;
-  const int blocks = (r + 63) / 64;
-  const size_t smem = (size_t)c->p.n_heads * 64 * sizeof(float2);
-  LaunchScope ls(c, XKV_PROF_KBAR, st);
-  const BufSet& b = c->buf[c->cur];
-  if (c->p.kv_bits == 16)
-    score_kernel<16, 1><<<blocks, 512, smem, st>>>(b, c->p.n_heads, c->cap, c->rest_base, r, nullptr, nullptr, nullptr,
-                                                   c->force_plain, c->kbar);
-  else
-    score_kernel<4, 1><<<blocks, 512, smem, st>>>(b, c->p.n_heads, c->cap, c->rest_base, r, nullptr, nullptr, nullptr,
-                                                  c->force_plain, c->kbar);
-  return cudaGetLastError();
-}
+// Shared memory of a block, one phase at a time.
+union __align__(16) Smem {
+  struct { float pooled[64 * 64]; } pool;                                          // [H <= 64][64]
+  struct { float2 par[64 * 64]; } kbar;                                            // [H][64] key parameters of one group
+  struct { float w[64]; float rows[kPoolRows * 64]; } score;
+  struct { unsigned long long cand[kCandSmem]; unsigned long long list[kSubList]; } sel;   // (key << 32) | ~position
+};
 
-// ---------------------------------------------------------------------------
-// Top-k of the scores (Sec. 3.2).  One CTA.  The order keys are held in shared
-// memory when they fit.  The k-th largest key tau is found in two stages: the
-// histogram of the top 12 bits (counted by the score kernel with global atomics)
-// gives the bin that holds it; the keys of that bin, normally a few hundred, are
-// collected and the remaining 20 bits are found by bisection on them.  Then a
-// stable compaction keeps every key above tau and the first (k - #above) keys
-// equal to it.  Each thread owns a run of consecutive positions.
-// ---------------------------------------------------------------------------
-constexpr int kSelThreads = 1024;
-constexpr int kSelSmemKeys = 44 * 1024;   // keys held in shared memory (176 KB)
-constexpr int kSelCand = 4096;            // candidates collected from the bin of tau
+struct Shared {
+  Smem u;
+  unsigned int warp[33];
+  unsigned int acc;
+  unsigned int bin, need;          // result of SEL1, used by SEL2
+  unsigned int sub, need2, n_list; // SEL2: the sub-bin of the k-th largest key, its rank there, listed candidates
+  int abort_flag;
+};
 
-__device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned int* s_warp,
-                                                        unsigned int& total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+__device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned int* s_warp, unsigned int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;     // 16 warps
   unsigned int x = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -509,15 +174,15 @@ __device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned
   if (lane == 31) s_warp[warp] = x;
   __syncthreads();
   if (warp == 0) {
-    unsigned int t = s_warp[lane];
+    const unsigned int t = (lane < kMT / 32) ? s_warp[lane] : 0u;
     unsigned int y = t;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const unsigned int z = __shfl_up_sync(0xffffffffu, y, o);
       if (lane >= o) y += z;
     }
-    s_warp[lane] = y - t;          // exclusive warp offsets
-    if (lane == 31) s_warp[32] = y;  // grand total
+    s_warp[lane] = y - t;
+    if (lane == 31) s_warp[32] = y;
   }
   __syncthreads();
   const unsigned int res = s_warp[warp] + x - v;
@@ -526,7 +191,7 @@ __device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned
   return res;
 }
 
-// sum of v over the block (all threads get it); s_acc must be zero on entry and is zero on exit
+// sum of v over the block (all threads get it); *s_acc must be zero on entry and is zero on exit
 __device__ __forceinline__ unsigned int block_sum(unsigned int v, unsigned int* s_acc) {
   v = __reduce_add_sync(0xffffffffu, v);
   if ((threadIdx.x & 31) == 0 && v) atomicAdd(s_acc, v);
@@ -534,180 +199,490 @@ __device__ __forceinline__ unsigned int block_sum(unsigned int v, unsigned int* 
   const unsigned int t = *s_acc;
   __syncthreads();
   if (threadIdx.x == 0) *s_acc = 0u;
+  __syncthreads();
   return t;
 }
 
-// KPT > 0: every thread's run has at most KPT keys and is held in registers after the first read.
-template <bool IN_SMEM, int KPT>
-__global__ void __launch_bounds__(kSelThreads)
-select_kernel(const float* __restrict__ scores, int tp, int k, int32_t* __restrict__ kept,
-              unsigned int* __restrict__ hist) {
-  extern __shared__ uint32_t s_keys[];
-  __shared__ uint32_t s_cand[kSelCand];
-  __shared__ unsigned int s_warp[33];
-  __shared__ unsigned int s_bin, s_need, s_ncand, s_acc;
-  const int tid = threadIdx.x;
-  const int lane = tid & 31;
-  // ---- stage 1: the bin of tau from the 12-bit histogram (thread t owns 4 bins counted from the top) ----
-  unsigned int hb[4], own = 0u;
-  {
-    const uint4 h4 = *reinterpret_cast<const uint4*>(hist + kSelBins - 4 - 4 * tid);   // bins 4095-4t-3 .. 4095-4t
-    hb[0] = h4.w; hb[1] = h4.z; hb[2] = h4.y; hb[3] = h4.x;
+// Grid-wide barrier.  Every block arrives once per barrier; the counter only grows (the host
+// passes the value it had when the kernel was launched).  The wait is bounded: when it runs out
+// the block records XKV_E_TIMEOUT and the kernel winds down without touching anything further.
+__device__ __forceinline__ bool grid_barrier(const MaintArgs& a, uint32_t& epoch, Shared& sh) {
+  __syncthreads();
+  if (threadIdx.x == 0 && !sh.abort_flag) {
+    __threadfence();
+    atomicAdd(a.bar, 1u);
+    const uint32_t target = a.bar_base + (epoch + 1u) * gridDim.x;
+    uint32_t it = 0;
+    while ((int)(ld_acquire_u32(a.bar) - target) < 0) {
+      if (++it > kBarSpin) {
+        sh.abort_flag = 1;
+        atomicExch(a.status, (int)XKV_E_TIMEOUT);
+        break;
+      }
+      __nanosleep(40);
+    }
+    __threadfence();
   }
-  if (IN_SMEM)
-    for (int j = tid; j < tp; j += kSelThreads) s_keys[j] = order_key(scores[j]);
-  if (tid == 0) { s_ncand = 0u; s_acc = 0u; }
-  auto key_at = [&](int j) -> uint32_t { return IN_SMEM ? s_keys[j] : order_key(scores[j]); };
-  *reinterpret_cast<uint4*>(hist + kSelBins - 4 - 4 * tid) = make_uint4(0u, 0u, 0u, 0u);   // ready for the next evicting step
+  ++epoch;
+  __syncthreads();
+  return sh.abort_flag == 0;
+}
+
+// ---------------------------------------------------------------------------
+// APPEND.  Thread = (head, token, 8-channel word).  Values: per-token min/max over
+// the 64 channels by xor-shuffle inside the 8-lane group, then codes -> one 32-bit
+// word per lane.  Keys: copied to the staging buffer (4-bit) or to their final
+// slot (16-bit).
+// ---------------------------------------------------------------------------
+template <int BITS>
+__device__ __forceinline__ void phase_append(const MaintArgs& a) {
+  const long long items = (long long)a.H * a.n * 8;
+  const int passes = (int)((items + kMT - 1) / kMT);
+  const BufSet& d0 = a.oth;
+  const BufSet& d1 = a.cur;
+  const bool two = a.first != 0;
+  // pass p goes to block G - 1 - (p mod G): the blocks that hold no pooled row start first
+  for (int p = (int)gridDim.x - 1 - (int)blockIdx.x; p < passes; p += gridDim.x) {
+    const long long g = (long long)p * kMT + threadIdx.x;
+    const int w = (int)(g & 7);
+    const long long th = g >> 3;
+    const bool valid = th < (long long)a.H * a.n;
+    const int h = valid ? (int)(th / a.n) : 0;
+    const int tok = valid ? (int)(th % a.n) : 0;
+    const int64_t src = (int64_t)h * a.hs_kv + (int64_t)tok * a.ts_kv + 8 * w;
+    const uint4 kv = *reinterpret_cast<const uint4*>(a.k + src);
+    const uint4 vv = *reinterpret_cast<const uint4*>(a.v + src);
+    const size_t slot = (size_t)h * a.cap + a.dst_slot + tok;
+    if (BITS == 16) {
+      if (valid) {
+        *reinterpret_cast<uint4*>(d0.k + slot * 128 + 16 * w) = kv;
+        *reinterpret_cast<uint4*>(d0.v + slot * 128 + 16 * w) = vv;
+        if (two) {
+          *reinterpret_cast<uint4*>(d1.k + slot * 128 + 16 * w) = kv;
+          *reinterpret_cast<uint4*>(d1.v + slot * 128 + 16 * w) = vv;
+        }
+      }
+    } else {
+      float x[8];
+      bf16x8_to_float(vv, x);
+      float mn = x[0], mx = x[0];
 #pragma unroll
-  for (int u = 0; u < 4; ++u) own += hb[u];
+      for (int j = 1; j < 8; ++j) { mn = fminf(mn, x[j]); mx = fmaxf(mx, x[j]); }
+#pragma unroll
+      for (int o = 1; o < 8; o <<= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      }
+      float s, inv, z;
+      quant_params(mn, mx, s, inv, z);
+      uint32_t c[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) c[j] = quant_code(x[j], inv, z);
+      const uint32_t word = pack8(c);
+      if (valid) {
+        *reinterpret_cast<uint32_t*>(d0.v + slot * 32 + 4 * w) = word;
+        if (w == 0) d0.vpar[slot] = make_float2(s, z);
+        if (two) {
+          *reinterpret_cast<uint32_t*>(d1.v + slot * 32 + 4 * w) = word;
+          if (w == 0) d1.vpar[slot] = make_float2(s, z);
+        }
+        __stcg(reinterpret_cast<uint4*>(a.kstage + ((size_t)h * a.max_n + tok) * 64 + 8 * w), kv);
+      }
+    }
+    if (valid && h == 0 && w == 0) {
+      const int32_t o = (a.frame << 16) | tok;
+      d0.origin[a.dst_slot + tok] = o;
+      if (two) d1.origin[a.dst_slot + tok] = o;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// POOL.  Pooled query, Eq. 2-3.  Block b takes pooled rows b, b + G, ...; thread
+// (c, hs) builds pooled[h][i][c] for heads h = hs, hs + 8, ... (sequential sum over
+// the group's tokens, divided by the group size); threads with hs == 0 add the
+// heads in order and scale by 1/H.  Loads are issued in batches ahead of the
+// (ordered) additions.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void phase_pool(const MaintArgs& a, Shared& sh) {
+  const int c = threadIdx.x & 63;
+  const int hslot = threadIdx.x >> 6;      // 0..7
+  for (int i = blockIdx.x; i < a.n_pooled; i += gridDim.x) {
+    int ta, tb;
+    if (i < a.n_special) { ta = i; tb = i + 1; }
+    else { ta = a.n_special + (i - a.n_special) * a.pool_g; tb = min(ta + a.pool_g, a.n); }
+    // heads h0 and h0 + 8 together: all loads of a batch (2 heads x 16 tokens) are issued before
+    // the first (ordered) addition; an index past the group is clamped, its value unused
+    for (int h0 = hslot; h0 < a.H; h0 += 16) {
+      const bool has1 = h0 + 8 < a.H;
+      const __nv_bfloat16* base0 = a.q + (int64_t)h0 * a.hs_q + c;
+      const __nv_bfloat16* base1 = a.q + (int64_t)(has1 ? h0 + 8 : h0) * a.hs_q + c;
+      float acc0 = 0.f, acc1 = 0.f;
+      for (int t0 = ta; t0 < tb; t0 += 16) {
+        float x0[16], x1[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+          const int64_t off = (int64_t)min(t0 + u, tb - 1) * a.ts_q;
+          x0[u] = __bfloat162float(base0[off]);
+          x1[u] = __bfloat162float(base1[off]);
+        }
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+          if (t0 + u < tb) {
+            acc0 = (t0 + u == ta) ? x0[u] : __fadd_rn(acc0, x0[u]);
+            acc1 = (t0 + u == ta) ? x1[u] : __fadd_rn(acc1, x1[u]);
+          }
+        }
+      }
+      if (i >= a.n_special) {
+        acc0 = __fdiv_rn(acc0, (float)(tb - ta));
+        acc1 = __fdiv_rn(acc1, (float)(tb - ta));
+      }
+      sh.u.pool.pooled[h0 * 64 + c] = acc0;
+      if (has1) sh.u.pool.pooled[(h0 + 8) * 64 + c] = acc1;
+    }
+    __syncthreads();
+    if (hslot == 0) {
+      float acc = 0.f;
+      for (int h0 = 0; h0 < a.H; h0 += 16) {
+        float v[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) v[u] = (h0 + u < a.H) ? sh.u.pool.pooled[(h0 + u) * 64 + c] : 0.f;
+#pragma unroll
+        for (int u = 0; u < 16; ++u)
+          if (h0 + u < a.H) acc = (h0 + u == 0) ? v[u] : __fadd_rn(acc, v[u]);
+      }
+      const float inv_h = __fdiv_rn(1.f, (float)a.H);
+      __stcg(&a.qbar[i * 64 + c], __fmul_rn(acc, inv_h));
+    }
+    __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------------------
+// KBAR.  Head means of the keys, Eq. 4, for the rest-local positions [lo, hi) of the
+// buffer set `b`: one pass per 64-slot key group (the rest segment starts on a
+// 128-slot boundary, so the tokens of a pass share their quantisation parameters).
+// Thread = (token, 8-channel word): dequantise the word of every head in order
+// (Eq. 10), accumulate the head sum sequentially, scale by 1/H.  The words of
+// sixteen heads (4-bit; four 16-byte pieces for 16-bit storage) are fetched ahead
+// of their (ordered) use.
+// ---------------------------------------------------------------------------
+template <int BITS>
+__device__ __forceinline__ void phase_kbar(const MaintArgs& a, Shared& sh, const BufSet& b, int lo, int hi) {
+  const int tid = threadIdx.x;
+  const int w = tid & 7;
+  const int tok = tid >> 3;
+  const int g_lo = lo >> 6, g_hi = (hi + 63) >> 6;
+  const int H = a.H, cap = a.cap;
+  for (int gb = g_lo + blockIdx.x; gb < g_hi; gb += gridDim.x) {
+    const int i = gb * 64 + tok;                  // rest-local index
+    const int slot = a.rest_base + i;
+    const int grp = (a.rest_base >> 6) + gb;
+    bool plain = false;
+    if (BITS == 4) {
+      // Parameters of the key group.  Fast path: float4 [H][4][8] = (s, magic + z) of channels
+      // 8w + 2v and 8w + 2v + 1 at [h][v][w], so that the eight lanes of a quarter-warp read
+      // consecutive 16-byte chunks.  Plain path: float2 (s, z) [H][64].
+      int big = a.force_plain;
+      for (int e = tid; e < H * 64; e += kMT) {
+        const float2 sz = __ldcg(&b.kpar[((size_t)(e >> 6) * (cap >> 6) + grp) * 64 + (e & 63)]);
+        big |= !(fabsf(sz.y) < kZLimit);
+      }
+      plain = __syncthreads_or(big) != 0;
+      for (int e = tid; e < H * 64; e += kMT) {
+        float2 sz = __ldcg(&b.kpar[((size_t)(e >> 6) * (cap >> 6) + grp) * 64 + (e & 63)]);
+        if (plain) {
+          sh.u.kbar.par[e] = sz;
+        } else {
+          const int h = e >> 6, ch = e & 63;
+          sz.y = __fadd_rn(magic_val(ch & 7), sz.y);
+          sh.u.kbar.par[((h * 4 + ((ch & 7) >> 1)) * 8 + (ch >> 3)) * 2 + (ch & 1)] = sz;
+        }
+      }
+      __syncthreads();
+    }
+    const bool valid = i >= lo && i < hi;
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    constexpr int kHB = (BITS == 4) ? 16 : 4;     // heads whose words are in flight together
+    for (int h0 = 0; h0 < H; h0 += kHB) {
+      uint32_t word[BITS == 4 ? kHB : 1];
+      uint4 wide[BITS == 4 ? 1 : kHB];
+#pragma unroll
+      for (int u = 0; u < kHB; ++u) {
+        const int h = h0 + u;
+        if (BITS == 4) word[u] = 0u; else wide[u] = make_uint4(0, 0, 0, 0);
+        if (valid && h < H) {
+          if (BITS == 4) word[u] = __ldcg(reinterpret_cast<const uint32_t*>(b.k + ((size_t)h * cap + slot) * 32 + 4 * w));
+          else wide[u] = __ldcg(reinterpret_cast<const uint4*>(b.k + ((size_t)h * cap + slot) * 128 + 16 * w));
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kHB; ++u) {
+        const int h = h0 + u;
+        if (h < H) {
+          float x[8];
+          if (BITS == 4) {
+            if (plain) {
+              dequant8_plain(word[BITS == 4 ? u : 0], sh.u.kbar.par + h * 64 + 8 * w, x);
+            } else {
+              float2 par[8];
+              const float4* pp = reinterpret_cast<const float4*>(sh.u.kbar.par) + h * 32 + w;
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                const float4 t = pp[v * 8];
+                par[2 * v] = make_float2(t.x, t.y);
+                par[2 * v + 1] = make_float2(t.z, t.w);
+              }
+              dequant8_magic(word[BITS == 4 ? u : 0], par, x);
+            }
+          } else {
+            bf16x8_to_float(wide[BITS == 4 ? 0 : u], x);
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[j] = (h == 0) ? x[j] : __fadd_rn(acc[j], x[j]);
+        }
+      }
+    }
+    const float inv_h = __fdiv_rn(1.f, (float)H);
+    if (valid) {
+      float4* dst = reinterpret_cast<float4*>(b.kbar + (size_t)i * 64 + 8 * w);
+      __stcg(dst, make_float4(__fmul_rn(acc[0], inv_h), __fmul_rn(acc[1], inv_h), __fmul_rn(acc[2], inv_h),
+                              __fmul_rn(acc[3], inv_h)));
+      __stcg(dst + 1, make_float4(__fmul_rn(acc[4], inv_h), __fmul_rn(acc[5], inv_h), __fmul_rn(acc[6], inv_h),
+                                  __fmul_rn(acc[7], inv_h)));
+    }
+    __syncthreads();       // the parameter table is rewritten by the next pass
+  }
+}
+
+// ---------------------------------------------------------------------------
+// SCORE.  w[c] = (sequential sum of the pooled rows) / N_pooled; S[j] = balanced
+// tree over the 64 products w[c] * K-bar[j][c] (three levels inside the lane, three
+// by xor-shuffle), Eq. 5-6.  Thread = (token, 8-channel word); block b takes the
+// 64-token runs b, b + G, ...
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void phase_score(const MaintArgs& a, Shared& sh) {
+  const int tid = threadIdx.x;
+  const int n_runs = (a.r_old + 63) >> 6;
+  if ((int)blockIdx.x >= n_runs && blockIdx.x != 0) return;
+  // the pooled rows come through shared memory, 128 at a time (one round trip), and one thread
+  // per channel adds them in order
+  for (int r0 = 0; r0 < a.n_pooled; r0 += kPoolRows) {
+    const int rows = min(kPoolRows, a.n_pooled - r0);
+    __syncthreads();
+    for (int e = tid; e < rows * 64; e += kMT) sh.u.score.rows[e] = __ldcg(&a.qbar[r0 * 64 + e]);
+    __syncthreads();
+    if (tid < 64) {
+      float acc = (r0 == 0) ? 0.f : sh.u.score.w[tid];
+      for (int q0 = 0; q0 < rows; q0 += 16) {
+        float v[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) v[u] = (q0 + u < rows) ? sh.u.score.rows[(q0 + u) * 64 + tid] : 0.f;
+#pragma unroll
+        for (int u = 0; u < 16; ++u)
+          if (q0 + u < rows) acc = (r0 == 0 && q0 + u == 0) ? v[u] : __fadd_rn(acc, v[u]);
+      }
+      sh.u.score.w[tid] = acc;
+    }
+  }
+  if (tid < 64) {
+    const float wv = __fdiv_rn(sh.u.score.w[tid], (float)a.n_pooled);
+    sh.u.score.w[tid] = wv;
+    if (blockIdx.x == 0) a.qvec[tid] = wv;
+  }
+  __syncthreads();
+  const int w = tid & 7, tok = tid >> 3;
+  float wq[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) wq[j] = sh.u.score.w[8 * w + j];
+  for (int run = blockIdx.x; run < n_runs; run += gridDim.x) {
+    const int i = run * 64 + tok;
+    const bool valid = i < a.r_old;
+    const float4* src = reinterpret_cast<const float4*>(a.cur.kbar + (size_t)(valid ? i : 0) * 64 + 8 * w);
+    const float4 x = __ldcg(src), y = __ldcg(src + 1);
+    const float kb[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
+    float p[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) p[j] = __fmul_rn(kb[j], wq[j]);
+    float t0 = __fadd_rn(p[0], p[1]), t1 = __fadd_rn(p[2], p[3]);
+    float t2 = __fadd_rn(p[4], p[5]), t3 = __fadd_rn(p[6], p[7]);
+    t0 = __fadd_rn(t0, t1);
+    t2 = __fadd_rn(t2, t3);
+    float s = __fadd_rn(t0, t2);
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) s = __fadd_rn(s, __shfl_xor_sync(0xffffffffu, s, o));
+    if (valid && w == 0) {
+      __stcg(&a.scores[i], s);
+      atomicAdd(&a.hist[(blockIdx.x & (kHistCopies - 1)) * kSelBins + (order_key(s) >> 20)], 1u);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// SEL1 / SEL2.  Top-k of the scores (Sec. 3.2), ties to the lower position, i.e.
+// the k largest of the unique pairs (key, -position).  Every block that owns tokens
+// repeats the global parts (histogram scan, bisection) for itself.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long composite(uint32_t key, int pos) {
+  return ((unsigned long long)key << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)pos);
+}
+
+__device__ __forceinline__ void phase_sel1(const MaintArgs& a, Shared& sh) {
+  const int tid = threadIdx.x;
+  const int n_runs = (a.r_old + 63) >> 6;
+  if (blockIdx.x == gridDim.x - 1) {                 // the next selecting launch's counter and sub-histogram:
+    if (tid == 0) *a.cand_count_next = 0u;           // nobody uses them in this launch
+    if (tid < kSubBins) a.hist2_next[tid] = 0u;
+  }
+  if ((int)blockIdx.x >= n_runs) return;
+  // thread t owns the bins 4095 - 8t - 7 .. 4095 - 8t; walked from the top
+  unsigned int hb[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+  {
+    uint4 lo4[kHistCopies], hi4[kHistCopies];
+#pragma unroll
+    for (int cpy = 0; cpy < kHistCopies; ++cpy) {
+      const uint4* hp = reinterpret_cast<const uint4*>(a.hist + cpy * kSelBins + kSelBins - 8 - 8 * tid);
+      lo4[cpy] = __ldcg(hp);
+      hi4[cpy] = __ldcg(hp + 1);
+    }
+#pragma unroll
+    for (int cpy = 0; cpy < kHistCopies; ++cpy) {
+      hb[0] += hi4[cpy].w; hb[1] += hi4[cpy].z; hb[2] += hi4[cpy].y; hb[3] += hi4[cpy].x;
+      hb[4] += lo4[cpy].w; hb[5] += lo4[cpy].z; hb[6] += lo4[cpy].y; hb[7] += lo4[cpy].x;
+    }
+  }
+  unsigned int own = 0u;
+#pragma unroll
+  for (int u = 0; u < 8; ++u) own += hb[u];
   unsigned int total;
-  unsigned int above = block_excl_scan(own, s_warp, total);   // keys in higher bins than this thread's
+  unsigned int above = block_excl_scan(own, sh.warp, total);   // keys in higher bins than this thread's
 #pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    if (above < (unsigned int)k && (unsigned int)k <= above + hb[u]) {
-      s_bin = (unsigned int)(kSelBins - 1 - (4 * tid + u));
-      s_need = (unsigned int)k - above;
+  for (int u = 0; u < 8; ++u) {
+    if (above < (unsigned int)a.kk && (unsigned int)a.kk <= above + hb[u]) {
+      sh.bin = (unsigned int)(kSelBins - 1 - (8 * tid + u));
+      sh.need = (unsigned int)a.kk - above;                       // the k-th largest is the need-th largest of its bin
     }
     above += hb[u];
   }
   __syncthreads();
-  const uint32_t bin = s_bin;
-  const unsigned int need = s_need;                  // tau is the need-th largest key of its bin
-
-  // ---- stage 2: collect the keys of that bin (each thread scans its run; a block scan places them) ----
-  const int ipt = ((tp + kSelThreads - 1) / kSelThreads) | 1;   // odd run length: a warp's runs on different banks
-  const int j0 = min(tid * ipt, tp), j1 = min(j0 + ipt, tp);
-  constexpr int kR = KPT > 0 ? KPT : 1;
-  uint32_t kr[kR];                                   // this thread's run (KPT > 0)
-  if (KPT > 0) {
-#pragma unroll
-    for (int i = 0; i < kR; ++i) kr[i] = (j0 + i < j1) ? key_at(j0 + i) : 0u;
-  }
-  // key i of the run: from registers when the loop over i is unrolled, else from memory
-#define XKV_RUN_LOOP(BODY)                                                              \
-  if (KPT > 0) {                                                                        \
-    _Pragma("unroll") for (int i = 0; i < kR; ++i) if (j0 + i < j1) { const int j = j0 + i; const uint32_t key = kr[i]; BODY } \
-  } else {                                                                              \
-    for (int j = j0; j < j1; ++j) { const uint32_t key = key_at(j); BODY }              \
-  }
-  unsigned int mine_n = 0u;
-  XKV_RUN_LOOP({ (void)j; mine_n += ((key >> 20) == bin); })
-  unsigned int ncand;
-  unsigned int at = block_excl_scan(mine_n, s_warp, ncand);
-  if (mine_n) {
-    XKV_RUN_LOOP({ (void)j; if ((key >> 20) == bin) { if (at < (unsigned int)kSelCand) s_cand[at] = key; ++at; } })
-  }
-  __syncthreads();
-
-  // ---- stage 3: the low 20 bits of tau by bisection on the candidates ----
-  uint32_t prefix = bin << 20;
-  unsigned int n_gt;                                 // candidates above tau
-  if (ncand <= (unsigned int)kSelThreads) {
-    const bool has = (unsigned int)tid < ncand;
-    const uint32_t mine = has ? s_cand[tid] : 0u;
-    for (int bit = 19; bit >= 0; --bit) {
-      const uint32_t trial = prefix | (1u << bit);
-      if ((unsigned int)__syncthreads_count(has && mine >= trial) >= need) prefix = trial;
-    }
-    n_gt = (unsigned int)__syncthreads_count(has && mine > prefix);
-  } else {
-    // rare (many equal or nearly equal scores): the same bisection over a list that does not fit
-    // one candidate per thread, or over all keys of the bin when it overflowed the list
-    const bool listed = ncand <= (unsigned int)kSelCand;
-    auto count = [&](uint32_t trial, bool strict) -> unsigned int {
-      unsigned int c = 0u;
-      if (listed) {
-        for (unsigned int i = tid; i < ncand; i += kSelThreads) c += strict ? (s_cand[i] > trial) : (s_cand[i] >= trial);
-      } else {
-        XKV_RUN_LOOP({ (void)j; if ((key >> 20) == bin) c += strict ? (key > trial) : (key >= trial); })
+  const uint32_t bin = sh.bin;
+  for (int run = blockIdx.x; run < n_runs; run += gridDim.x) {
+    const int i = run * 64 + tid;
+    bool hi = false;
+    if (tid < 64 && i < a.r_old) {
+      const uint32_t key = order_key(__ldcg(&a.scores[i]));
+      hi = (key >> 20) > bin;
+      if ((key >> 20) == bin) {
+        const unsigned int at = atomicAdd(a.cand_count, 1u);
+        __stcg(&a.cand[at], composite(key, i));
+        atomicAdd(&a.hist2[(key >> 12) & (kSubBins - 1)], 1u);
       }
-      return block_sum(c, &s_acc);
-    };
-    for (int bit = 19; bit >= 0; --bit) {
-      const uint32_t trial = prefix | (1u << bit);
-      if (count(trial, false) >= need) prefix = trial;
     }
-    n_gt = count(prefix, true);
+    const int cnt = __syncthreads_count(hi);
+    if (tid == 0) __stcg(&a.run_hi[run], (unsigned int)cnt);
   }
-  const uint32_t tau = prefix;
-  const unsigned int need_eq = need - n_gt;          // keys equal to tau that are kept (lowest positions)
-
-  // ---- stage 4: stable compaction ----
-  unsigned int cnt_eq = 0u, cnt_gt = 0u;
-  XKV_RUN_LOOP({ (void)j; cnt_eq += (key == tau); cnt_gt += (key > tau); })
-  const unsigned int eq_before = block_excl_scan(cnt_eq, s_warp, total);
-  unsigned int take_eq = 0u;
-  if (eq_before < need_eq) take_eq = min(cnt_eq, need_eq - eq_before);
-  unsigned int out = block_excl_scan(cnt_gt + take_eq, s_warp, total);
-  // The kept positions are listed in shared memory first (in the key array: a thread's keep flags
-  // are taken before anything is overwritten) and copied out in full lines; written from the
-  // runs directly, every store of a warp would touch 32 different sectors.
-  unsigned int flags = 0u;                           // runs longer than 32 keys take the direct route
-  const bool staged = IN_SMEM && ipt <= 32;
-  if (staged) {
-    XKV_RUN_LOOP({
-      bool keep = key > tau;
-      if (key == tau && take_eq > 0u) { keep = true; --take_eq; }
-      flags |= (keep ? 1u : 0u) << (j - j0);
-    })
-    __syncthreads();
-    int32_t* s_out = reinterpret_cast<int32_t*>(s_keys);
-    if (KPT > 0) {
-#pragma unroll
-      for (int i = 0; i < kR; ++i)
-        if ((flags >> i) & 1u) s_out[out++] = j0 + i;
-    } else {
-      for (int j = j0; j < j1; ++j)
-        if ((flags >> (j - j0)) & 1u) s_out[out++] = j;
-    }
-    __syncthreads();
-    for (int i = tid; i < k; i += kSelThreads) kept[i] = s_out[i];
-  } else {
-    XKV_RUN_LOOP({
-      bool keep = key > tau;
-      if (key == tau && take_eq > 0u) { keep = true; --take_eq; }
-      if (keep) kept[out++] = j;
-    })
-  }
-#undef XKV_RUN_LOOP
 }
 
-cudaError_t launch_select(xkv_cache* c, int r_old, int k, cudaStream_t st) {
+__device__ __forceinline__ void phase_sel2(const MaintArgs& a, Shared& sh) {
+  const int tid = threadIdx.x;
+  const int n_runs = (a.r_old + 63) >> 6;
+  if (blockIdx.x == gridDim.x - 1) {                 // every block has read the histogram: ready for the next step
+    for (int e = tid; e < kSelBins * kHistCopies; e += kMT) a.hist[e] = 0u;
+  }
+  if ((int)blockIdx.x >= n_runs) return;
+  const uint32_t bin = sh.bin;
+  const unsigned int need = sh.need;
+  const unsigned int ncand = __ldcg(a.cand_count);
+  const bool in_smem = ncand <= (unsigned int)kCandSmem;
+  if (in_smem)
+    for (unsigned int e = tid; e < ncand; e += kMT) sh.u.sel.cand[e] = __ldcg(&a.cand[e]);
+  __syncthreads();
+  auto cand_at = [&](unsigned int e) -> unsigned long long { return in_smem ? sh.u.sel.cand[e] : __ldcg(&a.cand[e]); };
+  // the need-th largest candidate: its bin bits are known, the positions lie below 2^pbits
+  int pbits = 1;
+  while ((1 << pbits) < a.r_old) ++pbits;
+  unsigned long long prefix = ((unsigned long long)bin << 52) | (unsigned long long)(0xFFFFFFFFu << pbits);
+  // The candidates share the top 12 key bits; a second histogram over their next 8 bits (filled by
+  // SEL1) narrows the k-th largest key down to one sub-bin, whose few members are listed and ranked.
   {
-    // opt-in to large dynamic shared memory: a per-device function attribute, set once per device
-    static std::mutex mu;
-    static bool attr_set[64] = {false};
-    int dev = -1;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    std::lock_guard<std::mutex> lock(mu);
-    if (!attr_set[dev]) {
-      e = cudaFuncSetAttribute(select_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               kSelSmemKeys * (int)sizeof(uint32_t));
-      if (e != cudaSuccess) return e;
-      e = cudaFuncSetAttribute(select_kernel<true, 17>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               kSelSmemKeys * (int)sizeof(uint32_t));
-      if (e != cudaSuccess) return e;
-      attr_set[dev] = true;
+    const unsigned int h2 = (tid < kSubBins) ? __ldcg(&a.hist2[kSubBins - 1 - tid]) : 0u;   // thread t: sub-bin 255 - t
+    unsigned int total;
+    const unsigned int above2 = block_excl_scan(h2, sh.warp, total);
+    if (tid == 0) sh.n_list = 0u;
+    if (tid < kSubBins && above2 < need && need <= above2 + h2) { sh.sub = kSubBins - 1 - tid; sh.need2 = need - above2; }
+    __syncthreads();
+  }
+  const uint32_t sub = sh.sub;
+  const unsigned int need2 = sh.need2;
+  if (in_smem) {
+    for (unsigned int e = tid; e < ncand; e += kMT) {
+      const unsigned long long cv = sh.u.sel.cand[e];
+      if ((((uint32_t)(cv >> 32) >> 12) & (kSubBins - 1)) == sub) {
+        const unsigned int at = atomicAdd(&sh.n_list, 1u);
+        if (at < (unsigned int)kSubList) sh.u.sel.list[at] = cv;
+      }
     }
   }
-  LaunchScope ls(c, XKV_PROF_SELECT, st);
-  const size_t smem = (size_t)r_old * sizeof(uint32_t);
-  const int ipt = ((r_old + kSelThreads - 1) / kSelThreads) | 1;
-  if (r_old > kSelSmemKeys)
-    select_kernel<false, 0><<<1, kSelThreads, 0, st>>>(c->scores, r_old, k, c->kept, c->sel_hist);
-  else if (ipt <= 17)
-    select_kernel<true, 17><<<1, kSelThreads, smem, st>>>(c->scores, r_old, k, c->kept, c->sel_hist);
-  else
-    select_kernel<true, 0><<<1, kSelThreads, smem, st>>>(c->scores, r_old, k, c->kept, c->sel_hist);
-  return cudaGetLastError();
+  __syncthreads();
+  const unsigned int m = sh.n_list;
+  if (in_smem && m <= 32u) {
+    // every warp ranks the listed candidates by itself: lane l holds candidate l and counts the
+    // larger ones; the one with need2 - 1 larger ones is the k-th largest of all
+    const int lane = tid & 31;
+    const unsigned long long mine = (unsigned int)lane < m ? sh.u.sel.list[lane] : 0ull;
+    unsigned int larger = 0u;
+    for (unsigned int j = 0; j < m; ++j) larger += __shfl_sync(0xffffffffu, mine, (int)j) > mine;
+    const unsigned int hit = __ballot_sync(0xffffffffu, (unsigned int)lane < m && larger == need2 - 1u);
+    prefix = __shfl_sync(0xffffffffu, mine, __ffs(hit) - 1);
+  } else {
+    // many candidates (many equal or nearly equal scores): the same bisection over the whole
+    // 64-bit pair, block-wide, on the list in shared memory or, if it does not fit, in global memory
+    for (int bit = 51; bit >= 0; --bit) {
+      if (bit < 32 && bit >= pbits) continue;
+      const unsigned long long trial = prefix | (1ull << bit);
+      unsigned int c = 0u;
+      for (unsigned int e = tid; e < ncand; e += kMT) c += cand_at(e) >= trial;
+      if (block_sum(c, &sh.acc) >= need) prefix = trial;
+    }
+  }
+  const unsigned long long tau = prefix;             // kept candidates: composite >= tau (exactly `need` of them)
+  for (int run = blockIdx.x; run < n_runs; run += gridDim.x) {
+    // survivors before this run: the sure keeps of the runs before it plus the kept candidates at
+    // lower positions
+    unsigned int part = 0u;
+    for (int r = tid; r < run; r += kMT) part += __ldcg(&a.run_hi[r]);
+    const uint32_t below = 0xFFFFFFFFu - (uint32_t)(run * 64);         // position part of position run * 64
+    for (unsigned int e = tid; e < ncand; e += kMT) {
+      const unsigned long long cv = cand_at(e);
+      part += (cv >= tau) && ((uint32_t)cv > below);                   // larger low word = lower position
+    }
+    const unsigned int base = block_sum(part, &sh.acc);
+    const int i = run * 64 + tid;
+    bool keep = false;
+    if (tid < 64 && i < a.r_old) {
+      const uint32_t key = order_key(__ldcg(&a.scores[i]));
+      keep = (key >> 20) > bin || ((key >> 20) == bin && composite(key, i) >= tau);
+    }
+    if (tid < 64) {
+      const unsigned int m = __ballot_sync(0xffffffffu, keep);
+      if (tid == 31) sh.warp[0] = __popc(m);
+      const unsigned int rank = __popc(m & ((1u << (tid & 31)) - 1u));
+      asm volatile("bar.sync 2, 64;" ::: "memory");
+      const unsigned int off = (tid >= 32) ? sh.warp[0] : 0u;
+      if (keep) __stcg(&a.kept[base + off + rank], i);
+    }
+    __syncthreads();
+  }
 }
 
 // ---------------------------------------------------------------------------
-// kv_quant_pack, 4-bit.  One CTA per (new 64-slot key group, four heads); 128
-// threads per head, thread = (8-channel word, four tokens 16 apart).
+// kv_quant_pack, 4-bit: a kernel of its own (one thread block per item, placed by the
+// hardware scheduler; the arithmetic needs more registers than the phases above).
+// Item = (new 64-slot key group, four heads); 128 threads per head, thread =
+// (8-channel word, four tokens 16 apart).
 // Keys: survivors are dequantised with the parameters of the group they came
 // from (Eq. 10), new keys come from the bf16 staging buffer; per-channel min/max
 // over the group's tokens; new parameters and codes (Eq. 7-8).  A complete group
@@ -897,51 +872,136 @@ regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int H, int cap, 
 }
 
 // ---------------------------------------------------------------------------
-// Survivor gather: rows of value codes (and of bf16 keys/values in 16-bit mode),
-// value parameters and origins move from the current buffer set to the other,
-// preserving order.  Thread = (head, survivor, 16-byte chunk).
+// PACK, 16-bit: rows of keys and values and the origins move from the current
+// buffer set to the other, preserving order.  Thread-item = (head, survivor,
+// 16-byte chunk).
 // ---------------------------------------------------------------------------
-template <int BITS>
-__global__ void __launch_bounds__(256)
-gather_kernel(BufSet src, BufSet dst, int H, int cap, int base_slot, int kk, const int32_t* __restrict__ kept) {
-  constexpr int kChunks = (BITS == 4) ? 2 : 8;
-  constexpr int kRow = (BITS == 4) ? 32 : 128;
-  const long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const int ch = (int)(g % kChunks);
-  const long long r = g / kChunks;
-  if (r >= (long long)H * kk) return;
-  const int i = (int)(r % kk);
-  const int h = (int)(r / kk);
-  const int old = kept ? kept[i] : i;
-  const size_t s = (size_t)h * cap + base_slot + old;
-  const size_t d = (size_t)h * cap + base_slot + i;
-  *reinterpret_cast<uint4*>(dst.v + d * kRow + 16 * ch) = *reinterpret_cast<const uint4*>(src.v + s * kRow + 16 * ch);
-  if (BITS == 16)
-    *reinterpret_cast<uint4*>(dst.k + d * kRow + 16 * ch) = *reinterpret_cast<const uint4*>(src.k + s * kRow + 16 * ch);
-  if (BITS == 4 && ch == 0) dst.vpar[d] = src.vpar[s];
-  if (h == 0 && ch == 0) dst.origin[base_slot + i] = src.origin[base_slot + old];
+__device__ __forceinline__ void phase_gather16(const MaintArgs& a) {
+  const BufSet& src = a.cur;
+  const BufSet& dst = a.oth;
+  const int32_t* kept = a.identity ? nullptr : a.kept;
+  const long long items = (long long)a.H * a.kk * 8;
+  for (long long g = (long long)blockIdx.x * kMT + threadIdx.x; g < items; g += (long long)gridDim.x * kMT) {
+    const int ch = (int)(g & 7);
+    const long long r = g >> 3;
+    const int i = (int)(r % a.kk);
+    const int h = (int)(r / a.kk);
+    const int old = kept ? __ldcg(&kept[i]) : i;
+    const size_t s = (size_t)h * a.cap + a.rest_base + old;
+    const size_t d = (size_t)h * a.cap + a.rest_base + i;
+    *reinterpret_cast<uint4*>(dst.v + d * 128 + 16 * ch) = *reinterpret_cast<const uint4*>(src.v + s * 128 + 16 * ch);
+    *reinterpret_cast<uint4*>(dst.k + d * 128 + 16 * ch) = *reinterpret_cast<const uint4*>(src.k + s * 128 + 16 * ch);
+    if (h == 0 && ch == 0) dst.origin[a.rest_base + i] = src.origin[a.rest_base + old];
+  }
 }
 
-cudaError_t launch_pack(xkv_cache* c, int n, int kk, bool identity, bool first, cudaStream_t st) {
-  const BufSet src = c->buf[c->cur];
-  const BufSet dst = c->buf[c->cur ^ 1];
-  const int32_t* kept = identity ? nullptr : c->kept;
-  const int H = c->p.n_heads;
-  if (c->p.kv_bits == 4) {
-    // one kernel: key regroup + survivor gather of values, value parameters and origins
-    const int base = first ? 0 : c->rest_base;
-    const int r_new = kk + n;
-    const dim3 grid((r_new + 63) / 64, (H + kRgHeads - 1) / kRgHeads);
-    LaunchScope ls(c, XKV_PROF_REGROUP, st);
-    regroup_k_kernel<<<grid, 128 * kRgHeads, 0, st>>>(src, dst, src, first, H, c->cap, c->p.max_frame_tokens, base,
-                                                     kk, r_new, kept, c->kstage, c->force_plain);
-    return cudaGetLastError();
+}  // namespace
+
+// ---------------------------------------------------------------------------
+// The kernel.
+// ---------------------------------------------------------------------------
+template <int BITS>
+__global__ void __launch_bounds__(kMT, kBlocksPerSM) maint_kernel(const __grid_constant__ MaintArgs a) {
+  __shared__ Shared sh;
+  if (threadIdx.x == 0) { sh.abort_flag = 0; sh.acc = 0u; sh.bin = 0u; sh.need = 0u; }
+  __syncthreads();
+  uint32_t epoch = 0;
+  const uint32_t ph = a.phases;
+  bool ran = false;                 // something has run since the last barrier
+
+  if (ph & kPhAppend) { phase_append<BITS>(a); ran = true; }
+  if (ph & kPhPool) { phase_pool(a, sh); ran = true; }
+  if (ph & kPhKbar) { phase_kbar<BITS>(a, sh, a.kbar_on_other ? a.oth : a.cur, a.kbar_lo, a.kbar_hi); ran = true; }
+
+  if (ph & kPhScore) {
+    if (ran && !grid_barrier(a, epoch, sh)) return;
+    phase_score(a, sh);
+    ran = true;
   }
-  if (kk > 0) {
-    LaunchScope ls(c, XKV_PROF_GATHER, st);
-    const long long threads = (long long)H * kk * 8;
-    gather_kernel<16><<<(int)((threads + 255) / 256), 256, 0, st>>>(src, dst, H, c->cap, c->rest_base, kk, kept);
+  if (ph & kPhSel) {
+    if (ran && !grid_barrier(a, epoch, sh)) return;
+    phase_sel1(a, sh);
+    if (!grid_barrier(a, epoch, sh)) return;
+    phase_sel2(a, sh);
+    ran = true;
   }
+  if (ph & kPhPack) {
+    if (ran && !grid_barrier(a, epoch, sh)) return;
+    if (BITS == 16 && a.kk > 0) phase_gather16(a);
+  }
+}
+
+// Grid barriers that a launch with these phases goes through (the same decisions as in the kernel).
+static int maint_barriers(uint32_t ph) {
+  int nb = 0;
+  bool ran = (ph & (kPhAppend | kPhPool | kPhKbar)) != 0;
+  if (ph & kPhScore) { nb += ran ? 1 : 0; ran = true; }
+  if (ph & kPhSel) { nb += (ran ? 1 : 0) + 1; ran = true; }
+  if (ph & kPhPack) nb += ran ? 1 : 0;
+  return nb;
+}
+
+// Per device, on first use with that device current: how many blocks of the kernel can be
+// resident at once (a cooperative launch needs the whole grid resident).
+static std::mutex g_maint_mutex;
+static int g_maint_grid[64] = {0};
+
+static cudaError_t maint_grid(int* grid) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_maint_mutex);
+  if (g_maint_grid[dev] == 0) {
+    int sms = 0, per_sm = kBlocksPerSM;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const void* fns[2] = {(const void*)maint_kernel<4>, (const void*)maint_kernel<16>};
+    for (const void* fn : fns) {
+      int nb = 0;
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, kMT, 0);
+      if (e != cudaSuccess) return e;
+      if (nb < per_sm) per_sm = nb;
+    }
+    if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+    g_maint_grid[dev] = sms * per_sm;
+  }
+  *grid = g_maint_grid[dev];
+  return cudaSuccess;
+}
+
+cudaError_t launch_regroup(xkv_cache* c, const MaintArgs& a, cudaStream_t st) {
+  const dim3 grid((a.r_new + 63) / 64, (a.H + kRgHeads - 1) / kRgHeads);
+  LaunchScope ls(c, XKV_PROF_PACK, st);
+  regroup_k_kernel<<<grid, 128 * kRgHeads, 0, st>>>(a.cur, a.oth, a.cur, a.first != 0, a.H, a.cap, a.max_n,
+                                                   a.first ? 0 : a.rest_base, a.kk, a.r_new,
+                                                   a.identity ? nullptr : a.kept, a.kstage, a.force_plain);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_maint(xkv_cache* c, MaintArgs& a, int prof_cat, cudaStream_t st) {
+  int grid = 0;
+  cudaError_t e = maint_grid(&grid);
+  if (e != cudaSuccess) return e;
+  const int nb = maint_barriers(a.phases);
+  a.bar = c->counters;
+  a.bar_base = c->bar_base;
+  a.status = c->status;
+  a.cand_count = c->counters + 2 + c->sel_parity;
+  a.cand_count_next = c->counters + 2 + (c->sel_parity ^ 1);
+  a.hist2 = c->counters + 64 + 256 * c->sel_parity;
+  a.hist2_next = c->counters + 64 + 256 * (c->sel_parity ^ 1);
+  if (a.phases & kPhSel) c->sel_parity ^= 1;
+  LaunchScope ls(c, prof_cat, st);
+  void* params[1] = {(void*)&a};
+  const void* fn = (c->p.kv_bits == 16) ? (const void*)maint_kernel<16> : (const void*)maint_kernel<4>;
+  if (nb > 0) {
+    e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kMT), params, 0, st);
+    c->bar_base += (uint32_t)nb * (uint32_t)grid;
+  } else {
+    e = cudaLaunchKernel(fn, dim3(grid), dim3(kMT), params, 0, st);
+  }
+  if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }
 

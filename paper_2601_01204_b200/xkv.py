@@ -36,8 +36,9 @@ EXPORTED = [
     "xkv_synth_fill", "xkv_profile_enable", "xkv_profile_read", "attn_packed_causal_static",
     "xkv_debug_rewind_attention", "attn_packed_causal_tail", "xkv_set_unquantised_tail",
     "xkv_debug_force_plain", "xkv_debug_limit_attention_blocks", "xkv_debug_timeout_probe",
+    "xkv_debug_head_means",
 ]
-PROF_NAMES = ["append", "pool_q", "score", "select", "regroup_k", "gather", "attn", "attn_combine", "kbar"]
+PROF_NAMES = ["append", "score_evict", "pack", "kbar", "maint", "attn", "attn_combine"]
 
 
 class xkv_params(C.Structure):
@@ -52,7 +53,7 @@ class xkv_info(C.Structure):
 
 
 class xkv_profile(C.Structure):
-    _fields_ = [("ms", C.c_double * 9), ("launches", C.c_int64 * 9)]
+    _fields_ = [("ms", C.c_double * 7), ("launches", C.c_int64 * 7)]
 
 
 _vp, _i32, _i64, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
@@ -100,6 +101,8 @@ lib.xkv_debug_force_plain.restype = C.c_int
 lib.xkv_debug_force_plain.argtypes = [_vp, _i32]
 lib.xkv_debug_limit_attention_blocks.restype = C.c_int
 lib.xkv_debug_limit_attention_blocks.argtypes = [_vp, _i32]
+lib.xkv_debug_head_means.restype = C.c_int
+lib.xkv_debug_head_means.argtypes = [_vp, _vp]
 lib.xkv_debug_timeout_probe.restype = C.c_int
 lib.xkv_debug_timeout_probe.argtypes = [_vp, _vp]
 lib.xkv_poll_status.restype = C.c_int
@@ -267,6 +270,9 @@ class Cache:
 
     def xkv_debug_limit_attention_blocks(self, max_blocks: int) -> None:
         _check(lib.xkv_debug_limit_attention_blocks(self.handle, max_blocks), "xkv_debug_limit_attention_blocks")
+
+    def xkv_debug_head_means(self) -> None:
+        _check(lib.xkv_debug_head_means(self.handle, _stream()), "xkv_debug_head_means")
 
     def xkv_debug_timeout_probe(self) -> None:
         _check(lib.xkv_debug_timeout_probe(self.handle, _stream()), "xkv_debug_timeout_probe")

@@ -197,14 +197,19 @@ def run_xkv(args) -> None:
     if args.layers > 0:
         w["layers"] = args.layers
         w["name"] += f"_reduced_to_{args.layers}_layers"
+    w["key_mode"] = 1 if args.keys == "once" else 0
+    if args.keys == "once":
+        w["name"] += "_keys_once"
     if args.budget > 0 or args.bits > 0 or args.tokens > 0:      # the ablation sweep and the long-stream shape
         w["budget"] = args.budget or w["budget"]
         w["kv_bits"] = args.bits or w["kv_bits"]
         w["n_tokens"] = args.tokens or w["n_tokens"]
         w["name"] = f"stack_{w['layers']}L_{w['n_tokens']}tok_budget{w['budget']}_{'int4' if w['kv_bits'] == 4 else 'bf16'}"
+        if args.keys == "once":
+            w["name"] += "_keys_once"
     L, H, d, n = w["layers"], w["n_heads"], w["head_dim"], w["n_tokens"]
     p = xkv.Params(n_heads=H, head_dim=d, n_special=w["n_special"], pool_g=w["pool_g"], quant_group=w["quant_group"],
-                   kv_bits=w["kv_bits"], budget=w["budget"], max_frame_tokens=n)
+                   kv_bits=w["kv_bits"], budget=w["budget"], max_frame_tokens=n, key_mode=w["key_mode"])
     caches = [xkv.Cache(p, device=f"cuda:{local}") for _ in range(L)]
     if args.tail:
         for c in caches:
@@ -319,7 +324,7 @@ def run_xkv(args) -> None:
         # the stream step is not a duration and is left out of the shares
         overlapped = ("kbar",)
         prof_total = sum(v[0] for k_, v in prof.items() if k_ not in overlapped)
-        nbytes = maintenance_bytes(H, n, d, w["budget"], w["kv_bits"])
+        nbytes = maintenance_bytes(H, n, d, w["budget"], w["kv_bits"], w["key_mode"])
 
         def entry(ms: float, cnt: int, per: int, key: str | None, **extra) -> dict:
             e = dict(ms_per_step=ms / per, launches_per_step=cnt / per, avg_launch_us=ms / max(cnt, 1) * 1e3, **extra)
@@ -344,7 +349,8 @@ def run_xkv(args) -> None:
                     ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f16",
                     data="synthetic",
                     config=dict(workload=w["name"], layers=L, heads=H, head_dim=d, tokens_per_frame=n,
-                                budget=w["budget"], kv_bits=w["kv_bits"], prefill_frames=fill, resident_frames=pool,
+                                budget=w["budget"], kv_bits=w["kv_bits"], keys="once" if w["key_mode"] else "regroup",
+                                prefill_frames=fill, resident_frames=pool,
                                 attention="unquantised_tail" if args.tail else "packed",
                                 l2="inputs exceed L2 (about 1.2 GB touched per step)", replicas=world),
                     clocks=clocks.summary(),
@@ -421,7 +427,7 @@ def run_uncompressed(args) -> None:
         flush=True)
 
 
-def maintenance_bytes(H: int, n: int, d: int, budget: int, bits: int) -> dict:
+def maintenance_bytes(H: int, n: int, d: int, budget: int, bits: int, key_mode: int = 0) -> dict:
     """Bytes that one steady-state launch of each cache-maintenance launch has to move (4-bit cache):
     what it reads plus what it writes, every array once.  prunable = budget - n middle tokens are
     scored, k = budget - 2 n of them survive, n new tokens arrive.  Keys are the profile categories:
@@ -440,6 +446,13 @@ def maintenance_bytes(H: int, n: int, d: int, budget: int, bits: int) -> dict:
     # keys regrouped (survivors' codes and parameters, new bf16 keys in; codes and parameters
     # out) and the survivors' value rows and parameters moved
     pack = H * (k * code + grp(k) + n * row + (k + n) * code + grp(k + n)) + 2 * H * k * (code + par)
+    if key_mode == 1:
+        # keys quantised once: the frame's key codes, group parameters and head means are written on
+        # arrival; packing moves the survivors' code rows, value parameters and head-mean rows
+        append = H * n * (2 * row) + H * n * (2 * code + par) + grp(n) * H * 2 + n * 4 * d
+        pack = 2 * H * k * (2 * code + par) + 2 * k * (4 * d + 8)
+        return {"append": append, "score_evict": pool + score + select, "pack": pack,
+                "maint": append + pool + score + select + pack}
     return {"append": append, "score_evict": pool + kbar + score + select, "pack": pack, "kbar": kbar,
             "maint": append + pool + score + select + pack}
 
@@ -454,6 +467,8 @@ def main() -> None:
     ap.add_argument("--budget", type=int, default=0, help="variant of the workload: token budget (ablation sweep)")
     ap.add_argument("--bits", type=int, default=0, choices=[0, 4, 16], help="variant: 4 or 16 (prune only)")
     ap.add_argument("--tokens", type=int, default=0, help="variant: tokens per frame (1004 = long-stream shape)")
+    ap.add_argument("--keys", default="regroup", choices=["regroup", "once"],
+                    help="variant: keys re-quantised per 64-position run every step (default) or quantised once on arrival")
     ap.add_argument("--uncompressed-frames", type=int, default=0,
                     help="instead of the benchmark: stream this many frames through 16-bit caches that never prune")
     ap.add_argument("--tail", action="store_true",

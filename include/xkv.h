@@ -73,7 +73,23 @@ typedef struct {
   int32_t kv_bits;           /* b: 4 or 16                                               */
   int32_t budget;            /* L_max, the token budget (Sec. 3.2), >= 1                 */
   int32_t max_frame_tokens;  /* largest n any frame will have, 1..65535                  */
+  int32_t key_mode;          /* XKV_KEYS_REGROUP (0) or XKV_KEYS_ONCE (1), see below; 4-bit only */
+  int32_t key_table_slots;   /* XKV_KEYS_ONCE: key groups the parameter table can hold;  */
+                             /* 0 = as many as the cache has token slots (never runs out)*/
 } xkv_params;
+
+/* How the per-channel key groups of Eq. 9 (64 tokens each, Sec. 4.1) live with eviction.
+ *   XKV_KEYS_REGROUP  a group is a run of 64 cache positions.  kv_quant_pack regroups the keys
+ *                     after the first frame every step and re-quantises every group whose
+ *                     members changed (Sec. 3.3: "the final KV cache" is quantised).
+ *   XKV_KEYS_ONCE     a group is a run of 64 tokens of one frame, quantised when the frame
+ *                     arrives and never again (the quantiser the paper names, Sec. 4.1, works
+ *                     this way).  A survivor keeps its codes and refers to its group's scales
+ *                     and zero-points in a parameter table; a group's entry is given back when
+ *                     its last token is evicted.  No re-quantisation error accumulates and
+ *                     kv_quant_pack only moves rows.  If the table is sized below the worst case
+ *                     (key_table_slots) and runs out, the status word reads XKV_E_LIMIT. */
+enum { XKV_KEYS_REGROUP = 0, XKV_KEYS_ONCE = 1 };
 
 /* Host-side counters and geometry; filled without touching the device. */
 typedef struct {
@@ -91,6 +107,8 @@ typedef struct {
   int32_t n_pending;         /* tokens of the frame in flight                            */
   int64_t launches;          /* kernels launched for this cache so far                   */
   uint64_t workspace_bytes;
+  int32_t key_table_slots;   /* XKV_KEYS_ONCE: slots of the key parameter table, else 0  */
+  int32_t reserved;
 } xkv_info;
 
 /* Sub-buffers that xkv_debug_export can copy out (physical layout, current
@@ -106,10 +124,15 @@ typedef struct {
  *   SCORES            : float [last_prunable]  importance scores S of Eq. 6 (last evicting step)
  *   KEPT              : int32 [last_kept]      kept middle positions, ascending (last evicting step)
  *   QVEC              : float [d]              row mean of the pooled query (last evicting step)
+ * XKV_KEYS_ONCE only (K_PARAMS is then unused):
+ *   K_SLOT            : int32 [capacity]       parameter-table slot of each token's key group
+ *   K_TABLE           : float2 (scale, zero) [key_table_slots][H][d]
+ *   K_REF             : int32 [key_table_slots] cached tokens that refer to each slot (0 = free)
  */
 typedef enum {
   XKV_BUF_K_CODES = 0, XKV_BUF_K_PARAMS = 1, XKV_BUF_V_CODES = 2, XKV_BUF_V_PARAMS = 3,
-  XKV_BUF_ORIGIN = 4, XKV_BUF_SCORES = 5, XKV_BUF_KEPT = 6, XKV_BUF_QVEC = 7
+  XKV_BUF_ORIGIN = 4, XKV_BUF_SCORES = 5, XKV_BUF_KEPT = 6, XKV_BUF_QVEC = 7,
+  XKV_BUF_K_SLOT = 8, XKV_BUF_K_TABLE = 9, XKV_BUF_K_REF = 10
 } xkv_buffer;
 
 /* ---- set-up ---------------------------------------------------------------- */
@@ -156,7 +179,9 @@ XKV_API int kv_score_evict(xkv_cache* cache, const void* q, int32_t n,
  * middle tokens, current frame: survivors' value codes and parameters are
  * gathered; the keys after the first frame are regrouped into runs of 64 and
  * re-quantised per channel (a complete group whose tokens all survive in place
- * is carried over unchanged).  Afterwards T <= max(L_max, T_first + n).
+ * is carried over unchanged).  With XKV_KEYS_ONCE the keys were quantised by kv_append and
+ * their code rows and group references are gathered like the values.
+ * Afterwards T <= max(L_max, T_first + n).
  * Errors: XKV_E_STATE unless kv_score_evict was the previous call. */
 XKV_API int kv_quant_pack(xkv_cache* cache, xkv_stream stream);
 

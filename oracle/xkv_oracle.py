@@ -97,7 +97,10 @@ class OracleParams:
 # Eq. 2-3: pooled query
 # --------------------------------------------------------------------------
 def n_pooled(n: int, n_special: int, g: int) -> int:
-    return n_special + (max(n - n_special, 0) + g - 1) // g
+    """Rows of the pooled query.  A frame with fewer tokens than special tokens has only special
+    tokens (Eq. 2 splits the frame's tokens; there is nothing else to split)."""
+    n_special = min(n_special, n)
+    return n_special + (n - n_special + g - 1) // g
 
 
 def pooled_query_literal(Q: np.ndarray, n_special: int, g: int) -> np.ndarray:
@@ -120,6 +123,7 @@ def pooled_query_canonical(Q: np.ndarray, n_special: int, g: int) -> np.ndarray:
     """
     Q = np.ascontiguousarray(Q, dtype=F32)
     H, n, d = Q.shape
+    n_special = min(n_special, n)
     Np = n_pooled(n, n_special, g)
     Qbar = np.zeros((Np, d), dtype=F32)
     inv_h = F32(1.0) / F32(H)

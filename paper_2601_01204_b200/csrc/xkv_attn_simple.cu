@@ -10,11 +10,13 @@ constexpr int kSimpleTile = 32;
 
 __device__ __forceinline__ int nib_shift_s(int j) { return ((j >> 1) << 2) + ((j & 1) << 4); }
 
+// ktab: quantise-once mode, the key parameter table [slot][H][64] that buf.kslot refers to
+// (null otherwise: the parameters of a 64-slot run are in buf.kpar).
 template <int BITS>
 __global__ void __launch_bounds__(128)
 attn_simple_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out, int n, int64_t ts,
                    int64_t hs, BufSet buf, int cap, int t_first, int rest_base, int t_phys,
-                   float scale_log2) {
+                   float scale_log2, const float2* __restrict__ ktab, int H) {
   __shared__ __align__(16) float s_k[kSimpleTile][64];
   __shared__ __align__(16) float s_v[kSimpleTile][64];
   const int tid = threadIdx.x;
@@ -51,7 +53,8 @@ attn_simple_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restric
         if (BITS == 4) {
           const uint32_t kw = *reinterpret_cast<const uint32_t*>(buf.k + slot * 32 + 4 * w);
           const uint32_t vw = *reinterpret_cast<const uint32_t*>(buf.v + slot * 32 + 4 * w);
-          const float2* kp = buf.kpar + ((size_t)h * (cap >> 6) + (p >> 6)) * 64 + 8 * w;
+          const float2* kp = ktab ? ktab + ((size_t)buf.kslot[p] * H + h) * 64 + 8 * w
+                                  : buf.kpar + ((size_t)h * (cap >> 6) + (p >> 6)) * 64 + 8 * w;
           const float2 vp = buf.vpar[slot];
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -148,10 +151,11 @@ cudaError_t launch_attn_simple(xkv_cache* c, const void* q, void* out, int n, in
   LaunchScope ls(c, XKV_PROF_ATTN, st);
   if (c->p.kv_bits == 16)
     attn_simple_kernel<16><<<grid, 128, 0, st>>>(qq, oo, n, ts, hs, c->buf[c->cur], c->cap, c->T_first,
-                                                 c->rest_base, t_phys, scale_log2);
+                                                 c->rest_base, t_phys, scale_log2, nullptr, c->p.n_heads);
   else
     attn_simple_kernel<4><<<grid, 128, 0, st>>>(qq, oo, n, ts, hs, c->buf[c->cur], c->cap, c->T_first,
-                                                c->rest_base, t_phys, scale_log2);
+                                                c->rest_base, t_phys, scale_log2,
+                                                c->p.key_mode == XKV_KEYS_ONCE ? c->ktab32 : nullptr, c->p.n_heads);
   return cudaGetLastError();
 }
 

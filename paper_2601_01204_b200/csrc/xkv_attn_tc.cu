@@ -115,6 +115,12 @@ struct Args {
   const __nv_bfloat16* v_tail;
   int64_t tail_ts, tail_hs;
   int tail_lo;
+  // Quantise-once mode: every token refers to the parameter-table slot of its key group
+  // (kslot [cap]); ktab16 [slot][n_heads][8][12] holds, per 8-channel word, the four fp16 pairs
+  // of scales, offsets and constants that dequant_word_h takes.
+  const int32_t* kslot;
+  const uint32_t* ktab16;
+  int n_heads;
 };
 
 __device__ __forceinline__ long long piece_start(long long total, int grid, int b) {
@@ -305,10 +311,7 @@ __device__ __forceinline__ uint32_t h2_fma(uint32_t a, uint32_t b, uint32_t c) {
 
 // Eight 4-bit codes of one packed word -> four fp16 pairs of s * (q - z)  (Eq. 10).
 // (w & 0x000F000F) | 0x6400 is the fp16 number 1024 + q and (w & 0x00F000F0) | 0x5400 is 64 + q.
-// Every pair is formed as  fma(biased - zo, s, c)  with constants chosen per group (dequant_consts):
-//   zo = bias + z, c = 0       when bias + z is an integer fp16 holds exactly (|bias + z| <= 2048):
-//                              the difference is q - z exactly and the product is rounded once;
-//   zo = bias,     c = -s z    otherwise (c formed in fp32): s q + c, valid for any zero-point.
+// Every pair is formed as  fma(biased - zo, s, c)  with the constants of dequant_consts.
 // Pairs 0 and 2 of a word carry the bias 1024, pairs 1 and 3 the bias 64.
 __device__ __forceinline__ uint4 dequant_word_h(uint32_t w, const uint32_t (&s2)[4], const uint32_t (&zo)[4],
                                                 const uint32_t (&c2)[4]) {
@@ -323,15 +326,6 @@ __device__ __forceinline__ uint4 dequant_word_h(uint32_t w, const uint32_t (&s2)
   r.z = h2_fma(h2_sub(a2, zo[2]), s2[2], c2[2]);
   r.w = h2_fma(h2_sub(a3, zo[3]), s2[3], c2[3]);
   return r;
-}
-
-// The constants of dequant_word_h for one (scale, zero-point): both biases must be exact for the
-// first form.  z is an integer-valued float (Eq. 8).
-__device__ __forceinline__ void dequant_consts(float s, float z, float& zo_1024, float& zo_64, float& c) {
-  const bool exact = fabsf(1024.f + z) <= 2048.f && fabsf(64.f + z) <= 2048.f;
-  zo_1024 = exact ? 1024.f + z : 1024.f;
-  zo_64 = exact ? 64.f + z : 64.f;
-  c = exact ? 0.f : -s * z;
 }
 
 // fp16 can hold magnitudes up to 65504; anything beyond (or not a number) is reported.
@@ -405,7 +399,9 @@ __device__ __forceinline__ void producer_sync() { asm volatile("bar.sync 1, 128;
 
 // TAIL: the newest frame's keys and values come unquantised from Args::k_tail, v_tail (a separate
 // instantiation, so that the kernel without a tail carries none of its code).
-template <int BITS, bool TAIL = false>
+// ONCE: the keys' dequantisation constants are looked up per token (quantise-once mode) instead of
+// per 64-slot run.
+template <int BITS, bool TAIL = false, bool ONCE = false>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
   using C = Cfg<BITS>;
   extern __shared__ uint8_t smem_raw[];
@@ -727,27 +723,61 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           // ---- fp16 parameter tables of this tile (one (group, channel) and one key per thread) ----
           uint8_t* tab = sgen + kOffTab + (g & 1) * kTabBytes;
           {
-            const float2 kp = *reinterpret_cast<const float2*>(raw + C::kRawK + C::kRawV + 8 * t);  // (group t>>6, channel t&63)
-            float zl, zh, kc;
-            dequant_consts(kp.x, kp.y, zl, zh, kc);
-            __half* ks = reinterpret_cast<__half*>(tab);              // [2][64] scales, [2][64] offsets, [2][64] constants
-            ks[t] = __float2half_rn(kp.x);
-            ks[128 + t] = __float2half_rn((((t & 7) >> 1) & 1) ? zh : zl);
-            ks[256 + t] = __float2half_rn(kc);
+            bool k_bad = false;
+            if (!ONCE) {
+              const float2 kp = *reinterpret_cast<const float2*>(raw + C::kRawK + C::kRawV + 8 * t);  // (group t>>6, channel t&63)
+              float zl, zh, kc;
+              dequant_consts(kp.x, kp.y, zl, zh, kc);
+              __half* ks = reinterpret_cast<__half*>(tab);              // [2][64] scales, [2][64] offsets, [2][64] constants
+              ks[t] = __float2half_rn(kp.x);
+              ks[128 + t] = __float2half_rn((((t & 7) >> 1) & 1) ? zh : zl);
+              ks[256 + t] = __float2half_rn(kc);
+              k_bad = beyond_fp16(fabsf(kp.x) * (fabsf(kp.y) + 15.f));
+            }
             const float2 vp = *reinterpret_cast<const float2*>(raw + C::kRawK + C::kRawV + C::kRawKP + 8 * t);   // key t
             float vl, vh, vc;
             dequant_consts(vp.x, vp.y, vl, vh, vc);
             *reinterpret_cast<uint4*>(tab + 768 + 16 * t) =
                 make_uint4(pack_h2(vp.x, vp.x), pack_h2(vl, vl), pack_h2(vh, vh), pack_h2(vc, vc));
             // largest magnitude a code of this group / token can dequantise to
-            if (beyond_fp16(fabsf(kp.x) * (fabsf(kp.y) + 15.f)) || beyond_fp16(fabsf(vp.x) * (fabsf(vp.y) + 15.f)))
-              report_range(a.status);
+            if (k_bad || beyond_fp16(fabsf(vp.x) * (fabsf(vp.y) + 15.f))) report_range(a.status);
           }
           producer_sync();
           // ---- keys ----
           uint32_t wd[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) wd[i] = *reinterpret_cast<const uint32_t*>(raw + (kb + 16 * i) * 32 + 4 * w);
+          if (ONCE) {
+            // constants of each token's own key group, from the table in global memory (the tokens of
+            // a group mostly sit next to each other, so the lines are shared); four tokens at a time
+            int sl[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sl[i] = *reinterpret_cast<const int*>(raw + C::kRawK + C::kRawV + 4 * (kb + 16 * i));
+            uint4 sv[4], zv[4], cv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint4* e = reinterpret_cast<const uint4*>(a.ktab16 + (((size_t)sl[i] * a.n_heads + h) * 8 + w) * 12);
+              sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2);
+            }
+            mbar_wait<256>(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const uint32_t s2[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w}, zo[4] = {zv[i].x, zv[i].y, zv[i].z, zv[i].w};
+                const uint32_t c2[4] = {cv[i].x, cv[i].y, cv[i].z, cv[i].w};
+                const uint4 o = dequant_word_h(wd[4 * half + i], s2, zo, c2);
+                *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (4 * half + i) * 2048) = o;
+              }
+              if (half == 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const uint4* e = reinterpret_cast<const uint4*>(a.ktab16 + (((size_t)sl[4 + i] * a.n_heads + h) * 8 + w) * 12);
+                  sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2);
+                }
+              }
+            }
+          } else {
           mbar_wait<256>(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
 #pragma unroll
           for (int grp = 0; grp < 2; ++grp) {
@@ -761,6 +791,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
               const uint4 o = dequant_word_h(wd[4 * grp + i], s2, zo, c2);
               *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (4 * grp + i) * 2048) = o;
             }
+          }
           }
           if (TAIL && tail_tile)
             tail_rows_over(sgen + kOffK + kbuf * 16384 + row_off, a.k_tail + tail_off, a.tail_ts, slot0, a.tail_lo, a.t_phys, a.status);
@@ -876,12 +907,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
         const uint32_t rs = g % C::kNR, ru = g / C::kNR;
         mbar_wait<256>(b_rfree + 8 * rs, (ru & 1) ^ 1, wc);
         const uint32_t dst = sRaw + rs * C::kRawStage, bar = b_rfull + 8 * rs;
-        mbar_expect_tx(bar, C::kRawStage);
+        const uint32_t kp_bytes = ONCE ? 512u : (uint32_t)C::kRawKP;    // 128 group references instead of 2 x 64 parameters
+        mbar_expect_tx(bar, C::kRawStage - C::kRawKP + kp_bytes);
         const size_t slot0 = head_slot + (size_t)tile * 128;
         if (BITS == 4) {
           tma_load_1d(dst, a.k + slot0 * 32, C::kRawK, bar);
           tma_load_1d(dst + C::kRawK, a.v + slot0 * 32, C::kRawV, bar);
-          tma_load_1d(dst + C::kRawK + C::kRawV, a.kpar + ((size_t)h * (a.cap >> 6) + 2 * tile) * 64, C::kRawKP, bar);
+          if (ONCE) tma_load_1d(dst + C::kRawK + C::kRawV, a.kslot + (size_t)tile * 128, kp_bytes, bar);
+          else tma_load_1d(dst + C::kRawK + C::kRawV, a.kpar + ((size_t)h * (a.cap >> 6) + 2 * tile) * 64, C::kRawKP, bar);
           tma_load_1d(dst + C::kRawK + C::kRawV + C::kRawKP, a.vpar + slot0, C::kRawVP, bar);
         } else {
           tma_load_1d(dst, a.k + slot0 * 128, C::kRawK, bar);
@@ -1008,6 +1041,10 @@ static cudaError_t attn_device_setup(int* sm_count) {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_tc_kernel<4, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_tc_kernel<4, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
+    if (e != cudaSuccess) return e;
     g_sm_count[dev] = sms;
   }
   *sm_count = g_sm_count[dev];
@@ -1046,6 +1083,7 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
   a.part_o = part;
   a.part_ml = reinterpret_cast<float2*>(part + slots * kSlotFloats);
   a.status = c->status;
+  a.kslot = b.kslot; a.ktab16 = c->ktab16; a.n_heads = H;
   a.k_tail = a.v_tail = nullptr;
   a.tail_ts = a.tail_hs = 0;
   a.tail_lo = a.t_phys;
@@ -1058,8 +1096,11 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
   }
   {
     LaunchScope ls(c, XKV_PROF_ATTN, st);
+    const bool once = c->p.key_mode == XKV_KEYS_ONCE;
     if (c->p.kv_bits == 16) attn_tc_kernel<16><<<(int)grid, kThreads, smem_bytes<16>(), st>>>(a);
+    else if (a.k_tail && once) attn_tc_kernel<4, true, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
     else if (a.k_tail) attn_tc_kernel<4, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
+    else if (once) attn_tc_kernel<4, false, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
     else attn_tc_kernel<4><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;

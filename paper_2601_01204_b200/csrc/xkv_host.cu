@@ -20,6 +20,8 @@ struct Layout {
   size_t off_k[2], off_kpar[2], off_v[2], off_vpar[2], off_origin[2], off_kbar[2];
   size_t off_kstage, off_qbar, off_qvec, off_scores, off_kept, off_counters, off_status, off_attn, off_hist;
   size_t off_run_hi, off_cand;
+  size_t off_kslot[2], off_ktab32, off_ktab16, off_ref, off_ring;
+  int n_slots;
   size_t attn_bytes;
   size_t total;
 };
@@ -32,6 +34,9 @@ bool params_ok(const xkv_params* p) {
   if (p->n_special < 0 || p->pool_g < 1 || p->budget < 1) return false;
   if (p->max_frame_tokens < 1 || p->max_frame_tokens > 65535) return false;
   if (p->budget > (1 << 24)) return false;
+  if (p->key_mode != XKV_KEYS_REGROUP && p->key_mode != XKV_KEYS_ONCE) return false;
+  if (p->key_mode == XKV_KEYS_ONCE && p->kv_bits != 4) return false;
+  if (p->key_table_slots < 0 || (p->key_mode != XKV_KEYS_ONCE && p->key_table_slots != 0)) return false;
   return true;
 }
 
@@ -66,6 +71,17 @@ Layout make_layout(const xkv_params* p) {
   L.off_kept = take((size_t)L.cap * sizeof(int32_t));
   L.off_run_hi = take((size_t)(L.cap / 64) * sizeof(unsigned int));
   L.off_cand = take((size_t)L.cap * sizeof(unsigned long long));
+  if (p->key_mode == XKV_KEYS_ONCE) {
+    // every live group holds at least one cached token, so one slot per token slot never runs out;
+    // at least the groups of two frames (the first and the one arriving) are needed in any case
+    const int least = 2 * ((max_n + 63) / 64) + 1;
+    L.n_slots = p->key_table_slots > 0 ? (p->key_table_slots > least ? p->key_table_slots : least) : L.cap;
+    for (int b = 0; b < 2; ++b) L.off_kslot[b] = take((size_t)L.cap * sizeof(int32_t));
+    L.off_ktab32 = take((size_t)L.n_slots * H * 64 * sizeof(float2));
+    L.off_ktab16 = take((size_t)L.n_slots * H * 8 * 12 * sizeof(uint32_t));
+    L.off_ref = take((size_t)L.n_slots * sizeof(int32_t));
+    L.off_ring = take((size_t)L.n_slots * sizeof(int32_t));
+  }
   L.attn_bytes = attn_tc_scratch_bytes(p);
   L.off_attn = take(L.attn_bytes);
   L.total = off;
@@ -76,7 +92,9 @@ bool strides_ok(int64_t ts, int64_t hs) { return ts >= kHeadDim && (ts % 8) == 0
 bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int zero_workspace(xkv_cache* c, cudaStream_t st) {
-  return cudaMemsetAsync(c->ws, 0, c->ws_bytes, st) == cudaSuccess ? XKV_OK : XKV_E_CUDA;
+  if (cudaMemsetAsync(c->ws, 0, c->ws_bytes, st) != cudaSuccess) return XKV_E_CUDA;
+  if (c->p.key_mode == XKV_KEYS_ONCE && launch_once_init(c, st) != cudaSuccess) return XKV_E_CUDA;
+  return XKV_OK;
 }
 
 void reset_host_state(xkv_cache* c) {
@@ -86,6 +104,7 @@ void reset_host_state(xkv_cache* c) {
   c->kbar_T = c->kbar_cur = c->kbar_frames = -1;
   c->bar_base = 0;
   c->sel_parity = 0;
+  c->pop_base = 0;
 }
 
 }  // namespace
@@ -125,7 +144,14 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
     c->buf[b].vpar = reinterpret_cast<float2*>(c->ws + L.off_vpar[b]);
     c->buf[b].origin = reinterpret_cast<int32_t*>(c->ws + L.off_origin[b]);
     c->buf[b].kbar = reinterpret_cast<float*>(c->ws + L.off_kbar[b]);
-    c->buf[b].kslot = nullptr;
+    c->buf[b].kslot = params->key_mode == XKV_KEYS_ONCE ? reinterpret_cast<int32_t*>(c->ws + L.off_kslot[b]) : nullptr;
+  }
+  if (params->key_mode == XKV_KEYS_ONCE) {
+    c->n_slots = L.n_slots;
+    c->ktab32 = reinterpret_cast<float2*>(c->ws + L.off_ktab32);
+    c->ktab16 = reinterpret_cast<uint32_t*>(c->ws + L.off_ktab16);
+    c->ref = reinterpret_cast<int32_t*>(c->ws + L.off_ref);
+    c->ring = reinterpret_cast<int32_t*>(c->ws + L.off_ring);
   }
   c->kstage = reinterpret_cast<__nv_bfloat16*>(c->ws + L.off_kstage);
   c->qbar = reinterpret_cast<float*>(c->ws + L.off_qbar);
@@ -212,7 +238,11 @@ void maint_args(const xkv_cache* c, MaintArgs* a) {
   a->kstage = c->kstage; a->qbar = c->qbar; a->qvec = c->qvec; a->scores = c->scores; a->kept = c->kept;
   a->hist = c->sel_hist; a->run_hi = c->run_hi; a->cand = c->cand;
   a->force_plain = c->force_plain;
+  a->ktab32 = c->ktab32; a->ktab16 = c->ktab16; a->ref = c->ref; a->ring = c->ring;
+  a->n_slots = c->n_slots; a->pop_base = c->pop_base;
 }
+
+bool keys_once(const xkv_cache* c) { return c->p.key_mode == XKV_KEYS_ONCE; }
 
 void set_pending(xkv_cache* c, int n, const FramePlan& p) {
   c->n_pending = n;
@@ -268,10 +298,12 @@ int kv_append(xkv_cache* c, const void* k, const void* v, int32_t n, int64_t ts,
   MaintArgs a;
   maint_args(c, &a);
   a.phases = kPhAppend;
+  if (keys_once(c) && !plan.first) a.phases |= kPhKbarNew;
   a.k = reinterpret_cast<const __nv_bfloat16*>(k);
   a.v = reinterpret_cast<const __nv_bfloat16*>(v);
   a.ts_kv = ts; a.hs_kv = hs;
   if (launch_maint(c, a, XKV_PROF_APPEND, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
+  if (keys_once(c)) c->pop_base += (uint32_t)((n + 63) / 64);
   c->stage = 1;
   return XKV_OK;
 }
@@ -285,14 +317,14 @@ int kv_score_evict(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t h
     MaintArgs a;
     maint_args(c, &a);
     a.phases = kPhPool | kPhScore | kPhSel;
-    if (!kbar_fresh(c)) {          // head means of the keys (Eq. 4) of the cache as it stands
+    if (!keys_once(c) && !kbar_fresh(c)) {          // head means of the keys (Eq. 4) of the cache as it stands
       a.phases |= kPhKbar;
       a.kbar_on_other = 0; a.kbar_lo = 0; a.kbar_hi = c->rold_pending;
     }
     a.q = reinterpret_cast<const __nv_bfloat16*>(q);
     a.ts_q = ts; a.hs_q = hs;
     if (launch_maint(c, a, XKV_PROF_SCORE_EVICT, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
-    c->kbar_T = c->T; c->kbar_cur = c->cur; c->kbar_frames = c->frames;
+    if (!keys_once(c)) { c->kbar_T = c->T; c->kbar_cur = c->cur; c->kbar_frames = c->frames; }
   }
   c->stage = 2;
   return XKV_OK;
@@ -303,9 +335,9 @@ int kv_quant_pack(xkv_cache* c, xkv_stream stream) {
   if (c->stage != 2) return XKV_E_STATE;
   MaintArgs a;
   maint_args(c, &a);
-  if (c->p.kv_bits == 4) {
+  if (c->p.kv_bits == 4 && !keys_once(c)) {
     if (launch_regroup(c, a, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
-  } else if (c->kk_pending > 0) {                   // a 16-bit cache without survivors to move has nothing to do
+  } else if (c->kk_pending > 0 || (keys_once(c) && c->rold_pending > 0)) {   // survivors to move, or table slots to release
     a.phases = kPhPack;
     if (launch_maint(c, a, XKV_PROF_PACK, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
   }
@@ -424,11 +456,15 @@ int run_layer(HostStepPipe* pipe, xkv_cache* c, const void* q, const void* k, co
   note_scored(c);
   MaintArgs a;
   maint_args(c, &a);
+  const bool once = keys_once(c);
   a.phases = kPhAppend;
-  if (c->p.kv_bits == 16 && c->kk_pending > 0) a.phases |= kPhPack;
+  if ((c->p.kv_bits == 16 && c->kk_pending > 0) || (once && (c->kk_pending > 0 || c->rold_pending > 0))) a.phases |= kPhPack;
+  if (once && !plan.first) a.phases |= kPhKbarNew;
   if (selecting(c)) {
     a.phases |= kPhPool | kPhScore | kPhSel;
-    if (kbar_fresh(c)) {
+    if (once) {
+      // the head means travel with the tokens: nothing to wait for, nothing to recompute
+    } else if (kbar_fresh(c)) {
       if (cudaStreamWaitEvent(st, c->kbar_done, 0) != cudaSuccess) return XKV_E_CUDA;
     } else {
       a.phases |= kPhKbar;
@@ -440,10 +476,11 @@ int run_layer(HostStepPipe* pipe, xkv_cache* c, const void* q, const void* k, co
   a.v = reinterpret_cast<const __nv_bfloat16*>(v);
   a.ts_q = a.ts_kv = ts; a.hs_q = a.hs_kv = hs;
   if (launch_maint(c, a, XKV_PROF_MAINT, st) != cudaSuccess) return XKV_E_CUDA;
-  if (c->p.kv_bits == 4 && launch_regroup(c, a, st) != cudaSuccess) return XKV_E_CUDA;
+  if (once) c->pop_base += (uint32_t)((n + 63) / 64);
+  if (c->p.kv_bits == 4 && !once && launch_regroup(c, a, st) != cudaSuccess) return XKV_E_CUDA;
   note_packed(c);
   c->stage = 3;
-  if (c->T > c->T_first) {
+  if (!once && c->T > c->T_first) {
     bool ok = cudaEventRecord(pipe->fork, st) == cudaSuccess && cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess;
     if (!ok) return XKV_E_CUDA;
     MaintArgs b;
@@ -573,6 +610,8 @@ int xkv_get_info(const xkv_cache* c, xkv_info* info) {
   info->n_pending = c->n_pending;
   info->launches = c->launches;
   info->workspace_bytes = c->ws_bytes;
+  info->key_table_slots = c->n_slots;
+  info->reserved = 0;
   return XKV_OK;
 }
 
@@ -593,6 +632,9 @@ int64_t xkv_debug_export(const xkv_cache* c, int32_t which, void* host_dst, size
     case XKV_BUF_SCORES: src = c->scores; avail = (size_t)c->last_prunable * sizeof(float); break;
     case XKV_BUF_KEPT: src = c->kept; avail = (size_t)c->last_kept * sizeof(int32_t); break;
     case XKV_BUF_QVEC: src = c->qvec; avail = 64 * sizeof(float); break;
+    case XKV_BUF_K_SLOT: src = b.kslot; avail = b.kslot ? (size_t)c->cap * sizeof(int32_t) : 0; break;
+    case XKV_BUF_K_TABLE: src = c->ktab32; avail = (size_t)c->n_slots * H * 64 * sizeof(float2); break;
+    case XKV_BUF_K_REF: src = c->ref; avail = (size_t)c->n_slots * sizeof(int32_t); break;
     default: return XKV_E_INVALID;
   }
   const size_t nbytes = bytes < avail ? bytes : avail;
@@ -613,7 +655,7 @@ int xkv_poll_status(const xkv_cache* c, xkv_stream stream) {
   int word = 0;
   if (cudaMemcpy(&word, c->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return XKV_E_CUDA;
   if (word == 0) return XKV_OK;
-  return word == (int)XKV_E_RANGE ? XKV_E_RANGE : XKV_E_TIMEOUT;
+  return (word == (int)XKV_E_RANGE || word == (int)XKV_E_LIMIT) ? word : XKV_E_TIMEOUT;
 }
 
 int xkv_debug_force_plain(xkv_cache* c, int32_t on) {
@@ -631,7 +673,7 @@ int xkv_debug_limit_attention_blocks(xkv_cache* c, int32_t max_blocks) {
 int xkv_debug_head_means(xkv_cache* c, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;
   if (c->stage != 0) return XKV_E_STATE;
-  if (c->T <= c->T_first) return XKV_OK;
+  if (c->T <= c->T_first || keys_once(c)) return XKV_OK;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (c->kbar_done && cudaStreamWaitEvent(st, c->kbar_done, 0) != cudaSuccess) return XKV_E_CUDA;
   MaintArgs a;

@@ -30,6 +30,7 @@ struct BufSet {
 
 // Phases of the maintenance kernel (bit mask) and its arguments.
 constexpr uint32_t kPhAppend = 1u, kPhPool = 2u, kPhKbar = 4u, kPhScore = 8u, kPhSel = 16u, kPhPack = 32u;
+constexpr uint32_t kPhKbarNew = 64u;   // quantise-once mode: head means of the frame just quantised
 struct MaintArgs {
   uint32_t phases;
   // the frame
@@ -53,7 +54,14 @@ struct MaintArgs {
   unsigned int* cand_count_next;   // counter of the next selecting launch (cleared by this one)
   unsigned int* hist2;             // [256] histogram of the candidates' next 8 key bits
   unsigned int* hist2_next;        // the next selecting launch's (cleared by this one)
-  int32_t* ref; int32_t* free_list; int* free_top;   // quantise-once mode: parameter-table bookkeeping
+  // quantise-once mode: the key parameter table and its bookkeeping
+  float2* ktab32;                  // [n_slots][H][64] (scale, zero)
+  uint32_t* ktab16;                // [n_slots][H][8][12] fp16 constants for the attention's operand path
+  int32_t* ref;                    // [n_slots] cached tokens per slot
+  int32_t* ring;                   // [n_slots] free slots, a ring: taken at host-known places, given back by atomics
+  unsigned int* push_pos;          // slots given back so far (+ n_slots: the ring starts full)
+  uint32_t pop_base;               // slots taken before this launch
+  int n_slots;
   int force_plain;
   unsigned int* bar; uint32_t bar_base;
   int* status;
@@ -92,6 +100,10 @@ struct xkv_cache {
   unsigned int* sel_hist;  // [4096] histogram of the top 12 bits of the score keys (self-clearing)
   unsigned int* run_hi;    // [cap / 64]
   unsigned long long* cand;  // [cap]
+  // quantise-once mode
+  float2* ktab32; uint32_t* ktab16; int32_t* ref; int32_t* ring;
+  int n_slots;
+  uint32_t pop_base;       // key groups that have taken a table slot so far
   int* status;             // device status word
   float* attn_part;        // split-KV partials of the attention kernel
   size_t attn_part_bytes;
@@ -113,6 +125,21 @@ struct xkv_cache {
 namespace xkv {
 
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+#ifdef __CUDACC__
+// Constants of the attention's fp16 dequantisation for one (scale, zero-point) of Eq. 8: a pair
+// of codes is formed as fma(biased_code - zo, s, c), the code carrying a bias of 1024 or 64
+// (its fp16 bit pattern is built by OR-ing the nibble into the mantissa of 1024 resp. 64).
+//   zo = bias + z, c = 0     when fp16 holds bias + z exactly (|bias + z| <= 2048, z an integer):
+//                            the difference is q - z exactly and the product is rounded once;
+//   zo = bias,     c = -s z  otherwise (c formed in fp32): s q + c, valid for any zero-point.
+__device__ __forceinline__ void dequant_consts(float s, float z, float& zo_1024, float& zo_64, float& c) {
+  const bool exact = fabsf(1024.f + z) <= 2048.f && fabsf(64.f + z) <= 2048.f;
+  zo_1024 = exact ? 1024.f + z : 1024.f;
+  zo_64 = exact ? 64.f + z : 64.f;
+  c = exact ? 0.f : -s * z;
+}
+#endif
 
 // Brackets one kernel launch with events when profiling is on; counts the launch.
 struct LaunchScope {
@@ -139,6 +166,8 @@ struct LaunchScope {
 // The maintenance kernel with the phases in a.phases (cooperative when it has a grid barrier).
 // Fills in the barrier and status fields of `a`; everything else is the caller's.
 cudaError_t launch_maint(xkv_cache* c, MaintArgs& a, int prof_cat, cudaStream_t st);
+// Quantise-once mode: fills the ring of free parameter-table slots (after the workspace was zeroed).
+cudaError_t launch_once_init(xkv_cache* c, cudaStream_t st);
 // kv_quant_pack of a 4-bit cache: key regroup + re-quantisation fused with the survivor gather.
 cudaError_t launch_regroup(xkv_cache* c, const MaintArgs& a, cudaStream_t st);
 cudaError_t launch_attn_simple(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,

@@ -152,6 +152,7 @@ union __align__(16) Smem {
   struct { float2 par[64 * 64]; } kbar;                                            // [H][64] key parameters of one group
   struct { float w[64]; float rows[kPoolRows * 64]; } score;
   struct { unsigned long long cand[kCandSmem]; unsigned long long list[kSubList]; } sel;   // (key << 32) | ~position
+  struct { float mn[4][4][64]; float mx[4][4][64]; float2 iz[4][64]; } kq;          // quantise-once: one key group, 4 heads
 };
 
 struct Shared {
@@ -234,7 +235,7 @@ __device__ __forceinline__ bool grid_barrier(const MaintArgs& a, uint32_t& epoch
 // word per lane.  Keys: copied to the staging buffer (4-bit) or to their final
 // slot (16-bit).
 // ---------------------------------------------------------------------------
-template <int BITS>
+template <int BITS, bool ONCE>
 __device__ __forceinline__ void phase_append(const MaintArgs& a) {
   const long long items = (long long)a.H * a.n * 8;
   const int passes = (int)((items + kMT - 1) / kMT);
@@ -286,7 +287,7 @@ __device__ __forceinline__ void phase_append(const MaintArgs& a) {
           *reinterpret_cast<uint32_t*>(d1.v + slot * 32 + 4 * w) = word;
           if (w == 0) d1.vpar[slot] = make_float2(s, z);
         }
-        __stcg(reinterpret_cast<uint4*>(a.kstage + ((size_t)h * a.max_n + tok) * 64 + 8 * w), kv);
+        if (!ONCE) __stcg(reinterpret_cast<uint4*>(a.kstage + ((size_t)h * a.max_n + tok) * 64 + 8 * w), kv);
       }
     }
     if (valid && h == 0 && w == 0) {
@@ -459,6 +460,198 @@ __device__ __forceinline__ void phase_kbar(const MaintArgs& a, Shared& sh, const
 }
 
 // ---------------------------------------------------------------------------
+// Quantise-once mode, APPEND: the frame's keys are quantised here, per channel in groups of 64
+// consecutive tokens of the frame (Eq. 7-9), and never again.  Item = (group, four heads); 128
+// threads per head, thread = (8-channel word, four tokens 16 apart).  Each group takes a slot
+// of the parameter table: fp32 (scale, zero) for the maintenance arithmetic and the constants
+// of the attention's fp16 operand path.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+__device__ __forceinline__ void phase_quant_keys_once(const MaintArgs& a, Shared& sh) {
+  const BufSet& d0 = a.oth;
+  const BufSet& d1 = a.cur;
+  const bool two = a.first != 0;
+  const int H = a.H, cap = a.cap, n = a.n;
+  const int tid = threadIdx.x;
+  const int hl = tid >> 7, t = tid & 127, w = t & 7, tq = t >> 3, wih = t >> 5;
+  const int n_groups = (n + 63) >> 6, n_quads = (H + 3) >> 2;
+  const int items = n_groups * n_quads;
+  for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    const int gamma = item / n_quads, quad = item - gamma * n_quads;
+    const int h = quad * 4 + hl;
+    const bool head_ok = h < H;
+    // the group's table slot: the ring of free slots is read at places the host has counted out
+    const uint32_t take = a.pop_base + (uint32_t)gamma;
+    const int slot = __ldcg(&a.ring[take % (uint32_t)a.n_slots]);
+    if (tid == 0 && quad == 0) {
+      if ((int)(take - __ldcg(a.push_pos)) >= 0) atomicCAS(a.status, 0, (int)XKV_E_LIMIT);   // the table has run out
+      a.ref[slot] = min(64, n - gamma * 64);
+    }
+    float x[4][8];
+    bool live[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int tok = gamma * 64 + tq + 16 * u;
+      live[u] = tok < n;
+      uint4 raw = make_uint4(0, 0, 0, 0);
+      if (live[u] && head_ok) raw = *reinterpret_cast<const uint4*>(a.k + (int64_t)h * a.hs_kv + (int64_t)tok * a.ts_kv + 8 * w);
+      bf16x8_to_float(raw, x[u]);
+    }
+    float mn[8], mx[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { mn[j] = INFINITY; mx[j] = -INFINITY; }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (live[u]) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { mn[j] = fminf(mn[j], x[u][j]); mx[j] = fmaxf(mx[j], x[u][j]); }
+      }
+    }
+#pragma unroll
+    for (int o = 8; o < 32; o <<= 1) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        mn[j] = fminf(mn[j], __shfl_xor_sync(0xffffffffu, mn[j], o));
+        mx[j] = fmaxf(mx[j], __shfl_xor_sync(0xffffffffu, mx[j], o));
+      }
+    }
+    __syncthreads();                 // the previous item's parameters have been read
+    if ((t & 31) < 8) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { sh.u.kq.mn[hl][wih][8 * w + j] = mn[j]; sh.u.kq.mx[hl][wih][8 * w + j] = mx[j]; }
+    }
+    __syncthreads();
+    if (t < 64) {                    // one thread per channel: the group's parameters (warps 0, 1 of the head)
+      float lo = sh.u.kq.mn[hl][0][t], hi = sh.u.kq.mx[hl][0][t];
+#pragma unroll
+      for (int r = 1; r < 4; ++r) { lo = fminf(lo, sh.u.kq.mn[hl][r][t]); hi = fmaxf(hi, sh.u.kq.mx[hl][r][t]); }
+      float sc, inv, z;
+      quant_params(lo, hi, sc, inv, z);
+      sh.u.kq.iz[hl][t] = make_float2(inv, z);
+      float zl, zh, cc;
+      dequant_consts(sc, z, zl, zh, cc);
+      const float zo = (((t & 7) >> 1) & 1) ? zh : zl;
+      // the neighbouring channel's constants: pairs (2p, 2p + 1) share a word
+      const float sc1 = __shfl_xor_sync(0xffffffffu, sc, 1), zo1 = __shfl_xor_sync(0xffffffffu, zo, 1);
+      const float cc1 = __shfl_xor_sync(0xffffffffu, cc, 1);
+      if (head_ok) {
+        a.ktab32[((size_t)slot * H + h) * 64 + t] = make_float2(sc, z);
+        if ((t & 1) == 0) {
+          uint32_t* e = a.ktab16 + (((size_t)slot * H + h) * 8 + (t >> 3)) * 12 + ((t & 7) >> 1);
+          e[0] = pack_half2(sc, sc1);
+          e[4] = pack_half2(zo, zo1);
+          e[8] = pack_half2(cc, cc1);
+        }
+        if (!(fabsf(sc) * (fabsf(z) + 15.f) <= 65504.f)) atomicCAS(a.status, 0, (int)XKV_E_RANGE);
+      }
+    }
+    __syncthreads();
+    if (head_ok) {
+      float2 iz[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) iz[j] = sh.u.kq.iz[hl][8 * w + j];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (!live[u]) continue;
+        uint32_t c[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) c[j] = quant_code(x[u][j], iz[j].x, iz[j].y);
+        const uint32_t word = pack8(c);
+        const size_t dslot = (size_t)h * cap + a.dst_slot + gamma * 64 + tq + 16 * u;
+        *reinterpret_cast<uint32_t*>(d0.k + dslot * 32 + 4 * w) = word;
+        if (two) *reinterpret_cast<uint32_t*>(d1.k + dslot * 32 + 4 * w) = word;
+      }
+    }
+    if (quad == 0 && tid < 64 && gamma * 64 + tid < n) {
+      d0.kslot[a.dst_slot + gamma * 64 + tid] = slot;
+      if (two) d1.kslot[a.dst_slot + gamma * 64 + tid] = slot;
+    }
+  }
+}
+
+// Quantise-once mode: head means (Eq. 4) of the frame just quantised, into the destination's
+// array.  Thread = (token, 8-channel word), heads in order, plain Eq. 10.
+__device__ __forceinline__ void phase_kbar_new_once(const MaintArgs& a) {
+  const int tid = threadIdx.x, w = tid & 7, tok = tid >> 3;
+  const int n_groups = (a.n + 63) >> 6;
+  const BufSet& d = a.oth;
+  for (int gamma = blockIdx.x; gamma < n_groups; gamma += gridDim.x) {
+    const int tix = gamma * 64 + tok;
+    if (tix >= a.n) continue;
+    const int slot = __ldcg(&d.kslot[a.dst_slot + tix]);
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    for (int h = 0; h < a.H; ++h) {
+      const uint32_t word = __ldcg(reinterpret_cast<const uint32_t*>(d.k + ((size_t)h * a.cap + a.dst_slot + tix) * 32 + 4 * w));
+      const float4* pp = reinterpret_cast<const float4*>(a.ktab32 + ((size_t)slot * a.H + h) * 64 + 8 * w);
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        const float4 p4 = __ldcg(pp + v);
+        const float x0 = __fmul_rn(p4.x, __fsub_rn((float)((word >> nib_shift(2 * v)) & 0xFu), p4.y));
+        const float x1 = __fmul_rn(p4.z, __fsub_rn((float)((word >> nib_shift(2 * v + 1)) & 0xFu), p4.w));
+        acc[2 * v] = (h == 0) ? x0 : __fadd_rn(acc[2 * v], x0);
+        acc[2 * v + 1] = (h == 0) ? x1 : __fadd_rn(acc[2 * v + 1], x1);
+      }
+    }
+    const float inv_h = __fdiv_rn(1.f, (float)a.H);
+    float4* dst = reinterpret_cast<float4*>(d.kbar + (size_t)(a.dst_slot - a.rest_base + tix) * 64 + 8 * w);
+    __stcg(dst, make_float4(__fmul_rn(acc[0], inv_h), __fmul_rn(acc[1], inv_h), __fmul_rn(acc[2], inv_h), __fmul_rn(acc[3], inv_h)));
+    __stcg(dst + 1, make_float4(__fmul_rn(acc[4], inv_h), __fmul_rn(acc[5], inv_h), __fmul_rn(acc[6], inv_h), __fmul_rn(acc[7], inv_h)));
+  }
+}
+
+// Quantise-once mode, PACK: the survivors' key and value code rows, value parameters, group
+// references, origins and head means move to their new places in the other buffer set.
+__device__ __forceinline__ void phase_gather_once(const MaintArgs& a) {
+  const BufSet& src = a.cur;
+  const BufSet& dst = a.oth;
+  const int32_t* kept = a.identity ? nullptr : a.kept;
+  const long long stride = (long long)gridDim.x * kMT;
+  const long long first = (long long)blockIdx.x * kMT + threadIdx.x;
+  if (a.kk == 0) {
+    // the budget leaves no room for the middle (k = 0): every token after the first frame leaves,
+    // without a selection; their key groups give their table slots back
+    for (long long i = first; i < a.r_old; i += stride) {
+      const int slot = __ldcg(&src.kslot[a.rest_base + i]);
+      if (atomicSub(&a.ref[slot], 1) == 1) a.ring[atomicAdd(a.push_pos, 1u) % (unsigned int)a.n_slots] = slot;
+    }
+    return;
+  }
+  const long long items = (long long)a.H * a.kk * 4;                 // (head, survivor, 16-byte chunk of K | V codes)
+  for (long long g = first; g < items; g += stride) {
+    const int ch = (int)(g & 3);
+    const long long r = g >> 2;
+    const int i = (int)(r % a.kk);
+    const int h = (int)(r / a.kk);
+    const int old = kept ? __ldcg(&kept[i]) : i;
+    const size_t s = (size_t)h * a.cap + a.rest_base + old;
+    const size_t d = (size_t)h * a.cap + a.rest_base + i;
+    if (ch < 2) {
+      *reinterpret_cast<uint4*>(dst.k + d * 32 + 16 * ch) = *reinterpret_cast<const uint4*>(src.k + s * 32 + 16 * ch);
+    } else {
+      *reinterpret_cast<uint4*>(dst.v + d * 32 + 16 * (ch - 2)) = *reinterpret_cast<const uint4*>(src.v + s * 32 + 16 * (ch - 2));
+      if (ch == 2) dst.vpar[d] = src.vpar[s];
+    }
+  }
+  const long long rows = (long long)a.kk * 16;                       // (survivor, 16-byte chunk of its head-mean row)
+  for (long long g = first; g < rows; g += stride) {
+    const int ch = (int)(g & 15);
+    const int i = (int)(g >> 4);
+    const int old = kept ? __ldcg(&kept[i]) : i;
+    reinterpret_cast<float4*>(dst.kbar + (size_t)i * 64)[ch] = __ldcg(reinterpret_cast<const float4*>(src.kbar + (size_t)old * 64) + ch);
+    if (ch == 0) {
+      dst.origin[a.rest_base + i] = src.origin[a.rest_base + old];
+      dst.kslot[a.rest_base + i] = src.kslot[a.rest_base + old];
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // SCORE.  w[c] = (sequential sum of the pooled rows) / N_pooled; S[j] = balanced
 // tree over the 64 products w[c] * K-bar[j][c] (three levels inside the lane, three
 // by xor-shuffle), Eq. 5-6.  Thread = (token, 8-channel word); block b takes the
@@ -586,6 +779,7 @@ __device__ __forceinline__ void phase_sel1(const MaintArgs& a, Shared& sh) {
   }
 }
 
+template <bool ONCE>
 __device__ __forceinline__ void phase_sel2(const MaintArgs& a, Shared& sh) {
   const int tid = threadIdx.x;
   const int n_runs = (a.r_old + 63) >> 6;
@@ -673,6 +867,11 @@ __device__ __forceinline__ void phase_sel2(const MaintArgs& a, Shared& sh) {
       asm volatile("bar.sync 2, 64;" ::: "memory");
       const unsigned int off = (tid >= 32) ? sh.warp[0] : 0u;
       if (keep) __stcg(&a.kept[base + off + rank], i);
+      if (ONCE && i < a.r_old && !keep) {
+        // the token leaves: its key group loses a member and gives its table slot back when empty
+        const int slot = __ldcg(&a.cur.kslot[a.rest_base + i]);
+        if (atomicSub(&a.ref[slot], 1) == 1) a.ring[atomicAdd(a.push_pos, 1u) % (unsigned int)a.n_slots] = slot;
+      }
     }
     __syncthreads();
   }
@@ -900,7 +1099,7 @@ __device__ __forceinline__ void phase_gather16(const MaintArgs& a) {
 // ---------------------------------------------------------------------------
 // The kernel.
 // ---------------------------------------------------------------------------
-template <int BITS>
+template <int BITS, bool ONCE>
 __global__ void __launch_bounds__(kMT, kBlocksPerSM) maint_kernel(const __grid_constant__ MaintArgs a) {
   __shared__ Shared sh;
   if (threadIdx.x == 0) { sh.abort_flag = 0; sh.acc = 0u; sh.bin = 0u; sh.need = 0u; }
@@ -909,33 +1108,51 @@ __global__ void __launch_bounds__(kMT, kBlocksPerSM) maint_kernel(const __grid_c
   const uint32_t ph = a.phases;
   bool ran = false;                 // something has run since the last barrier
 
-  if (ph & kPhAppend) { phase_append<BITS>(a); ran = true; }
+  if (ph & kPhAppend) {
+    phase_append<BITS, ONCE>(a);
+    if (ONCE) phase_quant_keys_once(a, sh);
+    ran = true;
+  }
   if (ph & kPhPool) { phase_pool(a, sh); ran = true; }
   if (ph & kPhKbar) { phase_kbar<BITS>(a, sh, a.kbar_on_other ? a.oth : a.cur, a.kbar_lo, a.kbar_hi); ran = true; }
 
-  if (ph & kPhScore) {
+  if (ph & (kPhScore | kPhKbarNew)) {
     if (ran && !grid_barrier(a, epoch, sh)) return;
-    phase_score(a, sh);
+    if (ONCE && (ph & kPhKbarNew)) phase_kbar_new_once(a);
+    if (ph & kPhScore) phase_score(a, sh);
     ran = true;
   }
   if (ph & kPhSel) {
     if (ran && !grid_barrier(a, epoch, sh)) return;
     phase_sel1(a, sh);
     if (!grid_barrier(a, epoch, sh)) return;
-    phase_sel2(a, sh);
+    phase_sel2<ONCE>(a, sh);
     ran = true;
   }
   if (ph & kPhPack) {
     if (ran && !grid_barrier(a, epoch, sh)) return;
-    if (BITS == 16 && a.kk > 0) phase_gather16(a);
+    if (ONCE) phase_gather_once(a);
+    else if (BITS == 16 && a.kk > 0) phase_gather16(a);
   }
+}
+
+// Quantise-once mode: the ring of free table slots starts full.
+__global__ void once_init_kernel(int32_t* ring, unsigned int* push_pos, int n_slots) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_slots) ring[i] = i;
+  if (i == 0) *push_pos = (unsigned int)n_slots;
+}
+
+cudaError_t launch_once_init(xkv_cache* c, cudaStream_t st) {
+  once_init_kernel<<<(c->n_slots + 255) / 256, 256, 0, st>>>(c->ring, c->counters + 8, c->n_slots);
+  return cudaGetLastError();
 }
 
 // Grid barriers that a launch with these phases goes through (the same decisions as in the kernel).
 static int maint_barriers(uint32_t ph) {
   int nb = 0;
   bool ran = (ph & (kPhAppend | kPhPool | kPhKbar)) != 0;
-  if (ph & kPhScore) { nb += ran ? 1 : 0; ran = true; }
+  if (ph & (kPhScore | kPhKbarNew)) { nb += ran ? 1 : 0; ran = true; }
   if (ph & kPhSel) { nb += (ran ? 1 : 0) + 1; ran = true; }
   if (ph & kPhPack) nb += ran ? 1 : 0;
   return nb;
@@ -956,7 +1173,8 @@ static cudaError_t maint_grid(int* grid) {
     int sms = 0, per_sm = kBlocksPerSM;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    const void* fns[2] = {(const void*)maint_kernel<4>, (const void*)maint_kernel<16>};
+    const void* fns[3] = {(const void*)maint_kernel<4, false>, (const void*)maint_kernel<16, false>,
+                          (const void*)maint_kernel<4, true>};
     for (const void* fn : fns) {
       int nb = 0;
       e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, kMT, 0);
@@ -994,7 +1212,10 @@ cudaError_t launch_maint(xkv_cache* c, MaintArgs& a, int prof_cat, cudaStream_t 
   if (a.phases & kPhSel) c->sel_parity ^= 1;
   LaunchScope ls(c, prof_cat, st);
   void* params[1] = {(void*)&a};
-  const void* fn = (c->p.kv_bits == 16) ? (const void*)maint_kernel<16> : (const void*)maint_kernel<4>;
+  a.push_pos = c->counters + 8;
+  const void* fn = (c->p.kv_bits == 16) ? (const void*)maint_kernel<16, false>
+                   : c->p.key_mode == XKV_KEYS_ONCE ? (const void*)maint_kernel<4, true>
+                                                    : (const void*)maint_kernel<4, false>;
   if (nb > 0) {
     e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kMT), params, 0, st);
     c->bar_base += (uint32_t)nb * (uint32_t)grid;

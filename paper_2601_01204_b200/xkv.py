@@ -28,6 +28,8 @@ XKV_E_LIMIT = -7
 XKV_E_RANGE = -8
 STATIC_SCRATCH_BYTES = 32 << 20
 BUF_K_CODES, BUF_K_PARAMS, BUF_V_CODES, BUF_V_PARAMS, BUF_ORIGIN, BUF_SCORES, BUF_KEPT, BUF_QVEC = range(8)
+BUF_K_SLOT, BUF_K_TABLE, BUF_K_REF = 8, 9, 10
+KEYS_REGROUP, KEYS_ONCE = 0, 1
 
 EXPORTED = [
     "xkv_workspace_bytes", "xkv_create", "xkv_reset", "xkv_destroy", "kv_append", "kv_score_evict",
@@ -43,13 +45,14 @@ PROF_NAMES = ["append", "score_evict", "pack", "kbar", "maint", "attn", "attn_co
 
 class xkv_params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_heads", "head_dim", "n_special", "pool_g", "quant_group",
-                                         "kv_bits", "budget", "max_frame_tokens")]
+                                         "kv_bits", "budget", "max_frame_tokens", "key_mode", "key_table_slots")]
 
 
 class xkv_info(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("frames", "T", "T_first", "rest_base", "T_phys", "capacity", "cur",
                                          "last_evicted", "last_kept", "last_prunable", "stage", "n_pending")] + \
-               [("launches", C.c_int64), ("workspace_bytes", C.c_uint64)]
+               [("launches", C.c_int64), ("workspace_bytes", C.c_uint64), ("key_table_slots", C.c_int32),
+                ("reserved", C.c_int32)]
 
 
 class xkv_profile(C.Structure):
@@ -147,10 +150,12 @@ class Params:
     kv_bits: int = 4
     budget: int = 2048
     max_frame_tokens: int = 1374
+    key_mode: int = 0          # KEYS_REGROUP or KEYS_ONCE
+    key_table_slots: int = 0   # KEYS_ONCE: 0 = one slot per token slot (never runs out)
 
     def c(self) -> xkv_params:
         return xkv_params(self.n_heads, self.head_dim, self.n_special, self.pool_g, self.quant_group,
-                          self.kv_bits, self.budget, self.max_frame_tokens)
+                          self.kv_bits, self.budget, self.max_frame_tokens, self.key_mode, self.key_table_slots)
 
 
 def xkv_workspace_bytes(p: Params) -> int:
@@ -308,6 +313,18 @@ class Cache:
         kp = self.xkv_debug_export(BUF_K_PARAMS, H * (cap // 64) * 64 * 8).view(np.float32).reshape(H, cap // 64, d, 2)
         vp = self.xkv_debug_export(BUF_V_PARAMS, H * cap * 8).view(np.float32).reshape(H, cap, 2)
         out["k_packed"], out["v_packed"] = k[:, sl].copy(), v[:, sl].copy()
+        if self.p.key_mode == KEYS_ONCE:
+            ns = info.key_table_slots
+            slots = self.xkv_debug_export(BUF_K_SLOT, cap * 4).view(np.int32)[sl]
+            tab = self.xkv_debug_export(BUF_K_TABLE, ns * H * d * 8).view(np.float32).reshape(ns, H, d, 2)
+            ref = self.xkv_debug_export(BUF_K_REF, ns * 4).view(np.int32)
+            out["k_s_tok"] = np.ascontiguousarray(tab[slots, :, :, 0].transpose(1, 0, 2))
+            out["k_z_tok"] = np.ascontiguousarray(tab[slots, :, :, 1].transpose(1, 0, 2))
+            out["k_groups_live"] = int((ref > 0).sum())
+            # bookkeeping of the table: every slot's count is the number of cached tokens that refer to it
+            assert np.array_equal(np.bincount(slots, minlength=ns), ref), "key table reference counts"
+            out["v_s"], out["v_z"] = vp[:, sl, 0].copy(), vp[:, sl, 1].copy()
+            return out
         ngf, ngr = (Tf + 63) // 64, (R + 63) // 64
         out["k_s_first"], out["k_z_first"] = kp[:, :ngf, :, 0].copy(), kp[:, :ngf, :, 1].copy()
         g0 = base // 64

@@ -26,13 +26,13 @@ def xkv():
     return m
 
 
-def _stream(xkv, n, budget, frames, seed, attn_from, bits=4, layer=0, via_stream_step=False):
+def _stream(xkv, n, budget, frames, seed, attn_from, bits=4, layer=0, via_stream_step=False, key_mode=0):
     """One layer's cache against the oracle.  via_stream_step: the frame goes through
     xkv_stream_step (scores and kept indices are read back after the step) instead of the four
     per-layer calls."""
     import torch
     H, d = 16, 64
-    p = xkv.Params(n_heads=H, head_dim=d, budget=budget, max_frame_tokens=n, kv_bits=bits)
+    p = xkv.Params(n_heads=H, head_dim=d, budget=budget, max_frame_tokens=n, kv_bits=bits, key_mode=key_mode)
     cache = xkv.Cache(p)
     ora = xo.OracleLayer(oracle_params(p))
     rng = np.random.default_rng(seed)
@@ -96,6 +96,13 @@ def test_full_stack_layer_1374_tokens_budget_16384(xkv):
 def test_long_stream_layer_1004_tokens_budget_16384(xkv):
     cache, evicting = _stream(xkv, 1004, 16384, 18, seed=4, attn_from=16)
     assert cache.xkv_get_info().T == 16384 and evicting >= 1
+
+
+def test_full_stack_layer_keys_quantised_once(xkv):
+    """The full-stack workload's layer 0 with XKV_KEYS_ONCE, through xkv_stream_step."""
+    cache, evicting = _stream(xkv, 1374, 16384, 15, seed=3, attn_from=12, via_stream_step=True, key_mode=1)
+    info = cache.xkv_get_info()
+    assert info.T == 16384 and evicting >= 3 and info.last_evicted == 1374
 
 
 def test_full_stack_last_layer_through_stream_step(xkv):

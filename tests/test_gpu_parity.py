@@ -376,3 +376,73 @@ def test_unquantised_tail_on_16bit_cache_is_the_packed_result(xkv):
     with pytest.raises(xkv.XkvError):
         cache.attn_packed_causal_tail(q[:, :100], k[:, :100], v[:, :100], o[:, :100])
     cache.attn_packed_causal_tail(q, k, v)
+
+
+# ------------------------------------------------------------------ keys quantised once
+@pytest.mark.parametrize("impl", [0, 1])
+def test_tiny_stream_keys_quantised_once(xkv, impl):
+    """XKV_KEYS_ONCE on the tiny workload: a frame's keys are quantised on arrival in groups of 64 of
+    its tokens, survivors keep codes and group parameters.  Codes, per-token parameters (through the
+    table), the number of live groups, scores, kept indices: bit-exact; attention in tolerance."""
+    p = xkv.Params(budget=1024, max_frame_tokens=261, kv_bits=4, key_mode=xkv.KEYS_ONCE)
+    cache, ora, worst = run_stream(xkv, p, 261, 9, seed=1, impl=impl)
+    info = cache.xkv_get_info()
+    assert info.T == 1024 and info.last_evicted == 261 and info.key_table_slots == info.capacity
+    print("tiny once impl", impl, "worst (max-abs, rel-L2)", worst)
+
+
+def test_keys_quantised_once_ragged_tail_and_block_cap(xkv):
+    """Ragged frame sizes (partial arrival groups, single-token frames), few heads, the unquantised
+    tail reading, token-major tensors, and a capped attention grid, all with XKV_KEYS_ONCE."""
+    p = xkv.Params(n_heads=3, budget=500, max_frame_tokens=150, kv_bits=4, pool_g=7, n_special=2, key_mode=xkv.KEYS_ONCE)
+    run_stream(xkv, p, [129, 64, 150, 5, 77, 150, 33, 128, 150, 1, 150], 11, seed=5)
+    run_stream(xkv, p, [129, 64, 150, 5, 77, 150, 33, 128], 8, seed=6, tail=True)
+    p = xkv.Params(budget=700, max_frame_tokens=261, key_mode=xkv.KEYS_ONCE)
+    run_stream(xkv, p, 261, 5, seed=7, token_major=True, max_blocks=7)
+    p = xkv.Params(n_heads=2, budget=100, max_frame_tokens=64, key_mode=xkv.KEYS_ONCE)      # k = 0: first + current only
+    run_stream(xkv, p, 64, 4, seed=8)
+
+
+def test_keys_quantised_once_stream_step_and_reset(xkv):
+    """xkv_stream_step (one maintenance launch per layer) against the per-call sequence, bit for bit,
+    with XKV_KEYS_ONCE; then both again after xkv_reset (the table's free ring is rebuilt)."""
+    import torch
+    L, H, n, d = 2, 4, 150, 64
+    p = xkv.Params(n_heads=H, budget=400, max_frame_tokens=n, kv_bits=4, key_mode=xkv.KEYS_ONCE)
+    step_caches = [xkv.Cache(p) for _ in range(L)]
+    call_caches = [xkv.Cache(p) for _ in range(L)]
+    for rnd in range(2):
+        for t in range(7):
+            frames = [synth.gen_frame(61 + rnd, l, t, H, n, d) for l in range(L)]
+            q, k, v = ([to_device_bf16(f[i]) for f in frames] for i in range(3))
+            out = [torch.empty_like(x) for x in q]
+            xkv.xkv_stream_step(step_caches, q, k, v, out)
+            for l, c in enumerate(call_caches):
+                c.kv_append(k[l], v[l]); c.kv_score_evict(q[l]); c.kv_quant_pack()
+                ref = c.attn_packed_causal(q[l])
+                torch.cuda.synchronize()
+                assert torch.equal(out[l].view(torch.int16), ref.view(torch.int16)), (rnd, t, l)
+                ea, eb = step_caches[l].export(), c.export()
+                assert all(np.array_equal(np.asarray(ea[key]), np.asarray(eb[key])) for key in eb), (rnd, t, l)
+                assert step_caches[l].xkv_poll_status() == 0 and c.xkv_poll_status() == 0
+        assert step_caches[0].xkv_get_info().last_evicted > 0
+        for c in step_caches + call_caches:
+            c.xkv_reset()
+
+
+def test_key_table_too_small_is_reported(xkv):
+    """A parameter table sized below the worst case can run out (every survivor of an old frame may
+    be the last of its group): the status word then reads XKV_E_LIMIT instead of anything silent."""
+    H, n, d = 2, 64, 64
+    p = xkv.Params(n_heads=H, budget=640, max_frame_tokens=n, kv_bits=4, key_mode=xkv.KEYS_ONCE, key_table_slots=3)
+    cache = xkv.Cache(p)
+    assert cache.xkv_get_info().key_table_slots == 3          # two frames' groups + 1 is the least the library accepts
+    status = 0
+    for t in range(6):                                         # no eviction before frame 10: a fourth live group appears at t = 3
+        q, k, v = (to_device_bf16(x) for x in synth.gen_frame(71, 0, t, H, n, d))
+        cache.step(q, k, v)
+        status = cache.xkv_poll_status()
+        if status:
+            break
+    assert status == xkv.XKV_E_LIMIT and t == 3
+    assert xkv.lib.xkv_create is not None

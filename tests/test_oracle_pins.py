@@ -145,6 +145,15 @@ def test_pooled_query_shapes_and_partial_group():
     np.testing.assert_allclose(xo.pooled_query_canonical(Q, nsp, g), Qbar, rtol=1e-5, atol=1e-6)
 
 
+def test_pooled_query_of_a_frame_shorter_than_the_special_tokens():
+    """Fewer tokens than special tokens: every token is a special token (literal and canonical agree)."""
+    Q = _rng(40).standard_normal((3, 2, 4)).astype(F32)
+    lit = xo.pooled_query_literal(Q, 5, 16)
+    assert lit.shape == (2, 4) == (xo.n_pooled(2, 5, 16), 4)
+    np.testing.assert_allclose(lit, Q.astype(np.float64).mean(0))
+    np.testing.assert_allclose(xo.pooled_query_canonical(Q, 5, 16), lit, rtol=1e-6, atol=1e-7)
+
+
 def test_score_canonical_matches_literal():
     rng = _rng(6)
     H, n, d, Tp = 16, 261, 64, 300

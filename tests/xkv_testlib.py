@@ -23,7 +23,8 @@ def bf16_tensor_to_f32(t) -> np.ndarray:
 
 def oracle_params(p) -> xo.OracleParams:
     return xo.OracleParams(n_heads=p.n_heads, head_dim=p.head_dim, n_special=p.n_special, pool_g=p.pool_g,
-                           quant_group=p.quant_group, kv_bits=p.kv_bits, budget=p.budget)
+                           quant_group=p.quant_group, kv_bits=p.kv_bits, budget=p.budget,
+                           key_mode="once" if getattr(p, "key_mode", 0) == 1 else "regroup")
 
 
 def compare_state(gpu: dict, ora: dict, tag: str = "") -> None:

@@ -459,11 +459,11 @@ int run_layer(HostStepPipe* pipe, xkv_cache* c, const void* q, const void* k, co
   const bool once = keys_once(c);
   a.phases = kPhAppend;
   if ((c->p.kv_bits == 16 && c->kk_pending > 0) || (once && (c->kk_pending > 0 || c->rold_pending > 0))) a.phases |= kPhPack;
-  if (once && !plan.first) a.phases |= kPhKbarNew;
   if (selecting(c)) {
     a.phases |= kPhPool | kPhScore | kPhSel;
     if (once) {
-      // the head means travel with the tokens: nothing to wait for, nothing to recompute
+      // the head means travel with the tokens; those of the frame before were computed beside its attention
+      if (c->kbar_frames == c->frames && cudaStreamWaitEvent(st, c->kbar_done, 0) != cudaSuccess) return XKV_E_CUDA;
     } else if (kbar_fresh(c)) {
       if (cudaStreamWaitEvent(st, c->kbar_done, 0) != cudaSuccess) return XKV_E_CUDA;
     } else {
@@ -480,6 +480,17 @@ int run_layer(HostStepPipe* pipe, xkv_cache* c, const void* q, const void* k, co
   if (c->p.kv_bits == 4 && !once && launch_regroup(c, a, st) != cudaSuccess) return XKV_E_CUDA;
   note_packed(c);
   c->stage = 3;
+  if (once && !plan.first) {
+    // head means (Eq. 4) of the frame just quantised: needed by the next frame's scoring only, so
+    // they are computed on the side stream, beside the attention
+    bool ok = cudaEventRecord(pipe->fork, st) == cudaSuccess && cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess;
+    if (!ok) return XKV_E_CUDA;
+    a.phases = kPhKbarNew;
+    const bool launched = launch_maint(c, a, XKV_PROF_KBAR, pipe->side) == cudaSuccess;
+    ok = cudaEventRecord(c->kbar_done, pipe->side) == cudaSuccess;
+    if (!launched || !ok) return XKV_E_CUDA;
+    c->kbar_T = c->T; c->kbar_cur = c->cur; c->kbar_frames = c->frames;
+  }
   if (!once && c->T > c->T_first) {
     bool ok = cudaEventRecord(pipe->fork, st) == cudaSuccess && cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess;
     if (!ok) return XKV_E_CUDA;

@@ -369,17 +369,19 @@ __device__ __forceinline__ void phase_pool(const MaintArgs& a, Shared& sh) {
 // sixteen heads (4-bit; four 16-byte pieces for 16-bit storage) are fetched ahead
 // of their (ordered) use.
 // ---------------------------------------------------------------------------
+// One run of up to 64 consecutive slots whose keys share their quantisation parameters:
+// slot0 = physical slot of the run's first token, i0 = its rest-local position, `count` tokens;
+// the parameters of (head h, channel ch) are par[h * par_stride + ch].
 template <int BITS>
-__device__ __forceinline__ void phase_kbar(const MaintArgs& a, Shared& sh, const BufSet& b, int lo, int hi) {
+__device__ __forceinline__ void kbar_run(const MaintArgs& a, Shared& sh, const BufSet& b, const float2* par,
+                                         size_t par_stride, int slot0, int i0, int count) {
   const int tid = threadIdx.x;
   const int w = tid & 7;
   const int tok = tid >> 3;
-  const int g_lo = lo >> 6, g_hi = (hi + 63) >> 6;
   const int H = a.H, cap = a.cap;
-  for (int gb = g_lo + blockIdx.x; gb < g_hi; gb += gridDim.x) {
-    const int i = gb * 64 + tok;                  // rest-local index
-    const int slot = a.rest_base + i;
-    const int grp = (a.rest_base >> 6) + gb;
+  {
+    const int i = i0 + tok;                       // rest-local index
+    const int slot = slot0 + tok;
     bool plain = false;
     if (BITS == 4) {
       // Parameters of the key group.  Fast path: float4 [H][4][8] = (s, magic + z) of channels
@@ -387,12 +389,12 @@ __device__ __forceinline__ void phase_kbar(const MaintArgs& a, Shared& sh, const
       // consecutive 16-byte chunks.  Plain path: float2 (s, z) [H][64].
       int big = a.force_plain;
       for (int e = tid; e < H * 64; e += kMT) {
-        const float2 sz = __ldcg(&b.kpar[((size_t)(e >> 6) * (cap >> 6) + grp) * 64 + (e & 63)]);
+        const float2 sz = __ldcg(&par[(size_t)(e >> 6) * par_stride + (e & 63)]);
         big |= !(fabsf(sz.y) < kZLimit);
       }
       plain = __syncthreads_or(big) != 0;
       for (int e = tid; e < H * 64; e += kMT) {
-        float2 sz = __ldcg(&b.kpar[((size_t)(e >> 6) * (cap >> 6) + grp) * 64 + (e & 63)]);
+        float2 sz = __ldcg(&par[(size_t)(e >> 6) * par_stride + (e & 63)]);
         if (plain) {
           sh.u.kbar.par[e] = sz;
         } else {
@@ -403,7 +405,7 @@ __device__ __forceinline__ void phase_kbar(const MaintArgs& a, Shared& sh, const
       }
       __syncthreads();
     }
-    const bool valid = i >= lo && i < hi;
+    const bool valid = tok < count;
     float acc[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = 0.f;
@@ -455,7 +457,19 @@ __device__ __forceinline__ void phase_kbar(const MaintArgs& a, Shared& sh, const
       __stcg(dst + 1, make_float4(__fmul_rn(acc[4], inv_h), __fmul_rn(acc[5], inv_h), __fmul_rn(acc[6], inv_h),
                                   __fmul_rn(acc[7], inv_h)));
     }
-    __syncthreads();       // the parameter table is rewritten by the next pass
+    __syncthreads();       // the parameter table is rewritten by the next run
+  }
+}
+
+// KBAR over the rest-local positions [0, hi) of the buffer set `b` (re-quantising mode and 16-bit):
+// one run per 64-slot key group (the rest segment starts on a 128-slot boundary).
+template <int BITS>
+__device__ __forceinline__ void phase_kbar(const MaintArgs& a, Shared& sh, const BufSet& b, int lo, int hi) {
+  const int g_lo = lo >> 6, g_hi = (hi + 63) >> 6;
+  for (int gb = g_lo + blockIdx.x; gb < g_hi; gb += gridDim.x) {
+    const int grp = (a.rest_base >> 6) + gb;
+    kbar_run<BITS>(a, sh, b, b.kpar + (size_t)grp * 64, (size_t)(a.cap >> 6) * 64, a.rest_base + gb * 64, gb * 64,
+                   min(64, hi - gb * 64));
   }
 }
 
@@ -574,34 +588,14 @@ __device__ __forceinline__ void phase_quant_keys_once(const MaintArgs& a, Shared
 }
 
 // Quantise-once mode: head means (Eq. 4) of the frame just quantised, into the destination's
-// array.  Thread = (token, 8-channel word), heads in order, plain Eq. 10.
-__device__ __forceinline__ void phase_kbar_new_once(const MaintArgs& a) {
-  const int tid = threadIdx.x, w = tid & 7, tok = tid >> 3;
+// array: one run per arrival group, whose parameters sit in the group's table slot.
+__device__ __forceinline__ void phase_kbar_new_once(const MaintArgs& a, Shared& sh) {
   const int n_groups = (a.n + 63) >> 6;
   const BufSet& d = a.oth;
   for (int gamma = blockIdx.x; gamma < n_groups; gamma += gridDim.x) {
-    const int tix = gamma * 64 + tok;
-    if (tix >= a.n) continue;
-    const int slot = __ldcg(&d.kslot[a.dst_slot + tix]);
-    float acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-    for (int h = 0; h < a.H; ++h) {
-      const uint32_t word = __ldcg(reinterpret_cast<const uint32_t*>(d.k + ((size_t)h * a.cap + a.dst_slot + tix) * 32 + 4 * w));
-      const float4* pp = reinterpret_cast<const float4*>(a.ktab32 + ((size_t)slot * a.H + h) * 64 + 8 * w);
-#pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        const float4 p4 = __ldcg(pp + v);
-        const float x0 = __fmul_rn(p4.x, __fsub_rn((float)((word >> nib_shift(2 * v)) & 0xFu), p4.y));
-        const float x1 = __fmul_rn(p4.z, __fsub_rn((float)((word >> nib_shift(2 * v + 1)) & 0xFu), p4.w));
-        acc[2 * v] = (h == 0) ? x0 : __fadd_rn(acc[2 * v], x0);
-        acc[2 * v + 1] = (h == 0) ? x1 : __fadd_rn(acc[2 * v + 1], x1);
-      }
-    }
-    const float inv_h = __fdiv_rn(1.f, (float)a.H);
-    float4* dst = reinterpret_cast<float4*>(d.kbar + (size_t)(a.dst_slot - a.rest_base + tix) * 64 + 8 * w);
-    __stcg(dst, make_float4(__fmul_rn(acc[0], inv_h), __fmul_rn(acc[1], inv_h), __fmul_rn(acc[2], inv_h), __fmul_rn(acc[3], inv_h)));
-    __stcg(dst + 1, make_float4(__fmul_rn(acc[4], inv_h), __fmul_rn(acc[5], inv_h), __fmul_rn(acc[6], inv_h), __fmul_rn(acc[7], inv_h)));
+    const int slot = __ldcg(&d.kslot[a.dst_slot + gamma * 64]);
+    kbar_run<4>(a, sh, d, a.ktab32 + (size_t)slot * a.H * 64, 64, a.dst_slot + gamma * 64,
+                a.dst_slot - a.rest_base + gamma * 64, min(64, a.n - gamma * 64));
   }
 }
 
@@ -622,31 +616,62 @@ __device__ __forceinline__ void phase_gather_once(const MaintArgs& a) {
     }
     return;
   }
+  // four items per thread and pass: the kept indices, then the rows, then the stores
   const long long items = (long long)a.H * a.kk * 4;                 // (head, survivor, 16-byte chunk of K | V codes)
-  for (long long g = first; g < items; g += stride) {
-    const int ch = (int)(g & 3);
-    const long long r = g >> 2;
-    const int i = (int)(r % a.kk);
-    const int h = (int)(r / a.kk);
-    const int old = kept ? __ldcg(&kept[i]) : i;
-    const size_t s = (size_t)h * a.cap + a.rest_base + old;
-    const size_t d = (size_t)h * a.cap + a.rest_base + i;
-    if (ch < 2) {
-      *reinterpret_cast<uint4*>(dst.k + d * 32 + 16 * ch) = *reinterpret_cast<const uint4*>(src.k + s * 32 + 16 * ch);
-    } else {
-      *reinterpret_cast<uint4*>(dst.v + d * 32 + 16 * (ch - 2)) = *reinterpret_cast<const uint4*>(src.v + s * 32 + 16 * (ch - 2));
-      if (ch == 2) dst.vpar[d] = src.vpar[s];
+  for (long long g0 = first; g0 < items; g0 += 4 * stride) {
+    int old[4]; size_t so[4], dd[4]; int chn[4]; bool ok[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const long long g = g0 + u * stride;
+      ok[u] = g < items;
+      chn[u] = (int)(g & 3);
+      const long long r = ok[u] ? (g >> 2) : 0;
+      const int i = (int)(r % a.kk), h = (int)(r / a.kk);
+      old[u] = kept ? __ldcg(&kept[i]) : i;
+      dd[u] = (size_t)h * a.cap + a.rest_base + i;
+      so[u] = (size_t)h * a.cap + a.rest_base;
+    }
+    uint4 row[4]; float2 vp[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const size_t s = so[u] + old[u];
+      const uint8_t* base = chn[u] < 2 ? src.k : src.v;
+      row[u] = ok[u] ? *reinterpret_cast<const uint4*>(base + s * 32 + 16 * (chn[u] & 1)) : make_uint4(0, 0, 0, 0);
+      vp[u] = (ok[u] && chn[u] == 2) ? src.vpar[s] : make_float2(0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (!ok[u]) continue;
+      uint8_t* base = chn[u] < 2 ? dst.k : dst.v;
+      *reinterpret_cast<uint4*>(base + dd[u] * 32 + 16 * (chn[u] & 1)) = row[u];
+      if (chn[u] == 2) dst.vpar[dd[u]] = vp[u];
     }
   }
   const long long rows = (long long)a.kk * 16;                       // (survivor, 16-byte chunk of its head-mean row)
-  for (long long g = first; g < rows; g += stride) {
-    const int ch = (int)(g & 15);
-    const int i = (int)(g >> 4);
-    const int old = kept ? __ldcg(&kept[i]) : i;
-    reinterpret_cast<float4*>(dst.kbar + (size_t)i * 64)[ch] = __ldcg(reinterpret_cast<const float4*>(src.kbar + (size_t)old * 64) + ch);
-    if (ch == 0) {
-      dst.origin[a.rest_base + i] = src.origin[a.rest_base + old];
-      dst.kslot[a.rest_base + i] = src.kslot[a.rest_base + old];
+  for (long long g0 = first; g0 < rows; g0 += 4 * stride) {
+    int old[4]; bool ok[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const long long g = g0 + u * stride;
+      ok[u] = g < rows;
+      old[u] = ok[u] ? (kept ? __ldcg(&kept[(int)(g >> 4)]) : (int)(g >> 4)) : 0;
+    }
+    float4 row[4]; int org[4], ks[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const long long g = g0 + u * stride;
+      const int ch = (int)(g & 15);
+      row[u] = ok[u] ? __ldcg(reinterpret_cast<const float4*>(src.kbar + (size_t)old[u] * 64) + ch) : make_float4(0, 0, 0, 0);
+      org[u] = (ok[u] && ch == 0) ? src.origin[a.rest_base + old[u]] : 0;
+      ks[u] = (ok[u] && ch == 0) ? src.kslot[a.rest_base + old[u]] : 0;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const long long g = g0 + u * stride;
+      if (!ok[u]) continue;
+      const int ch = (int)(g & 15), i = (int)(g >> 4);
+      reinterpret_cast<float4*>(dst.kbar + (size_t)i * 64)[ch] = row[u];
+      if (ch == 0) { dst.origin[a.rest_base + i] = org[u]; dst.kslot[a.rest_base + i] = ks[u]; }
     }
   }
 }
@@ -1118,7 +1143,7 @@ __global__ void __launch_bounds__(kMT, kBlocksPerSM) maint_kernel(const __grid_c
 
   if (ph & (kPhScore | kPhKbarNew)) {
     if (ran && !grid_barrier(a, epoch, sh)) return;
-    if (ONCE && (ph & kPhKbarNew)) phase_kbar_new_once(a);
+    if (ONCE && (ph & kPhKbarNew)) phase_kbar_new_once(a, sh);
     if (ph & kPhScore) phase_score(a, sh);
     ran = true;
   }

@@ -108,7 +108,7 @@ typedef struct {
   int64_t launches;          /* kernels launched for this cache so far                   */
   uint64_t workspace_bytes;
   int32_t key_table_slots;   /* XKV_KEYS_ONCE: slots of the key parameter table, else 0  */
-  int32_t reserved;
+  int32_t budget;            /* the token budget in force (xkv_set_budget)               */
 } xkv_info;
 
 /* Sub-buffers that xkv_debug_export can copy out (physical layout, current
@@ -263,6 +263,33 @@ XKV_API int attn_packed_causal_tail(xkv_cache* cache, const void* q, const void*
 XKV_API int attn_packed_causal_static(xkv_cache* cache, const void* q, void* out, int32_t n,
                               int64_t tok_stride, int64_t head_stride, float softmax_scale,
                               xkv_stream stream);
+
+/* Steps 2-3 with the pooled query supplied by the caller.  Eq. 5-6 average the rows of Q-bar K-bar^T,
+ * which by linearity is w . K-bar[j] with w the mean of the pooled rows of Eq. 2-3: whoever
+ * produces Q (the projection that writes it) can form w on the way (Sec. 3.2 notes that pooling is
+ * what keeps the scoring cheap) and hand it over.  w: DEVICE, 64 floats, exactly the value
+ * kv_score_evict would compute (fixed-order fp32: per head and pooled row the sequential sum over the
+ * row's tokens divided by their number; heads added in order, times 1/H; rows added in order,
+ * divided by their number).  n is the frame's token count.  State and errors as kv_score_evict. */
+XKV_API int kv_score_evict_w(xkv_cache* cache, const float* w, int32_t n, xkv_stream stream);
+
+/* The token budget L_max in force from the next frame on, 1 <= budget <= the budget the cache was
+ * created with (which sized the workspace).  A lower budget makes the next evicting step keep
+ * k = max(0, budget - T_first - n) middle tokens by the same rule; raising it again lets the cache
+ * grow back.  The paper names per-layer adaptive budgets as future work (Conclusion); this call
+ * and xkv_read_score_stats are the mechanism, the policy is the caller's.  Idle cache only. */
+XKV_API int xkv_set_budget(xkv_cache* cache, int32_t budget);
+
+/* Statistics of the last evicting step's scores S (Eq. 6), for such a policy.  Synchronises
+ * `stream`.  sum and sum_sq are accumulated with floating-point atomics (last digits may differ
+ * between runs); threshold is the smallest kept score, exact. */
+typedef struct {
+  int32_t count;        /* scored (middle) tokens; 0 if no step has evicted since the reset */
+  int32_t kept;         /* how many of them were kept                                        */
+  float   sum, sum_sq;  /* sum of S and of S^2                                               */
+  float   threshold;    /* the k-th largest score                                            */
+} xkv_score_stats;
+XKV_API int xkv_read_score_stats(const xkv_cache* cache, xkv_score_stats* out, xkv_stream stream);
 
 /* Chooses the attention that xkv_stream_step and xkv_stream_step_host run for this
  * cache: 0 (default) attn_packed_causal, 1 attn_packed_causal_tail with the K, V

@@ -358,6 +358,7 @@ class OracleLayer:
     def __init__(self, p: OracleParams):
         self.p = p
         H, d = p.n_heads, p.head_dim
+        self.budget = p.budget                         # L_max in force (set_budget may lower or restore it)
         self.frames = 0
         self.T_first = 0
         # quantised cache, logical order.  bits == 16: k_val/v_val hold fp32 copies of bf16.
@@ -437,9 +438,17 @@ class OracleLayer:
         self.last_scores = None
         self.last_kept_mid = None
 
+    def set_budget(self, budget: int) -> None:
+        """Token budget L_max used from the next frame on (per-layer adaptive budgets are the
+        paper's stated future work; this is only the mechanism).  At most the budget the layer was
+        created with."""
+        assert self._new_k is None and 1 <= budget <= self.p.budget
+        self.budget = int(budget)
+
     # ---- steps 2-3: score and evict ---------------------------------------
-    def score_evict(self, Q: np.ndarray) -> None:
-        """Decide which middle tokens survive (Sec. 3.2).  Q [H][n][d]."""
+    def score_evict(self, Q: np.ndarray | None, w: np.ndarray | None = None) -> None:
+        """Decide which middle tokens survive (Sec. 3.2).  Q [H][n][d]; or, with Q = None, the
+        row mean w [d] of the pooled query (Eq. 2-3, fp32) as computed by whoever produced Q."""
         p = self.p
         assert self._new_k is not None
         n = self._new_k.shape[1]
@@ -448,14 +457,16 @@ class OracleLayer:
             self._kept_rest = np.zeros(0, dtype=np.int64)
             return
         T = self.origin.shape[0] + n                   # cache length after the append
-        if T <= p.budget:                              # trigger: only when T > L_max
+        if T <= self.budget:                           # trigger: only when T > L_max
             self._kept_rest = np.arange(R_old, dtype=np.int64)
             return
-        k = max(0, p.budget - self.T_first - n)
+        k = max(0, self.budget - self.T_first - n)
         # the middle segment is exactly the old rest segment (first | middle | current)
         K_mid = self.keys_dequantized()[:, self.T_first:, :]
-        Qbar = pooled_query_canonical(Q, p.n_special, p.pool_g)
-        w = query_vector_canonical(Qbar)
+        if w is None:
+            Qbar = pooled_query_canonical(Q, p.n_special, p.pool_g)
+            w = query_vector_canonical(Qbar)
+        w = np.ascontiguousarray(w, dtype=F32)
         S = score_canonical(w, K_mid)
         kept = select_topk(S, k)
         self.last_w, self.last_scores, self.last_kept_mid = w, S, kept

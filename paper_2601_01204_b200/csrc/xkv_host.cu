@@ -104,6 +104,8 @@ void reset_host_state(xkv_cache* c) {
   c->kbar_T = c->kbar_cur = c->kbar_frames = -1;
   c->bar_base = 0;
   c->sel_parity = 0;
+  c->stats_parity = -1;
+  c->budget_now = c->p.budget;
   c->pop_base = 0;
 }
 
@@ -211,8 +213,8 @@ int plan_frame(const xkv_cache* c, int n, FramePlan* p) {
   p->r_old = p->kk = p->evict = p->dst_slot = 0;
   if (!p->first) {
     p->r_old = c->T - c->T_first;
-    p->evict = (c->T + n > c->p.budget) ? 1 : 0;               // pruning is triggered when T > L_max
-    p->kk = p->evict ? (c->p.budget - c->T_first - n) : p->r_old;   // k = max(0, L_max - T_first - T_current)
+    p->evict = (c->T + n > c->budget_now) ? 1 : 0;             // pruning is triggered when T > L_max
+    p->kk = p->evict ? (c->budget_now - c->T_first - n) : p->r_old;   // k = max(0, L_max - T_first - T_current)
     if (p->kk < 0) p->kk = 0;
     p->dst_slot = c->rest_base + p->kk;
     if (p->dst_slot + n > c->cap) return XKV_E_NOMEM;
@@ -327,6 +329,46 @@ int kv_score_evict(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t h
     if (!keys_once(c)) { c->kbar_T = c->T; c->kbar_cur = c->cur; c->kbar_frames = c->frames; }
   }
   c->stage = 2;
+  return XKV_OK;
+}
+
+int kv_score_evict_w(xkv_cache* c, const float* w, int32_t n, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  if (c->stage != 1) return XKV_E_STATE;
+  if (n != c->n_pending || !aligned16(w)) return XKV_E_INVALID;
+  note_scored(c);
+  if (selecting(c)) {
+    MaintArgs a;
+    maint_args(c, &a);
+    a.phases = kPhScore | kPhSel;
+    if (!keys_once(c) && !kbar_fresh(c)) {
+      a.phases |= kPhKbar;
+      a.kbar_on_other = 0; a.kbar_lo = 0; a.kbar_hi = c->rold_pending;
+    }
+    a.w_in = w;
+    if (launch_maint(c, a, XKV_PROF_SCORE_EVICT, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
+    if (!keys_once(c)) { c->kbar_T = c->T; c->kbar_cur = c->cur; c->kbar_frames = c->frames; }
+  }
+  c->stage = 2;
+  return XKV_OK;
+}
+
+int xkv_set_budget(xkv_cache* c, int32_t budget) {
+  if (!c || budget < 1 || budget > c->p.budget) return XKV_E_INVALID;
+  if (c->stage != 0) return XKV_E_STATE;
+  c->budget_now = budget;
+  return XKV_OK;
+}
+
+int xkv_read_score_stats(const xkv_cache* c, xkv_score_stats* out, xkv_stream stream) {
+  if (!c || !out) return XKV_E_INVALID;
+  if (cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return XKV_E_CUDA;
+  memset(out, 0, sizeof(*out));
+  if (c->stats_parity < 0) return XKV_OK;
+  float v[4];
+  if (cudaMemcpy(v, c->counters + 16 + 4 * c->stats_parity, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return XKV_E_CUDA;
+  out->count = c->last_prunable; out->kept = c->last_kept;
+  out->sum = v[0]; out->sum_sq = v[1]; out->threshold = v[2];
   return XKV_OK;
 }
 
@@ -622,7 +664,7 @@ int xkv_get_info(const xkv_cache* c, xkv_info* info) {
   info->launches = c->launches;
   info->workspace_bytes = c->ws_bytes;
   info->key_table_slots = c->n_slots;
-  info->reserved = 0;
+  info->budget = c->budget_now;
   return XKV_OK;
 }
 

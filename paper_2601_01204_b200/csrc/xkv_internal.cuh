@@ -46,6 +46,9 @@ struct MaintArgs {
   int kbar_on_other, kbar_lo, kbar_hi;   // KBAR phase: buffer set and rest-local range
   __nv_bfloat16* kstage;
   float* qbar; float* qvec; float* scores;
+  const float* w_in;               // the pooled query's row mean from the caller (no POOL phase), or null
+  float* stats;                    // [4] sum S, sum S^2, k-th largest score, -   of this launch
+  float* stats_next;               // the next selecting launch's (cleared by this one)
   int32_t* kept;
   unsigned int* hist;
   unsigned int* run_hi;            // [cap / 64] sure keeps of every 64-token run
@@ -113,6 +116,8 @@ struct xkv_cache {
   int last_evicted, last_kept, last_prunable;
   long long launches;
   int force_plain;         // 1: kernels take the plain (conversion-based) arithmetic forms everywhere
+  int budget_now;          // the token budget in force (xkv_set_budget), <= p.budget
+  int stats_parity;        // which statistics block the last selecting launch wrote (-1: none)
   int tail_mode;           // 1: the stream-step calls attend with the step's K, V unquantised
   int attn_max_blocks;     // test hook: cap on the thread blocks of the tensor-core attention (0: none)
   // head means of the keys after the first frame (Eq. 4; BufSet::kbar), filled by the stream step

@@ -161,6 +161,7 @@ struct Shared {
   unsigned int acc;
   unsigned int bin, need;          // result of SEL1, used by SEL2
   unsigned int sub, need2, n_list; // SEL2: the sub-bin of the k-th largest key, its rank there, listed candidates
+  float fsum[2];                   // SCORE: block sums of S and S^2
   int abort_flag;
 };
 
@@ -686,9 +687,9 @@ __device__ __forceinline__ void phase_score(const MaintArgs& a, Shared& sh) {
   const int tid = threadIdx.x;
   const int n_runs = (a.r_old + 63) >> 6;
   if ((int)blockIdx.x >= n_runs && blockIdx.x != 0) return;
-  // the pooled rows come through shared memory, 128 at a time (one round trip), and one thread
-  // per channel adds them in order
-  for (int r0 = 0; r0 < a.n_pooled; r0 += kPoolRows) {
+  // the pooled rows come through shared memory, 120 at a time (one round trip), and one thread
+  // per channel adds them in order -- unless the caller supplied the row mean
+  for (int r0 = 0; a.w_in == nullptr && r0 < a.n_pooled; r0 += kPoolRows) {
     const int rows = min(kPoolRows, a.n_pooled - r0);
     __syncthreads();
     for (int e = tid; e < rows * 64; e += kMT) sh.u.score.rows[e] = __ldcg(&a.qbar[r0 * 64 + e]);
@@ -707,7 +708,7 @@ __device__ __forceinline__ void phase_score(const MaintArgs& a, Shared& sh) {
     }
   }
   if (tid < 64) {
-    const float wv = __fdiv_rn(sh.u.score.w[tid], (float)a.n_pooled);
+    const float wv = a.w_in ? a.w_in[tid] : __fdiv_rn(sh.u.score.w[tid], (float)a.n_pooled);
     sh.u.score.w[tid] = wv;
     if (blockIdx.x == 0) a.qvec[tid] = wv;
   }
@@ -736,6 +737,14 @@ __device__ __forceinline__ void phase_score(const MaintArgs& a, Shared& sh) {
       __stcg(&a.scores[i], s);
       atomicAdd(&a.hist[(blockIdx.x & (kHistCopies - 1)) * kSelBins + (order_key(s) >> 20)], 1u);
     }
+    // statistics of the scores (for budget policies): block sums, then one atomic per block
+    float s1 = (valid && w == 0) ? s : 0.f, s2 = s1 * s1;
+#pragma unroll
+    for (int o = 8; o < 32; o <<= 1) { s1 += __shfl_xor_sync(0xffffffffu, s1, o); s2 += __shfl_xor_sync(0xffffffffu, s2, o); }
+    if ((tid & 31) == 0) { atomicAdd(&sh.fsum[0], s1); atomicAdd(&sh.fsum[1], s2); }
+    __syncthreads();
+    if (tid == 0) { atomicAdd(&a.stats[0], sh.fsum[0]); atomicAdd(&a.stats[1], sh.fsum[1]); sh.fsum[0] = sh.fsum[1] = 0.f; }
+    __syncthreads();
   }
 }
 
@@ -754,6 +763,7 @@ __device__ __forceinline__ void phase_sel1(const MaintArgs& a, Shared& sh) {
   if (blockIdx.x == gridDim.x - 1) {                 // the next selecting launch's counter and sub-histogram:
     if (tid == 0) *a.cand_count_next = 0u;           // nobody uses them in this launch
     if (tid < kSubBins) a.hist2_next[tid] = 0u;
+    if (tid < 4) a.stats_next[tid] = 0.f;
   }
   if ((int)blockIdx.x >= n_runs) return;
   // thread t owns the bins 4095 - 8t - 7 .. 4095 - 8t; walked from the top
@@ -868,6 +878,10 @@ __device__ __forceinline__ void phase_sel2(const MaintArgs& a, Shared& sh) {
     }
   }
   const unsigned long long tau = prefix;             // kept candidates: composite >= tau (exactly `need` of them)
+  if (blockIdx.x == 0 && tid == 0) {                 // the k-th largest score itself, for the statistics
+    const uint32_t key = (uint32_t)(tau >> 32);
+    a.stats[2] = __uint_as_float((key & 0x80000000u) ? (key ^ 0x80000000u) : ~key);
+  }
   for (int run = blockIdx.x; run < n_runs; run += gridDim.x) {
     // survivors before this run: the sure keeps of the runs before it plus the kept candidates at
     // lower positions
@@ -1127,7 +1141,7 @@ __device__ __forceinline__ void phase_gather16(const MaintArgs& a) {
 template <int BITS, bool ONCE>
 __global__ void __launch_bounds__(kMT, kBlocksPerSM) maint_kernel(const __grid_constant__ MaintArgs a) {
   __shared__ Shared sh;
-  if (threadIdx.x == 0) { sh.abort_flag = 0; sh.acc = 0u; sh.bin = 0u; sh.need = 0u; }
+  if (threadIdx.x == 0) { sh.abort_flag = 0; sh.acc = 0u; sh.bin = 0u; sh.need = 0u; sh.fsum[0] = sh.fsum[1] = 0.f; }
   __syncthreads();
   uint32_t epoch = 0;
   const uint32_t ph = a.phases;
@@ -1234,6 +1248,9 @@ cudaError_t launch_maint(xkv_cache* c, MaintArgs& a, int prof_cat, cudaStream_t 
   a.cand_count_next = c->counters + 2 + (c->sel_parity ^ 1);
   a.hist2 = c->counters + 64 + 256 * c->sel_parity;
   a.hist2_next = c->counters + 64 + 256 * (c->sel_parity ^ 1);
+  a.stats = reinterpret_cast<float*>(c->counters + 16 + 4 * c->sel_parity);
+  a.stats_next = reinterpret_cast<float*>(c->counters + 16 + 4 * (c->sel_parity ^ 1));
+  if (a.phases & kPhSel) c->stats_parity = c->sel_parity;
   if (a.phases & kPhSel) c->sel_parity ^= 1;
   LaunchScope ls(c, prof_cat, st);
   void* params[1] = {(void*)&a};

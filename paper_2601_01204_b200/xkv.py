@@ -38,7 +38,7 @@ EXPORTED = [
     "xkv_synth_fill", "xkv_profile_enable", "xkv_profile_read", "attn_packed_causal_static",
     "xkv_debug_rewind_attention", "attn_packed_causal_tail", "xkv_set_unquantised_tail",
     "xkv_debug_force_plain", "xkv_debug_limit_attention_blocks", "xkv_debug_timeout_probe",
-    "xkv_debug_head_means",
+    "xkv_debug_head_means", "kv_score_evict_w", "xkv_set_budget", "xkv_read_score_stats",
 ]
 PROF_NAMES = ["append", "score_evict", "pack", "kbar", "maint", "attn", "attn_combine"]
 
@@ -52,7 +52,12 @@ class xkv_info(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("frames", "T", "T_first", "rest_base", "T_phys", "capacity", "cur",
                                          "last_evicted", "last_kept", "last_prunable", "stage", "n_pending")] + \
                [("launches", C.c_int64), ("workspace_bytes", C.c_uint64), ("key_table_slots", C.c_int32),
-                ("reserved", C.c_int32)]
+                ("budget", C.c_int32)]
+
+
+class xkv_score_stats(C.Structure):
+    _fields_ = [("count", C.c_int32), ("kept", C.c_int32), ("sum", C.c_float), ("sum_sq", C.c_float),
+                ("threshold", C.c_float)]
 
 
 class xkv_profile(C.Structure):
@@ -76,6 +81,12 @@ lib.kv_append.restype = C.c_int
 lib.kv_append.argtypes = [_vp, _vp, _vp, _i32, _i64, _i64, _vp]
 lib.kv_score_evict.restype = C.c_int
 lib.kv_score_evict.argtypes = [_vp, _vp, _i32, _i64, _i64, _vp]
+lib.kv_score_evict_w.restype = C.c_int
+lib.kv_score_evict_w.argtypes = [_vp, _vp, _i32, _vp]
+lib.xkv_set_budget.restype = C.c_int
+lib.xkv_set_budget.argtypes = [_vp, _i32]
+lib.xkv_read_score_stats.restype = C.c_int
+lib.xkv_read_score_stats.argtypes = [_vp, C.POINTER(xkv_score_stats), _vp]
 lib.kv_quant_pack.restype = C.c_int
 lib.kv_quant_pack.argtypes = [_vp, _vp]
 lib.attn_packed_causal.restype = C.c_int
@@ -199,6 +210,18 @@ class Cache:
     def kv_score_evict(self, q) -> None:
         ts, hs = _strides(q)
         _check(lib.kv_score_evict(self.handle, q.data_ptr(), q.shape[1], ts, hs, _stream()), "kv_score_evict")
+
+    def kv_score_evict_w(self, w, n: int) -> None:
+        """kv_score_evict with the pooled query's row mean w (device tensor, 64 fp32) from the caller."""
+        _check(lib.kv_score_evict_w(self.handle, w.data_ptr(), n, _stream()), "kv_score_evict_w")
+
+    def xkv_set_budget(self, budget: int) -> None:
+        _check(lib.xkv_set_budget(self.handle, budget), "xkv_set_budget")
+
+    def xkv_read_score_stats(self) -> xkv_score_stats:
+        st = xkv_score_stats()
+        _check(lib.xkv_read_score_stats(self.handle, C.byref(st), _stream()), "xkv_read_score_stats")
+        return st
 
     def kv_quant_pack(self) -> None:
         _check(lib.kv_quant_pack(self.handle, _stream()), "kv_quant_pack")

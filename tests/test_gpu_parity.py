@@ -446,3 +446,51 @@ def test_key_table_too_small_is_reported(xkv):
             break
     assert status == xkv.XKV_E_LIMIT and t == 3
     assert xkv.lib.xkv_create is not None
+
+
+# ------------------------------------------------------------------ budget changes, caller's w
+@pytest.mark.parametrize("key_mode", [0, 1])
+def test_budget_changes_query_vector_from_caller_and_score_statistics(xkv, key_mode):
+    """xkv_set_budget lowers and restores the budget mid-stream (the cache shrinks to it at the next
+    frame, bit-exact against the oracle's set_budget); kv_score_evict_w takes the pooled query's row
+    mean from the caller and gives the state kv_score_evict gives; xkv_read_score_stats returns sum,
+    sum of squares and the k-th largest of the scores S (Eq. 6)."""
+    import torch
+    from xkv_testlib import compare_state, oracle_params, bf16_tensor_to_f32, check_attention
+    from oracle import xkv_oracle as xo
+    H, n, d = 4, 100, 64
+    p = xkv.Params(n_heads=H, budget=700, max_frame_tokens=n, kv_bits=4, key_mode=key_mode)
+    ca, cb = xkv.Cache(p), xkv.Cache(p)
+    ora = xo.OracleLayer(oracle_params(p))
+    assert ca.xkv_read_score_stats().count == 0
+    for t in range(12):
+        if t == 6:
+            for c in (ca, cb): c.xkv_set_budget(380)
+            ora.set_budget(380)
+        if t == 10:
+            for c in (ca, cb): c.xkv_set_budget(700)
+            ora.set_budget(700)
+        qb, kb, vb = synth.gen_frame(81, 0, t, H, n, d)
+        qf, kf, vf = (synth.bf16_bits_to_f32(x) for x in (qb, kb, vb))
+        q, k, v = (to_device_bf16(x) for x in (qb, kb, vb))
+        ca.kv_append(k, v); ca.kv_score_evict(q); ca.kv_quant_pack()
+        ora.append(kf, vf); ora.score_evict(qf); ora.quant_pack()
+        compare_state(ca.export(), ora.export(), f"frame {t}")
+        check_attention(bf16_tensor_to_f32(ca.attn_packed_causal(q)).transpose(1, 0, 2), ora.attend(qf), f"frame {t}")
+        # the second cache gets w from "the producer of Q" (here: the oracle's canonical arithmetic)
+        w = xo.query_vector_canonical(xo.pooled_query_canonical(qf, p.n_special, p.pool_g))
+        cb.kv_append(k, v); cb.kv_score_evict_w(torch.from_numpy(w).cuda(), n); cb.kv_quant_pack()
+        cb.attn_packed_causal(q)
+        ea, eb = ca.export(), cb.export()
+        assert all(np.array_equal(np.asarray(ea[key]), np.asarray(eb[key])) for key in ea), f"frame {t}: given w"
+        if ora.last_scores is not None:
+            st = ca.xkv_read_score_stats()
+            S = ora.last_scores.astype(np.float64)
+            assert st.count == len(S) and st.kept == len(ora.last_kept_mid)
+            assert abs(st.sum - S.sum()) <= 1e-4 * np.abs(S).sum() and abs(st.sum_sq - (S * S).sum()) <= 1e-4 * (S * S).sum()
+            assert np.float32(st.threshold) == np.sort(ora.last_scores)[::-1][st.kept - 1]
+        info = ca.xkv_get_info()
+        assert info.budget == (380 if 6 <= t < 10 else 700) and info.T == ora.T
+    assert ca.xkv_get_info().T == 380 + 2 * n and ca.xkv_poll_status() == 0
+    with pytest.raises(xkv.XkvError):
+        ca.xkv_set_budget(701)

@@ -223,6 +223,38 @@ def pin_regroup_rule_on_crafted_steps(xo):
         assert np.array_equal(L.k_s_rest[:, gi], s) and np.array_equal(L.k_z_rest[:, gi], z), f"B: group {gi} parameters"
 
 
+def pin_budget_change_and_given_query_vector(xo):
+    """The budget in force can be lowered between frames (mechanism for per-layer adaptive budgets,
+    the paper's stated future work): the next step evicts down to it with the same rule (first and
+    current frame whole, top-k of the middle).  And the row mean w of the pooled query (Eq. 2-3) may
+    come from the caller instead of Q: same scores, same survivors."""
+    H, n, d, G = 4, 37, 16, 8
+    p = xo.OracleParams(n_heads=H, head_dim=d, n_special=5, pool_g=4, quant_group=G, kv_bits=4, budget=260)
+    La, Lb = xo.OracleLayer(p), xo.OracleLayer(p)
+    for t in range(9):
+        q, k, v = _frame(29, t, H, n, d)
+        if t == 5:
+            La.set_budget(150); Lb.set_budget(150)
+        if t == 8:
+            La.set_budget(260); Lb.set_budget(260)
+        T_before, Tf = La.T, La.T_first
+        K_before = La.keys_dequantized().copy() if t else None
+        La.step(q, k, v)
+        w = xo_real.query_vector_canonical(xo_real.pooled_query_canonical(q, p.n_special, p.pool_g))
+        Lb.append(k, v); Lb.score_evict(None, w=w); Lb.quant_pack()
+        ea, eb = La.export(), Lb.export()
+        assert all(np.array_equal(ea[key], eb[key]) for key in ea), f"frame {t}: given w"
+        budget = 150 if 5 <= t < 8 else 260
+        assert La.T == min(T_before + n, max(budget, 2 * n if t else n)), f"frame {t}: length {La.T}"
+        assert np.array_equal(La.origin[:n], (1 << 16) | np.arange(n)) and np.array_equal(La.origin[-n:], ((t + 1) << 16) | np.arange(n))
+        if T_before + n > budget:
+            kk = budget - Tf - n
+            S = xo_real.score_literal(q, K_before[:, Tf:T_before], p.n_special, p.pool_g)
+            assert len(La.last_kept_mid) == kk and np.array_equal(La.last_kept_mid, xo_real.select_topk(La.last_scores, kk))
+            assert np.all(np.abs(La.last_scores - S) <= 1e-4 * (np.abs(S) + 1.0))
+    assert La.T == 150 + n                      # the raised budget lets the cache grow again
+
+
 PINS = [
     ("survivors-4bit", lambda xo: pin_survivor_data_follows_origins(xo, 4)),
     ("survivors-8bit", lambda xo: pin_survivor_data_follows_origins(xo, 8, seed=24)),
@@ -231,6 +263,7 @@ PINS = [
     ("once-4bit", lambda xo: pin_survivor_data_follows_origins(xo, 4, seed=26, key_mode="once")),
     ("once-8bit", lambda xo: pin_survivor_data_follows_origins(xo, 8, seed=27, key_mode="once")),
     ("once-no-pruning", pin_quantise_once_without_pruning_is_framewise_quantisation),
+    ("budget-and-given-w", pin_budget_change_and_given_query_vector),
 ]
 
 
@@ -277,8 +310,8 @@ MUTATIONS = [
      "self.origin = np.concatenate([self.origin[keep_abs], frame_origin])",
      "self.origin = np.concatenate([self.origin[:len(keep_abs)], frame_origin])"),
     ("k counted without the first frame",
-     "k = max(0, p.budget - self.T_first - n)",
-     "k = max(0, p.budget - n)"),
+     "k = max(0, self.budget - self.T_first - n)",
+     "k = max(0, self.budget - n)"),
     ("survivors re-quantised from their codes, not their values",
      "old_deq = dequantize_keys(old_codes, self.k_s_rest, self.k_z_rest, G)",
      "old_deq = old_codes.astype(F32)"),
@@ -295,6 +328,9 @@ MUTATIONS = [
      "codes, s, z = quantize_keys(K_new, p.quant_group, p.kv_bits)\n        base",
      "codes, s, z = quantize_keys(np.concatenate([K_new[:, :self.T % p.quant_group], K_new], 1), p.quant_group, p.kv_bits)\n"
      "        codes = codes[:, self.T % p.quant_group:]\n        base"),
+    ("changed budget ignored by the trigger",
+     "if T <= self.budget:                           # trigger",
+     "if T <= p.budget:                           # trigger"),
     ("first frame re-quantised with the rest",
      "self.k_codes = np.concatenate([self.k_codes[:, :Tf], new_codes], axis=1)",
      "self.k_codes = np.concatenate([self.k_codes[:, :Tf] * 0, new_codes], axis=1)"),

@@ -170,7 +170,8 @@ XKV_API int kv_append(xkv_cache* cache, const void* k, const void* v, int32_t n,
  * in groups of g, then averaged over heads), head-averaged dequantised keys of
  * the middle segment, scores S, and the k = max(0, L_max - T_first - n) highest
  * scores kept (ties: lower position wins), in ascending position.  Otherwise a
- * no-op.  q is frame t's query, same n as the append.  Errors: XKV_E_STATE
+ * no-op.  q is frame t's query, same n as the append (after a chunk of frames was appended: the
+ * query and size of the chunk's last frame, see attn_packed_frame_causal).  Errors: XKV_E_STATE
  * unless kv_append was the previous call; XKV_E_INVALID as above. */
 XKV_API int kv_score_evict(xkv_cache* cache, const void* q, int32_t n,
                    int64_t tok_stride, int64_t head_stride, xkv_stream stream);
@@ -263,6 +264,26 @@ XKV_API int attn_packed_causal_tail(xkv_cache* cache, const void* q, const void*
 XKV_API int attn_packed_causal_static(xkv_cache* cache, const void* q, void* out, int32_t n,
                               int64_t tok_stride, int64_t head_stride, float softmax_scale,
                               xkv_stream stream);
+
+/* A chunk of frames at once (offline sequences arrive many frames at a time; Eq. 1 is frame-causal:
+ * a query sees the keys of its own and of earlier frames).  The chunk is one arrival for the cache
+ * maintenance of Sec. 3.2 - it plays the part of the current frame: kv_append takes all its tokens
+ * (n = their total, frames one after the other along the token axis, at most max_frame_tokens),
+ * kv_score_evict takes the query of the chunk's LAST frame (n = that frame's size) and keeps
+ * k = max(0, L_max - T_first - total) middle tokens, kv_quant_pack packs - and then this call
+ * attends frame-causally: the queries of the chunk's frame f see every cached token that is older
+ * than the chunk and the chunk's frames 0..f (the cache keeps arrival order, so that is a prefix
+ * of it; one launch of the tensor-core kernel per frame).  q, out: the chunk's tensors,
+ * [H][total][d] with the given strides; frame_tokens: HOST array of n_frames sizes that add up to
+ * the appended total.  A chunk of one frame is attn_packed_causal.  State and errors as attn_packed_causal. */
+XKV_API int attn_packed_frame_causal(xkv_cache* cache, const void* q, void* out, const int32_t* frame_tokens,
+                             int32_t n_frames, int64_t tok_stride, int64_t head_stride, float softmax_scale,
+                             xkv_stream stream);
+
+/* The four calls above for one chunk, softmax_scale = 1/sqrt(head_dim). */
+XKV_API int xkv_prefill_chunk(xkv_cache* cache, const void* q, const void* k, const void* v, void* out,
+                      const int32_t* frame_tokens, int32_t n_frames, int64_t tok_stride, int64_t head_stride,
+                      xkv_stream stream);
 
 /* Steps 2-3 with the pooled query supplied by the caller.  Eq. 5-6 average the rows of Q-bar K-bar^T,
  * which by linearity is w . K-bar[j] with w the mean of the pooled rows of Eq. 2-3: whoever

@@ -590,6 +590,28 @@ class OracleLayer:
         self.quant_pack()
         return self.attend(Q, scale, full_precision_tail)
 
+    # ---- a chunk of frames at once -----------------------------------------
+    def step_chunk(self, Qs, Ks, Vs, scale: float | None = None):
+        """Several frames arriving together (offline sequences): the chunk is one arrival for the
+        maintenance of Sec. 3.2 -- it plays the part of the current frame, the middle segment is
+        scored with the query of the chunk's last frame -- and its attention is frame-causal
+        (Eq. 1): frame f of the chunk sees everything older than the chunk and the chunk's frames
+        0..f, i.e. a prefix of the cache.  Returns the outputs per frame, each fp32 [n_f][H][d]."""
+        if scale is None:
+            scale = 1.0 / np.sqrt(self.p.head_dim)
+        self.append(np.concatenate(Ks, axis=1), np.concatenate(Vs, axis=1))
+        self.score_evict(Qs[-1])
+        self.quant_pack()
+        K, V = self.keys_dequantized(), self.values_dequantized()
+        total = sum(q.shape[1] for q in Qs)
+        end = self.T - total
+        outs = []
+        for q in Qs:
+            end += q.shape[1]
+            O = attention(q, K[:, :end], V[:, :end], scale)
+            outs.append(np.ascontiguousarray(np.transpose(O, (1, 0, 2))))
+        return outs
+
     # ---- export for bit-exact comparison ----------------------------------
     def export(self) -> dict:
         """Logical-order arrays in the storage formats of the library."""

@@ -1053,7 +1053,7 @@ static cudaError_t attn_device_setup(int* sm_count) {
 
 static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
                                      float scale, float* part, size_t part_bytes, cudaStream_t st,
-                                     const TailArgs* tail = nullptr) {
+                                     const TailArgs* tail = nullptr, int prefix = 0) {
   int sm_count = 0;
   {
     const cudaError_t e = attn_device_setup(&sm_count);
@@ -1068,6 +1068,12 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
   a.cap = c->cap; a.t_first = c->T_first;
   a.t_phys = c->rest_base + (c->T - c->T_first);
   if (c->T == c->T_first) a.t_phys = c->T_first;          // only the first frame: no pad tile beyond it
+  if (prefix > 0 && prefix < c->T) {
+    // a prefix of the cache in logical order: inside the first frame it ends the first segment,
+    // after it the rest segment
+    if (prefix <= c->T_first) { a.t_first = prefix; a.t_phys = prefix; }
+    else a.t_phys = c->rest_base + (prefix - c->T_first);
+  }
   a.scale_log2 = scale * 1.4426950408889634f;
   a.n_tiles = (a.t_phys + 127) / 128;
   a.q_tiles = (n + kQRows - 1) / kQRows;
@@ -1120,8 +1126,8 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
 }
 
 cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs, float scale,
-                           cudaStream_t st) {
-  return launch_attn_tc_on(c, q, out, n, ts, hs, scale, c->attn_part, c->attn_part_bytes, st);
+                           cudaStream_t st, int prefix) {
+  return launch_attn_tc_on(c, q, out, n, ts, hs, scale, c->attn_part, c->attn_part_bytes, st, nullptr, prefix);
 }
 
 cudaError_t launch_attn_tc_tail(xkv_cache* c, const void* q, const void* k_t, const void* v_t, void* out, int n,

@@ -230,13 +230,14 @@ void maint_args(const xkv_cache* c, MaintArgs* a) {
   a->first = c->first_pending;
   a->cur = c->buf[c->cur]; a->oth = c->buf[c->cur ^ 1];
   a->n = c->n_pending;
+  a->n_q = c->nq_pending > 0 ? c->nq_pending : c->n_pending;
   a->rest_base = c->rest_base; a->r_old = c->rold_pending; a->kk = c->kk_pending;
   a->r_new = c->kk_pending + c->n_pending;
   a->dst_slot = c->first_pending ? 0 : c->rest_base + c->kk_pending;
   a->identity = !(c->evict_pending && c->kk_pending > 0 && c->kk_pending < c->rold_pending);
-  a->n_special = c->p.n_special < c->n_pending ? c->p.n_special : c->n_pending;
+  a->n_special = c->p.n_special < a->n_q ? c->p.n_special : a->n_q;
   a->pool_g = c->p.pool_g;
-  a->n_pooled = a->n_special + (c->n_pending - a->n_special + c->p.pool_g - 1) / c->p.pool_g;
+  a->n_pooled = a->n_special + (a->n_q - a->n_special + c->p.pool_g - 1) / c->p.pool_g;
   a->kstage = c->kstage; a->qbar = c->qbar; a->qvec = c->qvec; a->scores = c->scores; a->kept = c->kept;
   a->hist = c->sel_hist; a->run_hi = c->run_hi; a->cand = c->cand;
   a->force_plain = c->force_plain;
@@ -248,6 +249,7 @@ bool keys_once(const xkv_cache* c) { return c->p.key_mode == XKV_KEYS_ONCE; }
 
 void set_pending(xkv_cache* c, int n, const FramePlan& p) {
   c->n_pending = n;
+  c->nq_pending = 0;
   c->kk_pending = p.kk;
   c->rold_pending = p.r_old;
   c->evict_pending = p.evict;
@@ -313,7 +315,9 @@ int kv_append(xkv_cache* c, const void* k, const void* v, int32_t n, int64_t ts,
 int kv_score_evict(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t hs, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;
   if (c->stage != 1) return XKV_E_STATE;
-  if (n != c->n_pending || !aligned16(q) || !strides_ok(ts, hs)) return XKV_E_INVALID;
+  // n is the frame's size; after a chunk of frames was appended, the size of its last frame
+  if (n < 1 || n > c->n_pending || !aligned16(q) || !strides_ok(ts, hs)) return XKV_E_INVALID;
+  c->nq_pending = n;
   note_scored(c);
   if (selecting(c)) {
     MaintArgs a;
@@ -335,7 +339,7 @@ int kv_score_evict(xkv_cache* c, const void* q, int32_t n, int64_t ts, int64_t h
 int kv_score_evict_w(xkv_cache* c, const float* w, int32_t n, xkv_stream stream) {
   if (!c) return XKV_E_INVALID;
   if (c->stage != 1) return XKV_E_STATE;
-  if (n != c->n_pending || !aligned16(w)) return XKV_E_INVALID;
+  if (n < 1 || n > c->n_pending || !aligned16(w)) return XKV_E_INVALID;
   note_scored(c);
   if (selecting(c)) {
     MaintArgs a;
@@ -421,6 +425,52 @@ int attn_packed_causal_tail(xkv_cache* c, const void* q, const void* k_t, const 
   if (e != cudaSuccess) return XKV_E_CUDA;
   c->stage = 0;
   return XKV_OK;
+}
+
+int attn_packed_frame_causal(xkv_cache* c, const void* q, void* out, const int32_t* frame_tokens, int32_t n_frames,
+                             int64_t ts, int64_t hs, float softmax_scale, xkv_stream stream) {
+  if (!c) return XKV_E_INVALID;
+  if (c->stage != 3) return XKV_E_STATE;
+  if (!frame_tokens || n_frames < 1 || !aligned16(q) || !aligned16(out) || !strides_ok(ts, hs) || !(softmax_scale > 0.f))
+    return XKV_E_INVALID;
+  long long total = 0;
+  for (int f = 0; f < n_frames; ++f) {
+    if (frame_tokens[f] < 1) return XKV_E_INVALID;
+    total += frame_tokens[f];
+  }
+  if (total != c->n_pending) return XKV_E_INVALID;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int before = c->T - c->n_pending;              // cached tokens older than the chunk
+  int r0 = 0;
+  for (int f = 0; f < n_frames; ++f) {
+    const int nf = frame_tokens[f];
+    const __nv_bfloat16* qf = reinterpret_cast<const __nv_bfloat16*>(q) + (int64_t)r0 * ts;
+    __nv_bfloat16* of = reinterpret_cast<__nv_bfloat16*>(out) + (int64_t)r0 * ts;
+    // (strides are multiples of 8 elements, so every frame's first row is 16-byte aligned)
+    const cudaError_t e = launch_attn_tc(c, qf, of, nf, ts, hs, softmax_scale, st, before + r0 + nf);
+    if (e == cudaErrorNotSupported) return XKV_E_UNSUPPORTED;
+    if (e != cudaSuccess) return XKV_E_CUDA;
+    r0 += nf;
+  }
+  c->stage = 0;
+  return XKV_OK;
+}
+
+int xkv_prefill_chunk(xkv_cache* c, const void* q, const void* k, const void* v, void* out,
+                      const int32_t* frame_tokens, int32_t n_frames, int64_t ts, int64_t hs, xkv_stream stream) {
+  if (!c || !frame_tokens || n_frames < 1) return XKV_E_INVALID;
+  long long total = 0;
+  for (int f = 0; f < n_frames; ++f) { if (frame_tokens[f] < 1) return XKV_E_INVALID; total += frame_tokens[f]; }
+  if (total > c->p.max_frame_tokens) return XKV_E_INVALID;
+  const int n = (int)total, n_last = frame_tokens[n_frames - 1];
+  int rc = kv_append(c, k, v, n, ts, hs, stream);
+  if (rc != XKV_OK) return rc;
+  const __nv_bfloat16* q_last = reinterpret_cast<const __nv_bfloat16*>(q) + (int64_t)(n - n_last) * ts;
+  rc = kv_score_evict(c, q_last, n_last, ts, hs, stream);
+  if (rc != XKV_OK) return rc;
+  rc = kv_quant_pack(c, stream);
+  if (rc != XKV_OK) return rc;
+  return attn_packed_frame_causal(c, q, out, frame_tokens, n_frames, ts, hs, 1.0f / sqrtf((float)c->p.head_dim), stream);
 }
 
 int xkv_set_unquantised_tail(xkv_cache* c, int32_t on) {

@@ -35,7 +35,8 @@ struct MaintArgs {
   uint32_t phases;
   // the frame
   const __nv_bfloat16* q; const __nv_bfloat16* k; const __nv_bfloat16* v;
-  int n;
+  int n;                           // tokens that arrive (one frame, or a chunk of frames)
+  int n_q;                         // tokens of the scoring query (the frame; of a chunk, its last frame)
   int64_t ts_q, hs_q, ts_kv, hs_kv;
   // the cache
   int H, cap, max_n, frame, first;
@@ -112,7 +113,7 @@ struct xkv_cache {
   size_t attn_part_bytes;
   // stream state (host)
   int frames, T, T_first, rest_base, cur, stage;
-  int n_pending, kk_pending, rold_pending, evict_pending, first_pending;
+  int n_pending, nq_pending, kk_pending, rold_pending, evict_pending, first_pending;
   int last_evicted, last_kept, last_prunable;
   long long launches;
   int force_plain;         // 1: kernels take the plain (conversion-based) arithmetic forms everywhere
@@ -178,8 +179,10 @@ cudaError_t launch_regroup(xkv_cache* c, const MaintArgs& a, cudaStream_t st);
 cudaError_t launch_attn_simple(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
                                float scale, cudaStream_t st);
 // Returns cudaErrorNotSupported when the tensor-core kernel cannot take the call.
+// prefix > 0: only the first `prefix` tokens of the cache (logical order) are visible to these queries
+// (frame-causal attention inside a chunk of frames); 0: all of them.
 cudaError_t launch_attn_tc(xkv_cache* c, const void* q, void* out, int n, int64_t ts, int64_t hs,
-                           float scale, cudaStream_t st);
+                           float scale, cudaStream_t st, int prefix = 0);
 // Same kernel with the newest frame's keys and values taken unquantised from k_t, v_t (the tensors
 // given to kv_append, same strides as q).
 cudaError_t launch_attn_tc_tail(xkv_cache* c, const void* q, const void* k_t, const void* v_t, void* out, int n,

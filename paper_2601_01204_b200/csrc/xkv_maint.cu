@@ -312,7 +312,7 @@ __device__ __forceinline__ void phase_pool(const MaintArgs& a, Shared& sh) {
   for (int i = blockIdx.x; i < a.n_pooled; i += gridDim.x) {
     int ta, tb;
     if (i < a.n_special) { ta = i; tb = i + 1; }
-    else { ta = a.n_special + (i - a.n_special) * a.pool_g; tb = min(ta + a.pool_g, a.n); }
+    else { ta = a.n_special + (i - a.n_special) * a.pool_g; tb = min(ta + a.pool_g, a.n_q); }
     // heads h0 and h0 + 8 together: all loads of a batch (2 heads x 16 tokens) are issued before
     // the first (ordered) addition; an index past the group is clamped, its value unused
     for (int h0 = hslot; h0 < a.H; h0 += 16) {

@@ -39,6 +39,7 @@ EXPORTED = [
     "xkv_debug_rewind_attention", "attn_packed_causal_tail", "xkv_set_unquantised_tail",
     "xkv_debug_force_plain", "xkv_debug_limit_attention_blocks", "xkv_debug_timeout_probe",
     "xkv_debug_head_means", "kv_score_evict_w", "xkv_set_budget", "xkv_read_score_stats",
+    "attn_packed_frame_causal", "xkv_prefill_chunk",
 ]
 PROF_NAMES = ["append", "score_evict", "pack", "kbar", "maint", "attn", "attn_combine"]
 
@@ -87,6 +88,10 @@ lib.xkv_set_budget.restype = C.c_int
 lib.xkv_set_budget.argtypes = [_vp, _i32]
 lib.xkv_read_score_stats.restype = C.c_int
 lib.xkv_read_score_stats.argtypes = [_vp, C.POINTER(xkv_score_stats), _vp]
+lib.attn_packed_frame_causal.restype = C.c_int
+lib.attn_packed_frame_causal.argtypes = [_vp, _vp, _vp, C.POINTER(_i32), _i32, _i64, _i64, C.c_float, _vp]
+lib.xkv_prefill_chunk.restype = C.c_int
+lib.xkv_prefill_chunk.argtypes = [_vp, _vp, _vp, _vp, _vp, C.POINTER(_i32), _i32, _i64, _i64, _vp]
 lib.kv_quant_pack.restype = C.c_int
 lib.kv_quant_pack.argtypes = [_vp, _vp]
 lib.attn_packed_causal.restype = C.c_int
@@ -222,6 +227,32 @@ class Cache:
         st = xkv_score_stats()
         _check(lib.xkv_read_score_stats(self.handle, C.byref(st), _stream()), "xkv_read_score_stats")
         return st
+
+    def attn_packed_frame_causal(self, q, frame_tokens, out=None, scale: float | None = None):
+        """Frame-causal attention of a chunk of frames (q, out: [H][sum(frame_tokens)][d])."""
+        import torch
+        if out is None:
+            out = torch.empty_like(q)
+        ts, hs = _strides(q)
+        assert _strides(out) == (ts, hs)
+        if scale is None:
+            scale = 1.0 / float(np.sqrt(self.p.head_dim))
+        ft = (_i32 * len(frame_tokens))(*frame_tokens)
+        _check(lib.attn_packed_frame_causal(self.handle, q.data_ptr(), out.data_ptr(), ft, len(frame_tokens), ts, hs,
+                                            C.c_float(scale), _stream()), "attn_packed_frame_causal")
+        return out
+
+    def xkv_prefill_chunk(self, q, k, v, frame_tokens, out=None):
+        """A chunk of frames through append, scoring (last frame's query), packing and frame-causal attention."""
+        import torch
+        if out is None:
+            out = torch.empty_like(q)
+        ts, hs = _strides(q)
+        assert _strides(out) == (ts, hs) and _strides(k) == (ts, hs) and _strides(v) == (ts, hs)
+        ft = (_i32 * len(frame_tokens))(*frame_tokens)
+        _check(lib.xkv_prefill_chunk(self.handle, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), ft,
+                                     len(frame_tokens), ts, hs, _stream()), "xkv_prefill_chunk")
+        return out
 
     def kv_quant_pack(self) -> None:
         _check(lib.kv_quant_pack(self.handle, _stream()), "kv_quant_pack")

@@ -236,7 +236,7 @@ def test_state_machine_and_argument_errors(xkv):
         cache.kv_append(q, q)
     assert e.value.status == xkv.XKV_E_STATE
     with pytest.raises(xkv.XkvError) as e:
-        cache.kv_score_evict(q[:, :50])
+        cache.kv_score_evict(big)              # more tokens than were appended (fewer is the last frame of a chunk)
     assert e.value.status == xkv.XKV_E_INVALID
     cache.kv_score_evict(q)
     cache.kv_quant_pack()
@@ -494,3 +494,44 @@ def test_budget_changes_query_vector_from_caller_and_score_statistics(xkv, key_m
     assert ca.xkv_get_info().T == 380 + 2 * n and ca.xkv_poll_status() == 0
     with pytest.raises(xkv.XkvError):
         ca.xkv_set_budget(701)
+
+
+# ------------------------------------------------------------------ chunks of frames
+@pytest.mark.parametrize("bits,key_mode", [(4, 0), (4, 1), (16, 0)])
+def test_chunked_prefill_is_frame_causal(xkv, bits, key_mode):
+    """xkv_prefill_chunk: several frames arrive together; the chunk is one arrival for the cache
+    maintenance (scored with its last frame's query) and its attention is frame-causal (Eq. 1): frame
+    f of the chunk sees the older cache and the chunk's frames 0..f.  Against the oracle's step_chunk:
+    state bit-exact, every frame's output within tolerance; chunk sizes that put frame boundaries
+    inside key tiles and query tiles, the first chunk being the first arrival, pruning active later."""
+    import torch
+    from xkv_testlib import compare_state, oracle_params, bf16_tensor_to_f32, check_attention
+    from oracle import xkv_oracle as xo
+    H, d = 4, 64
+    p = xkv.Params(n_heads=H, budget=1100, max_frame_tokens=700, kv_bits=bits, key_mode=key_mode)
+    cache, ora = xkv.Cache(p), xo.OracleLayer(oracle_params(p))
+    chunks = [[150, 261], [261], [100, 200, 150, 37], [261, 261], [8, 136, 300]]
+    t = 0
+    for ci, chunk in enumerate(chunks):
+        fr = [synth.gen_frame(91, 0, t + j, H, n, d) for j, n in enumerate(chunk)]
+        t += len(chunk)
+        qf, kf, vf = ([synth.bf16_bits_to_f32(f[i]) for f in fr] for i in range(3))
+        q, k, v = (to_device_bf16(np.concatenate([f[i] for f in fr], axis=1)) for i in range(3))
+        out = cache.xkv_prefill_chunk(q, k, v, chunk)
+        refs = ora.step_chunk(qf, kf, vf)
+        compare_state(cache.export(), ora.export(), f"chunk {ci}")
+        got = bf16_tensor_to_f32(out).transpose(1, 0, 2)
+        r0 = 0
+        for f, n in enumerate(chunk):
+            check_attention(got[r0:r0 + n], refs[f], f"chunk {ci} frame {f}")
+            r0 += n
+        assert cache.xkv_poll_status() == 0
+    assert cache.xkv_get_info().T == 1100 and ora.last_scores is not None
+    # the pieces by hand, and the argument checks
+    fr = [synth.gen_frame(91, 0, t + j, H, n, d) for j, n in enumerate([64, 64])]
+    q, k, v = (to_device_bf16(np.concatenate([f[i] for f in fr], axis=1)) for i in range(3))
+    cache.kv_append(k, v); cache.kv_score_evict(q[:, 64:], ); cache.kv_quant_pack()
+    with pytest.raises(xkv.XkvError):
+        cache.attn_packed_frame_causal(q, [64, 32])              # sizes must add up to what was appended
+    cache.attn_packed_frame_causal(q, [64, 64])
+    assert cache.xkv_get_info().stage == 0

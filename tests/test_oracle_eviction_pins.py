@@ -255,6 +255,69 @@ def pin_budget_change_and_given_query_vector(xo):
     assert La.T == 150 + n                      # the raised budget lets the cache grow again
 
 
+def pin_chunked_prefill_is_frame_causal(xo):
+    """step_chunk.  (1) Nothing pruned, 16-bit: two chunks of frames give, frame by frame, what
+    one-shot frame-causal attention over all tokens gives (block-triangular mask, Eq. 1), and what
+    streaming the frames one by one gives.  (2) A chunk of one frame is step().  (3) With pruning
+    and 4-bit storage: the cache is first arrival + top-k of the middle + the whole chunk, and frame
+    f's output is attention over the dequantised cache with every token of a later chunk frame
+    masked (mask built from the origins, by the independently written masked routine)."""
+    H, d, G = 2, 16, 8
+    sizes = [[11, 24], [16, 9, 20]]
+    p16 = xo.OracleParams(n_heads=H, head_dim=d, n_special=5, pool_g=4, quant_group=G, kv_bits=16, budget=10 ** 6)
+    Lc, Ls = xo.OracleLayer(p16), xo.OracleLayer(p16)
+    allq, allk, allv, fid, outs_c, outs_s = [], [], [], [], [], []
+    t = 0
+    for chunk in sizes:
+        fr = []
+        for n in chunk:
+            q, k, v = _frame(41, t, H, n, d)
+            fr.append((q, k, v)); allq.append(q); allk.append(k); allv.append(v); fid.append(np.full(n, t)); t += 1
+            outs_s.append(Ls.step(q, k, v))
+        outs_c += Lc.step_chunk([f[0] for f in fr], [f[1] for f in fr], [f[2] for f in fr])
+    fid = np.concatenate(fid)
+    ref = xo_real.attention_frame_causal(np.concatenate(allq, 1), np.concatenate(allk, 1), np.concatenate(allv, 1),
+                                         fid, fid, 1.0 / np.sqrt(d))
+    np.testing.assert_allclose(np.concatenate(outs_c, 0).transpose(1, 0, 2), ref, rtol=1e-5, atol=1e-6)
+    np.testing.assert_allclose(np.concatenate(outs_c, 0), np.concatenate(outs_s, 0), rtol=1e-5, atol=1e-6)
+    # (2)
+    p4 = xo.OracleParams(n_heads=H, head_dim=d, n_special=5, pool_g=4, quant_group=G, kv_bits=4, budget=60)
+    La, Lb = xo.OracleLayer(p4), xo.OracleLayer(p4)
+    for tt in range(5):
+        q, k, v = _frame(42, tt, H, 20, d)
+        oa = La.step(q, k, v)
+        ob = Lb.step_chunk([q], [k], [v])[0]
+        assert np.array_equal(oa, ob) and all(np.array_equal(La.export()[key], Lb.export()[key]) for key in La.export())
+    # (3)
+    L = xo.OracleLayer(xo.OracleParams(n_heads=H, head_dim=d, n_special=5, pool_g=4, quant_group=G, kv_bits=4, budget=90))
+    chunks = [[24], [16, 16], [12, 20, 8], [16, 24]]
+    t = 0
+    for ci, chunk in enumerate(chunks):
+        fr = [_frame(43, t + j, H, n, d) for j, n in enumerate(chunk)]
+        t += len(chunk)
+        T_before, org_before = L.T, L.origin.copy()
+        K_before = L.keys_dequantized().copy() if ci else None
+        outs = L.step_chunk([f[0] for f in fr], [f[1] for f in fr], [f[2] for f in fr])
+        M = sum(chunk)
+        org = L.origin
+        assert np.array_equal(org[-M:], ((ci + 1) << 16) | np.arange(M))                 # the chunk is whole, as one arrival
+        assert np.array_equal(org[:24], (1 << 16) | np.arange(24))                       # so is the first arrival
+        if T_before + M > 90:
+            assert L.T == max(90, 24 + M) and len(L.last_kept_mid) == max(0, 90 - 24 - M)
+            assert np.array_equal(org[24:L.T - M], org_before[24:][L.last_kept_mid])
+            if len(L.last_kept_mid):                                                     # scored with the LAST frame's query
+                S = xo_real.score_literal(fr[-1][0], K_before[:, 24:T_before], 5, 4)
+                assert np.all(np.abs(L.last_scores - S) <= 1e-4 * (np.abs(S) + 1.0))
+        # frame ids of the cached tokens: older than the chunk -> -1, chunk tokens -> their frame in the chunk
+        kf = np.full(L.T, -1)
+        kf[-M:] = np.repeat(np.arange(len(chunk)), chunk)
+        K, V = L.keys_dequantized(), L.values_dequantized()
+        for f, (q, _, _) in enumerate(fr):
+            ref = xo_real.attention_frame_causal(q, K, V, np.full(q.shape[1], f), kf, 1.0 / np.sqrt(d))
+            np.testing.assert_allclose(outs[f].transpose(1, 0, 2), ref, rtol=1e-5, atol=1e-6)
+    assert L.T == 90
+
+
 PINS = [
     ("survivors-4bit", lambda xo: pin_survivor_data_follows_origins(xo, 4)),
     ("survivors-8bit", lambda xo: pin_survivor_data_follows_origins(xo, 8, seed=24)),
@@ -264,6 +327,7 @@ PINS = [
     ("once-8bit", lambda xo: pin_survivor_data_follows_origins(xo, 8, seed=27, key_mode="once")),
     ("once-no-pruning", pin_quantise_once_without_pruning_is_framewise_quantisation),
     ("budget-and-given-w", pin_budget_change_and_given_query_vector),
+    ("chunked-prefill", pin_chunked_prefill_is_frame_causal),
 ]
 
 
@@ -331,6 +395,12 @@ MUTATIONS = [
     ("changed budget ignored by the trigger",
      "if T <= self.budget:                           # trigger",
      "if T <= p.budget:                           # trigger"),
+    ("chunk: every frame sees the whole chunk",
+     "            O = attention(q, K[:, :end], V[:, :end], scale)",
+     "            O = attention(q, K, V, scale)"),
+    ("chunk: scored with the first frame's query",
+     "        self.score_evict(Qs[-1])",
+     "        self.score_evict(Qs[0])"),
     ("first frame re-quantised with the rest",
      "self.k_codes = np.concatenate([self.k_codes[:, :Tf], new_codes], axis=1)",
      "self.k_codes = np.concatenate([self.k_codes[:, :Tf] * 0, new_codes], axis=1)"),

@@ -953,30 +953,43 @@ regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int H, int cap, 
   }
   __syncthreads();
 
-  // ---- values, parameters and origins of the survivors (first frame: nothing to move) ----
-  if (kk > 0) {
-    for (int e = tid; e < kRgHeads * 64 * 2; e += 128 * kRgHeads) {
-      const int half = e & 1, tok = (e >> 1) & 63, hh = blockIdx.y * kRgHeads + (e >> 7);
-      const int i = gamma * 64 + tok;
-      if (hh < H && i < kk) {
-        const size_t s_slot = (size_t)hh * cap + base_slot + s_old[tok];
-        const size_t d_slot = (size_t)hh * cap + base_slot + i;
-        *reinterpret_cast<uint4*>(dst.v + d_slot * 32 + 16 * half) =
-            *reinterpret_cast<const uint4*>(src.v + s_slot * 32 + 16 * half);
-        if (half == 0) dst.vpar[d_slot] = src.vpar[s_slot];
-      }
+  // ---- values, parameters and origins of the survivors (first frame: nothing to move): the row is
+  // fetched here and stored after the key loads below have been issued, so that the two round
+  // trips overlap (thread = (head, token, half row): exactly one item per thread) ----
+  uint4 v_row = make_uint4(0, 0, 0, 0);
+  float2 v_par = make_float2(0.f, 0.f);
+  int v_org = 0;
+  size_t v_dst = 0;
+  bool v_move = false, o_move = false;
+  {
+    const int half = tid & 1, tok = (tid >> 1) & 63, hh = blockIdx.y * kRgHeads + (tid >> 7);
+    const int i = gamma * 64 + tok;
+    if (kk > 0 && hh < H && i < kk) {
+      const size_t s_slot = (size_t)hh * cap + base_slot + s_old[tok];
+      v_dst = (size_t)hh * cap + base_slot + i;
+      v_row = *reinterpret_cast<const uint4*>(src.v + s_slot * 32 + 16 * half);
+      if (half == 0) v_par = src.vpar[s_slot];
+      v_move = true;
     }
-    if (blockIdx.y == 0 && tid < 64) {
-      const int i = gamma * 64 + tid;
-      if (i < kk) dst.origin[base_slot + i] = src.origin[base_slot + s_old[tid]];
+    if (kk > 0 && blockIdx.y == 0 && tid < 64 && gamma * 64 + tid < kk) {
+      v_org = src.origin[base_slot + s_old[tid]];
+      o_move = true;
     }
   }
+  auto store_values = [&]() {
+    if (v_move) {
+      *reinterpret_cast<uint4*>(dst.v + v_dst * 32 + 16 * (tid & 1)) = v_row;
+      if ((tid & 1) == 0) dst.vpar[v_dst] = v_par;
+    }
+    if (o_move) dst.origin[base_slot + gamma * 64 + tid] = v_org;
+  };
 
   // ---- keys ----
   const int last = gamma * 64 + 63;
   const bool carried = (last < kk) && (s_old[63] == last);
   const size_t dgrp = ((size_t)h * (cap >> 6) + (base_slot >> 6) + gamma) * 64;
   if (carried) {
+    store_values();
     if (head_ok) {
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -1009,6 +1022,7 @@ regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int H, int cap, 
     else if (head_ok && old[u] == -1)
       fresh[u] = *reinterpret_cast<const uint4*>(kstage + ((size_t)h * max_n + (i - kk)) * 64 + 8 * w);
   }
+  store_values();
   int par_grp = -1;
   float2 par[8];
   bool par_plain = false;

@@ -106,13 +106,37 @@ __device__ __forceinline__ void dequant8_magic(uint32_t word, const float2 (&par
   }
 }
 
-// clamp(rint(x * inv) + z, 0, 15) for |x * inv| < 2^21 and integer |z| < 2^22; zadj = int(z) - bits(magic).
-__device__ __forceinline__ uint32_t quant_code_magic(float x, float inv, int zadj) {
-  const float t = __fadd_rn(__fmul_rn(x, inv), kRoundMagic);
-  const int q = (int)__float_as_uint(t) + zadj;
-  int r;
-  asm("min.relu.s32 %0, %1, 15;" : "=r"(r) : "r"(q));   // max(min(q, 15), 0)
-  return (uint32_t)r;
+// Two fp32 numbers in one 64-bit register and the packed forms of the IEEE operations (each half
+// is rounded exactly like the scalar operation, so results do not change; one instruction does two).
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpk2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+// dequant8_magic on channel pairs: s2[p] = (s of channel 2p, s of channel 2p + 1), mz2[p] the same
+// for magic + z.
+__device__ __forceinline__ void dequant8_magic2(uint32_t word, const uint64_t (&s2)[4], const uint64_t (&mz2)[4],
+                                                float (&x)[8]) {
+  const uint32_t hi = word >> 16;
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    const uint32_t be = (word & (0xFu << (4 * p))) | magic_bits(2 * p);
+    const uint32_t bo = (hi & (0xFu << (4 * p))) | magic_bits(2 * p);
+    unpk2(mul2(s2[p], sub2(pk2(__uint_as_float(be), __uint_as_float(bo)), mz2[p])), x[2 * p], x[2 * p + 1]);
+  }
 }
 
 // The plain forms as real calls on scalars, so that the rarely taken fallback costs a branch and
@@ -1024,7 +1048,8 @@ regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int H, int cap, 
   }
   store_values();
   int par_grp = -1;
-  float2 par[8];
+  const float2* par_src = nullptr; // the group's (s, z) in global memory (the plain path reads them there)
+  uint64_t s2[4], mz2[4];          // fast path: (s, s) and (magic + z, magic + z) of the channel pairs
   bool par_plain = false;
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
@@ -1036,19 +1061,16 @@ regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int H, int cap, 
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
           const float4 q4 = __ldg(pp + v);
-          par[2 * v] = make_float2(q4.x, q4.y);
-          par[2 * v + 1] = make_float2(q4.z, q4.w);
           zmax = fmaxf(zmax, fmaxf(fabsf(q4.y), fabsf(q4.w)));
+          s2[v] = pk2(q4.x, q4.z);
+          mz2[v] = pk2(__fadd_rn(magic_val(2 * v), q4.y), __fadd_rn(magic_val(2 * v), q4.w));
         }
         par_plain = !(zmax < kZLimit) || force_plain;
-        if (!par_plain) {
-#pragma unroll
-          for (int j = 0; j < 8; ++j) par[j].y = __fadd_rn(magic_val(j), par[j].y);
-        }
+        par_src = reinterpret_cast<const float2*>(pp);
         par_grp = g;
       }
-      if (par_plain) dequant8_plain(word[u], par, x[u]);
-      else dequant8_magic(word[u], par, x[u]);
+      if (par_plain) dequant8_plain(word[u], par_src, x[u]);
+      else dequant8_magic2(word[u], s2, mz2, x[u]);
     } else {
       bf16x8_to_float(fresh[u], x[u]);
     }
@@ -1098,11 +1120,14 @@ regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int H, int cap, 
   if (!head_ok) return;
   float2 iz[8];
   int zadj[8];
+  uint64_t inv2[4];
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     iz[j] = s_iz[hl][8 * w + j];
     zadj[j] = slow ? 0 : (int)iz[j].y - (int)0x4B400000;
   }
+#pragma unroll
+  for (int p = 0; p < 4; ++p) inv2[p] = pk2(iz[2 * p].x, iz[2 * p + 1].x);
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
     if (old[u] == -2) continue;
@@ -1114,8 +1139,21 @@ regroup_k_kernel(BufSet src, BufSet dst, BufSet dst2, bool two, int H, int cap, 
     } else {
       packed = 0u;
 #pragma unroll
-      for (int j = 0; j < 8; ++j)   // the nibbles do not overlap: multiply-add places them
-        packed = quant_code_magic(x[u][j], iz[j].x, zadj[j]) * (1u << nib_shift(j)) + packed;
+      for (int p = 0; p < 4; ++p) {
+        // x * inv for two channels at once; the addition of 1.5 * 2^23 stays scalar: a packed
+        // multiplication followed by a packed addition was observed to round once, like a fused
+        // multiply-add, which breaks the ties of Eq. 7's rounding
+        float te, to;
+        unpk2(mul2(pk2(x[u][2 * p], x[u][2 * p + 1]), inv2[p]), te, to);
+        te = __fadd_rn(te, kRoundMagic);
+        to = __fadd_rn(to, kRoundMagic);
+        int qe = (int)__float_as_uint(te) + zadj[2 * p], qo = (int)__float_as_uint(to) + zadj[2 * p + 1];
+        asm("min.relu.s32 %0, %1, 15;" : "=r"(qe) : "r"(qe));
+        asm("min.relu.s32 %0, %1, 15;" : "=r"(qo) : "r"(qo));
+        // the nibbles do not overlap: multiply-add places them
+        packed = (uint32_t)qe * (1u << nib_shift(2 * p)) + packed;
+        packed = (uint32_t)qo * (1u << nib_shift(2 * p + 1)) + packed;
+      }
     }
     const size_t dslot = (size_t)h * cap + base_slot + gamma * 64 + tq + 16 * u;
     *reinterpret_cast<uint32_t*>(dst.k + dslot * 32 + 4 * w) = packed;

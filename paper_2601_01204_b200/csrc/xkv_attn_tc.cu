@@ -359,15 +359,17 @@ __device__ __noinline__ void tail_rows_over(uint8_t* tile_row, const __nv_bfloat
     u[i] = make_uint4(0, 0, 0, 0);
     if (slot >= tail_lo && slot < t_phys) u[i] = *reinterpret_cast<const uint4*>(src + (int64_t)(slot - tail_lo) * ts);
   }
+  uint32_t seen = 0u;       // exponent bits of everything written: all ones somewhere = beyond fp16
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int slot = slot0 + 16 * i;
     if (slot >= tail_lo && slot < t_phys) {
       const uint4 hv = bf16x8_to_h8(u[i]);
       *reinterpret_cast<uint4*>(tile_row + i * 2048) = hv;
-      if (h2_not_finite(hv.x) || h2_not_finite(hv.y) || h2_not_finite(hv.z) || h2_not_finite(hv.w)) report_range(status);
+      seen |= (h2_not_finite(hv.x) || h2_not_finite(hv.y) || h2_not_finite(hv.z) || h2_not_finite(hv.w)) ? 1u : 0u;
     }
   }
+  if (seen) report_range(status);
 }
 
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {

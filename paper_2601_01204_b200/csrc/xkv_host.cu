@@ -572,34 +572,35 @@ int run_layer(HostStepPipe* pipe, xkv_cache* c, const void* q, const void* k, co
   if (c->p.kv_bits == 4 && !once && launch_regroup(c, a, st) != cudaSuccess) return XKV_E_CUDA;
   note_packed(c);
   c->stage = 3;
-  if (once && !plan.first) {
-    // head means (Eq. 4) of the frame just quantised: needed by the next frame's scoring only, so
-    // they are computed on the side stream, beside the attention
-    bool ok = cudaEventRecord(pipe->fork, st) == cudaSuccess && cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess;
-    if (!ok) return XKV_E_CUDA;
-    a.phases = kPhKbarNew;
-    const bool launched = launch_maint(c, a, XKV_PROF_KBAR, pipe->side) == cudaSuccess;
-    ok = cudaEventRecord(c->kbar_done, pipe->side) == cudaSuccess;
-    if (!launched || !ok) return XKV_E_CUDA;
-    c->kbar_T = c->T; c->kbar_cur = c->cur; c->kbar_frames = c->frames;
-  }
-  if (!once && c->T > c->T_first) {
-    bool ok = cudaEventRecord(pipe->fork, st) == cudaSuccess && cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess;
-    if (!ok) return XKV_E_CUDA;
+  // Head means of the keys (Eq. 4), needed by the next frame's scoring only: on the side stream,
+  // beside the attention.  The side stream forks here (after the packing) but its kernel is
+  // launched after the attention has been enqueued, so that the attention's blocks get the
+  // multiprocessors first and the head means fill in as they retire.
+  const bool want_kbar = once ? !plan.first : (c->T > c->T_first);
+  if (want_kbar && !(cudaEventRecord(pipe->fork, st) == cudaSuccess &&
+                     cudaStreamWaitEvent(pipe->side, pipe->fork, 0) == cudaSuccess))
+    return XKV_E_CUDA;
+  const float scale = 1.0f / sqrtf((float)c->p.head_dim);
+  rc = c->tail_mode ? attn_packed_causal_tail(c, q, k, v, out, n, ts, hs, scale, stream)
+                    : attn_packed_causal(c, q, out, n, ts, hs, scale, 0, stream);
+  if (want_kbar && rc == XKV_OK) {
     MaintArgs b;
-    maint_args(c, &b);
-    b.phases = kPhKbar;
-    b.kbar_on_other = 0; b.kbar_lo = 0; b.kbar_hi = c->T - c->T_first;
+    if (once) {               // of the frame just quantised (the rest travelled with their tokens)
+      b = a;
+      b.phases = kPhKbarNew;
+    } else {                  // of the whole cache after the first frame: re-quantisation changed the keys
+      maint_args(c, &b);
+      b.phases = kPhKbar;
+      b.kbar_on_other = 0; b.kbar_lo = 0; b.kbar_hi = c->T - c->T_first;
+    }
     const bool launched = launch_maint(c, b, XKV_PROF_KBAR, pipe->side) == cudaSuccess;
-    ok = cudaEventRecord(c->kbar_done, pipe->side) == cudaSuccess;
+    const bool ok = cudaEventRecord(c->kbar_done, pipe->side) == cudaSuccess;
     // (the caller's stream waits for it at the end of the stream-step call, and at the next
     // frame's scoring)
     if (!launched || !ok) return XKV_E_CUDA;
     c->kbar_T = c->T; c->kbar_cur = c->cur; c->kbar_frames = c->frames;
   }
-  const float scale = 1.0f / sqrtf((float)c->p.head_dim);
-  return c->tail_mode ? attn_packed_causal_tail(c, q, k, v, out, n, ts, hs, scale, stream)
-                      : attn_packed_causal(c, q, out, n, ts, hs, scale, 0, stream);
+  return rc;
 }
 
 // Everything a stream-step call started on the side stream is ordered before what the caller

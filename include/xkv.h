@@ -340,10 +340,10 @@ XKV_API int xkv_stream_step(xkv_cache* const* layers, int32_t n_layers,
  * gives asynchronous copies).  q, k, v, out are HOST arrays of n_layers HOST
  * pointers to bf16 [H][n][d] tensors; dev_staging is device scratch of at least
  * xkv_stream_step_host_bytes(layers[0] params, n) bytes.  The layers run on
- * `stream`; the inputs of the next layer are copied on a second stream while a
- * layer runs and the outputs go back on a third (both created by the library on
- * first use, one pair per device), so that copies overlap the kernels.  All three
- * are synchronised before the call returns.  Not for use inside a stream capture. */
+ * `stream`; the inputs of the next layer are copied on two further streams (two copy
+ * engines) while a layer runs and the outputs go back on a fourth (all created by the
+ * library on first use, one set per device), so that copies overlap the kernels.  All
+ * of them are synchronised before the call returns.  Not for use inside a stream capture. */
 XKV_API size_t xkv_stream_step_host_bytes(const xkv_params* params, int32_t n);
 XKV_API int xkv_stream_step_host(xkv_cache* const* layers, int32_t n_layers,
                          const void* const* q, const void* const* k, const void* const* v,

@@ -197,6 +197,8 @@ def run_xkv(args) -> None:
     if args.layers > 0:
         w["layers"] = args.layers
         w["name"] += f"_reduced_to_{args.layers}_layers"
+    if args.bits == 8:
+        args.keys = "once"
     w["key_mode"] = 1 if args.keys == "once" else 0
     if args.keys == "once":
         w["name"] += "_keys_once"
@@ -204,7 +206,7 @@ def run_xkv(args) -> None:
         w["budget"] = args.budget or w["budget"]
         w["kv_bits"] = args.bits or w["kv_bits"]
         w["n_tokens"] = args.tokens or w["n_tokens"]
-        w["name"] = f"stack_{w['layers']}L_{w['n_tokens']}tok_budget{w['budget']}_{'int4' if w['kv_bits'] == 4 else 'bf16'}"
+        w["name"] = f"stack_{w['layers']}L_{w['n_tokens']}tok_budget{w['budget']}_{ {4: 'int4', 8: 'int8', 16: 'bf16'}[w['kv_bits']] }"
         if args.keys == "once":
             w["name"] += "_keys_once"
     L, H, d, n = w["layers"], w["n_heads"], w["head_dim"], w["n_tokens"]
@@ -465,7 +467,8 @@ def main() -> None:
     ap.add_argument("--impl", default="xkv", choices=["xkv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--budget", type=int, default=0, help="variant of the workload: token budget (ablation sweep)")
-    ap.add_argument("--bits", type=int, default=0, choices=[0, 4, 16], help="variant: 4 or 16 (prune only)")
+    ap.add_argument("--bits", type=int, default=0, choices=[0, 4, 8, 16],
+                    help="variant: 4, 16 (prune only) or 8 (implies --keys once)")
     ap.add_argument("--tokens", type=int, default=0, help="variant: tokens per frame (1004 = long-stream shape)")
     ap.add_argument("--keys", default="regroup", choices=["regroup", "once"],
                     help="variant: keys re-quantised per 64-position run every step (default) or quantised once on arrival")

@@ -63,14 +63,15 @@ typedef enum {
 
 /* Method parameters.  Defaults of the paper: n_special = 5 (1 camera + 4
  * register tokens, Sec. 3.1), pool_g = 16, quant_group = 64, kv_bits = 4
- * (Sec. 4.1).  kv_bits = 16 keeps bf16 values (pruning only). */
+ * (Sec. 4.1).  kv_bits = 16 keeps bf16 values (pruning only).  kv_bits = 8 applies the same
+ * Eq. 7-9 with 256 levels (the paper evaluates INT4 only); it is built for XKV_KEYS_ONCE. */
 typedef struct {
   int32_t n_heads;           /* H, 1..64                                                 */
   int32_t head_dim;          /* d, only 64                                               */
   int32_t n_special;         /* special tokens at the head of each frame, >= 0           */
   int32_t pool_g;            /* g of GroupAvg (Eq. 2), >= 1                              */
   int32_t quant_group;       /* G, cache positions per key group, only 64                */
-  int32_t kv_bits;           /* b: 4 or 16                                               */
+  int32_t kv_bits;           /* b: 4, 16, or 8 (XKV_KEYS_ONCE only)                      */
   int32_t budget;            /* L_max, the token budget (Sec. 3.2), >= 1                 */
   int32_t max_frame_tokens;  /* largest n any frame will have, 1..65535                  */
   int32_t key_mode;          /* XKV_KEYS_REGROUP (0) or XKV_KEYS_ONCE (1), see below; 4-bit only */
@@ -117,6 +118,8 @@ typedef struct {
  *   K_CODES / V_CODES : kv_bits = 4 : uint8 [H][capacity][d/2]; the 8 codes of channels
  *                       8w..8w+7 form the little-endian 32-bit word
  *                       c0 | c2<<4 | c4<<8 | c6<<12 | c1<<16 | c3<<20 | c5<<24 | c7<<28
+ *                       kv_bits = 8 : uint8 [H][capacity][d]; the 4 codes of channels 4w..4w+3 form the
+ *                       little-endian word c0 | c2<<8 | c1<<16 | c3<<24
  *                       kv_bits = 16: bf16 [H][capacity][d]
  *   K_PARAMS          : float2 (scale, zero) [H][capacity/64][d], group = 64 slots
  *   V_PARAMS          : float2 (scale, zero) [H][capacity]

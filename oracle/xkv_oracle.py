@@ -84,7 +84,7 @@ class OracleParams:
     n_special: int = 5       # camera + register tokens at the head of a frame (Sec. 3.1)
     pool_g: int = 16         # g, pooling size (Sec. 4.1)
     quant_group: int = 64    # G, tokens per key group (Sec. 4.1)
-    kv_bits: int = 4         # b; 16 = keep bf16 values (prune only)
+    kv_bits: int = 4         # b: 4 (the paper's), 8 (same Eq. 7-8, beyond what the paper evaluates); 16 = keep bf16 values
     budget: int = 2048       # L_max
     # how the per-channel key groups (Eq. 9) live with eviction:
     #   "regroup": groups are runs of G cache positions; a group that changed is re-quantised
@@ -307,6 +307,22 @@ def unpack_nibbles(packed: np.ndarray) -> np.ndarray:
     for i in range(8):
         out[..., i] = ((words >> _NIBBLE_SHIFT[i]) & np.uint32(0xF)).astype(np.uint8)
     return out.reshape(packed.shape[:-1] + (dh * 2,))
+
+
+# 8-bit packing: 4 channels -> one little-endian 32-bit word c0 | c2<<8 | c1<<16 | c3<<24, i.e. the
+# bytes of channels (0, 2, 1, 3) in memory order, so that the mask 0x00FF00FF selects the adjacent
+# channels (0, 1) and the same mask on the word shifted right by 8 selects (2, 3).
+def pack_bytes8(codes: np.ndarray) -> np.ndarray:
+    """uint8 codes [...][d] (values 0..255) -> uint8 [...][d] in storage order."""
+    d = codes.shape[-1]
+    assert d % 4 == 0
+    c = codes.reshape(codes.shape[:-1] + (d // 4, 4))
+    return np.ascontiguousarray(c[..., [0, 2, 1, 3]]).reshape(codes.shape)
+
+
+def unpack_bytes8(packed: np.ndarray) -> np.ndarray:
+    """Inverse of pack_bytes8 (the permutation is its own inverse)."""
+    return pack_bytes8(packed)
 
 
 # --------------------------------------------------------------------------
@@ -622,8 +638,9 @@ class OracleLayer:
             out["k_val"] = self.k_val.copy()
             out["v_val"] = self.v_val.copy()
         else:
-            out["k_packed"] = pack_nibbles(self.k_codes)
-            out["v_packed"] = pack_nibbles(self.v_codes)
+            pack = pack_nibbles if p.kv_bits == 4 else pack_bytes8
+            out["k_packed"] = pack(self.k_codes)
+            out["v_packed"] = pack(self.v_codes)
             if p.key_mode == "once":
                 out["k_s_tok"], out["k_z_tok"] = self.key_params_per_token()
                 out["k_groups_live"] = len(self.k_table)

@@ -62,6 +62,20 @@ attn_simple_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restric
             kx[j] = sz.x * ((float)((kw >> nib_shift_s(j)) & 0xFu) - sz.y);
             vx[j] = vp.x * ((float)((vw >> nib_shift_s(j)) & 0xFu) - vp.y);
           }
+        } else if (BITS == 8) {
+          // 8-bit codes (keys quantised once): bytes of channels (0, 2, 1, 3) per word
+          const uint2 kw = *reinterpret_cast<const uint2*>(buf.k + slot * 64 + 8 * w);
+          const uint2 vw = *reinterpret_cast<const uint2*>(buf.v + slot * 64 + 8 * w);
+          const float2* kp = ktab + ((size_t)buf.kslot[p] * H + h) * 64 + 8 * w;
+          const float2 vp = buf.vpar[slot];
+          const uint32_t kws[2] = {kw.x, kw.y}, vws[2] = {vw.x, vw.y};
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int sh = ((j & 3) == 0) ? 0 : ((j & 3) == 1) ? 16 : ((j & 3) == 2) ? 8 : 24;
+            const float2 sz = kp[j];
+            kx[j] = sz.x * ((float)((kws[j >> 2] >> sh) & 0xFFu) - sz.y);
+            vx[j] = vp.x * ((float)((vws[j >> 2] >> sh) & 0xFFu) - vp.y);
+          }
         } else {
           const uint4 ku = *reinterpret_cast<const uint4*>(buf.k + slot * 128 + 16 * w);
           const uint4 vu = *reinterpret_cast<const uint4*>(buf.v + slot * 128 + 16 * w);
@@ -149,7 +163,10 @@ cudaError_t launch_attn_simple(xkv_cache* c, const void* q, void* out, int n, in
   auto qq = reinterpret_cast<const __nv_bfloat16*>(q);
   auto oo = reinterpret_cast<__nv_bfloat16*>(out);
   LaunchScope ls(c, XKV_PROF_ATTN, st);
-  if (c->p.kv_bits == 16)
+  if (c->p.kv_bits == 8)
+    attn_simple_kernel<8><<<grid, 128, 0, st>>>(qq, oo, n, ts, hs, c->buf[c->cur], c->cap, c->T_first,
+                                                c->rest_base, t_phys, scale_log2, c->ktab32, c->p.n_heads);
+  else if (c->p.kv_bits == 16)
     attn_simple_kernel<16><<<grid, 128, 0, st>>>(qq, oo, n, ts, hs, c->buf[c->cur], c->cap, c->T_first,
                                                  c->rest_base, t_phys, scale_log2, nullptr, c->p.n_heads);
   else

@@ -63,6 +63,11 @@ template <> struct Cfg<4> {
   static constexpr int kRawK = 4096, kRawV = 4096, kRawKP = 1024, kRawVP = 1024;
   static constexpr int kRawStage = kRawK + kRawV + kRawKP + kRawVP;
 };
+template <> struct Cfg<8> {                    // 8-bit codes, keys quantised once: K, V rows of 64 bytes,
+  static constexpr int kNR = 4;               // 128 group references (in the K-parameter region), V parameters
+  static constexpr int kRawK = 8192, kRawV = 8192, kRawKP = 1024, kRawVP = 1024;
+  static constexpr int kRawStage = kRawK + kRawV + kRawKP + kRawVP;
+};
 template <> struct Cfg<16> {
   static constexpr int kNR = 2;
   static constexpr int kRawK = 16384, kRawV = 16384, kRawKP = 0, kRawVP = 0;
@@ -320,6 +325,23 @@ __device__ __forceinline__ uint4 dequant_word_h(uint32_t w, const uint32_t (&s2)
   const uint32_t a1 = (w & 0x00F000F0u) | 0x54005400u;
   const uint32_t a2 = (t & 0x000F000Fu) | 0x64006400u;
   const uint32_t a3 = (t & 0x00F000F0u) | 0x54005400u;
+  uint4 r;
+  r.x = h2_fma(h2_sub(a0, zo[0]), s2[0], c2[0]);
+  r.y = h2_fma(h2_sub(a1, zo[1]), s2[1], c2[1]);
+  r.z = h2_fma(h2_sub(a2, zo[2]), s2[2], c2[2]);
+  r.w = h2_fma(h2_sub(a3, zo[3]), s2[3], c2[3]);
+  return r;
+}
+
+// The same for eight 8-bit codes (two words, channels 4i..4i+3 as c0 | c2<<8 | c1<<16 | c3<<24):
+// (w & 0x00FF00FF) | 0x6400 is the fp16 pair (1024 + c0, 1024 + c1), the word shifted by 8 gives
+// (1024 + c2, 1024 + c3); every pair carries the bias 1024.
+__device__ __forceinline__ uint4 dequant_words8_h(uint2 w, const uint32_t (&s2)[4], const uint32_t (&zo)[4],
+                                                  const uint32_t (&c2)[4]) {
+  const uint32_t a0 = (w.x & 0x00FF00FFu) | 0x64006400u;
+  const uint32_t a1 = ((w.x >> 8) & 0x00FF00FFu) | 0x64006400u;
+  const uint32_t a2 = (w.y & 0x00FF00FFu) | 0x64006400u;
+  const uint32_t a3 = ((w.y >> 8) & 0x00FF00FFu) | 0x64006400u;
   uint4 r;
   r.x = h2_fma(h2_sub(a0, zo[0]), s2[0], c2[0]);
   r.y = h2_fma(h2_sub(a1, zo[1]), s2[1], c2[1]);
@@ -819,6 +841,63 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           // the fence above: released right after the loads, the refill of the stage was observed
           // to reach some of those loads when the wait in between was long.
           mbar_arrive(b_rfree + 8 * rs);
+        } else if (BITS == 8) {
+          // ---- 8-bit codes (keys quantised once): the same steps with rows of 64 bytes ----
+          uint8_t* tab = sgen + kOffTab + (g & 1) * kTabBytes;
+          {
+            const float2 vp = *reinterpret_cast<const float2*>(raw + C::kRawK + C::kRawV + C::kRawKP + 8 * t);   // key t
+            float vl, vh, vc;
+            dequant_consts(vp.x, vp.y, vl, vh, vc);
+            *reinterpret_cast<uint4*>(tab + 768 + 16 * t) = make_uint4(pack_h2(vp.x, vp.x), pack_h2(vl, vl), 0u, pack_h2(vc, vc));
+            if (beyond_fp16(fabsf(vp.x) * (fabsf(vp.y) + 255.f))) report_range(a.status);
+          }
+          producer_sync();
+          uint2 wd8[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) wd8[i] = *reinterpret_cast<const uint2*>(raw + (kb + 16 * i) * 64 + 8 * w);
+          int sl[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) sl[i] = *reinterpret_cast<const int*>(raw + C::kRawK + C::kRawV + 4 * (kb + 16 * i));
+          uint4 sv[4], zv[4], cv[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint4* e = reinterpret_cast<const uint4*>(a.ktab16 + (((size_t)sl[i] * a.n_heads + h) * 8 + w) * 12);
+            sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2);
+          }
+          mbar_wait<256>(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t s2[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w}, zo[4] = {zv[i].x, zv[i].y, zv[i].z, zv[i].w};
+              const uint32_t c2[4] = {cv[i].x, cv[i].y, cv[i].z, cv[i].w};
+              const uint4 o = dequant_words8_h(wd8[4 * half + i], s2, zo, c2);
+              *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (4 * half + i) * 2048) = o;
+            }
+            if (half == 0) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const uint4* e = reinterpret_cast<const uint4*>(a.ktab16 + (((size_t)sl[4 + i] * a.n_heads + h) * 8 + w) * 12);
+                sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2);
+              }
+            }
+          }
+          fence_proxy_async();
+          mbar_arrive(b_kfull + 8 * kbuf);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) wd8[i] = *reinterpret_cast<const uint2*>(raw + C::kRawK + (kb + 16 * i) * 64 + 8 * w);
+          mbar_wait<256>(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint4 pv = *reinterpret_cast<const uint4*>(tab + 768 + 16 * (kb + 16 * i));
+            const uint32_t s2[4] = {pv.x, pv.x, pv.x, pv.x}, zo[4] = {pv.y, pv.y, pv.y, pv.y};
+            const uint32_t c2[4] = {pv.w, pv.w, pv.w, pv.w};
+            const uint4 o = dequant_words8_h(wd8[i], s2, zo, c2);
+            *reinterpret_cast<uint4*>(sgen + kOffV + vbuf * 16384 + row_off + i * 2048) = o;
+          }
+          fence_proxy_async();
+          mbar_arrive(b_vfull + 8 * vbuf);
+          mbar_arrive(b_rfree + 8 * rs);
         } else {
           uint4 rowk[8];
 #pragma unroll
@@ -917,6 +996,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
           tma_load_1d(dst + C::kRawK, a.v + slot0 * 32, C::kRawV, bar);
           if (ONCE) tma_load_1d(dst + C::kRawK + C::kRawV, a.kslot + (size_t)tile * 128, kp_bytes, bar);
           else tma_load_1d(dst + C::kRawK + C::kRawV, a.kpar + ((size_t)h * (a.cap >> 6) + 2 * tile) * 64, C::kRawKP, bar);
+          tma_load_1d(dst + C::kRawK + C::kRawV + C::kRawKP, a.vpar + slot0, C::kRawVP, bar);
+        } else if (BITS == 8) {
+          tma_load_1d(dst, a.k + slot0 * 64, C::kRawK, bar);
+          tma_load_1d(dst + C::kRawK, a.v + slot0 * 64, C::kRawV, bar);
+          tma_load_1d(dst + C::kRawK + C::kRawV, a.kslot + (size_t)tile * 128, kp_bytes, bar);
           tma_load_1d(dst + C::kRawK + C::kRawV + C::kRawKP, a.vpar + slot0, C::kRawVP, bar);
         } else {
           tma_load_1d(dst, a.k + slot0 * 128, C::kRawK, bar);
@@ -1047,6 +1131,8 @@ static cudaError_t attn_device_setup(int* sm_count) {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<4, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_tc_kernel<8, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<8>());
+    if (e != cudaSuccess) return e;
     g_sm_count[dev] = sms;
   }
   *sm_count = g_sm_count[dev];
@@ -1095,6 +1181,7 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
   a.k_tail = a.v_tail = nullptr;
   a.tail_ts = a.tail_hs = 0;
   a.tail_lo = a.t_phys;
+  if (tail && c->p.kv_bits == 8) return cudaErrorNotSupported;      // (the unquantised tail is built for 4-bit caches)
   if (tail && c->p.kv_bits == 4) {      // a 16-bit cache holds the frame exactly as it arrived
     a.k_tail = reinterpret_cast<const __nv_bfloat16*>(tail->k);
     a.v_tail = reinterpret_cast<const __nv_bfloat16*>(tail->v);
@@ -1106,6 +1193,7 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
     LaunchScope ls(c, XKV_PROF_ATTN, st);
     const bool once = c->p.key_mode == XKV_KEYS_ONCE;
     if (c->p.kv_bits == 16) attn_tc_kernel<16><<<(int)grid, kThreads, smem_bytes<16>(), st>>>(a);
+    else if (c->p.kv_bits == 8) attn_tc_kernel<8, false, true><<<(int)grid, kThreads, smem_bytes<8>(), st>>>(a);
     else if (a.k_tail && once) attn_tc_kernel<4, true, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
     else if (a.k_tail) attn_tc_kernel<4, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
     else if (once) attn_tc_kernel<4, false, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);

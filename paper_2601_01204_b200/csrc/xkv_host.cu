@@ -30,12 +30,13 @@ bool params_ok(const xkv_params* p) {
   if (!p) return false;
   if (p->n_heads < 1 || p->n_heads > 64) return false;
   if (p->head_dim != kHeadDim || p->quant_group != kGroup) return false;
-  if (p->kv_bits != 4 && p->kv_bits != 16) return false;
+  if (p->kv_bits != 4 && p->kv_bits != 8 && p->kv_bits != 16) return false;
   if (p->n_special < 0 || p->pool_g < 1 || p->budget < 1) return false;
   if (p->max_frame_tokens < 1 || p->max_frame_tokens > 65535) return false;
   if (p->budget > (1 << 24)) return false;
   if (p->key_mode != XKV_KEYS_REGROUP && p->key_mode != XKV_KEYS_ONCE) return false;
-  if (p->key_mode == XKV_KEYS_ONCE && p->kv_bits != 4) return false;
+  if (p->key_mode == XKV_KEYS_ONCE && p->kv_bits == 16) return false;
+  if (p->kv_bits == 8 && p->key_mode != XKV_KEYS_ONCE) return false;      // 8-bit codes: quantise-once mode only
   if (p->key_table_slots < 0 || (p->key_mode != XKV_KEYS_ONCE && p->key_table_slots != 0)) return false;
   return true;
 }
@@ -48,7 +49,7 @@ Layout make_layout(const xkv_params* p) {
   const int cap_first = round_up(max_n, kTile);
   const int cap_rest = round_up(p->budget > max_n ? p->budget : max_n, kTile) + kTile;
   L.cap = cap_first + cap_rest;
-  L.row_bytes = (p->kv_bits == 4) ? 32 : 128;
+  L.row_bytes = (p->kv_bits == 4) ? 32 : (p->kv_bits == 8) ? 64 : 128;
   const size_t H = (size_t)p->n_heads;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + kAlign - 1) / kAlign * kAlign; return o; };
@@ -125,7 +126,7 @@ int xkv_create(const xkv_params* params, void* dev_workspace, size_t bytes, xkv_
   if (!params_ok(params)) {
     if (params->head_dim != kHeadDim && params->head_dim > 0) return XKV_E_UNSUPPORTED;
     if (params->quant_group != kGroup && params->quant_group > 0) return XKV_E_UNSUPPORTED;
-    if (params->kv_bits == 2 || params->kv_bits == 8) return XKV_E_UNSUPPORTED;
+    if (params->kv_bits == 2 || params->kv_bits == 8) return XKV_E_UNSUPPORTED;   // 8 needs XKV_KEYS_ONCE
     return XKV_E_INVALID;
   }
   if (!dev_workspace || (reinterpret_cast<uintptr_t>(dev_workspace) % kAlign) != 0) return XKV_E_INVALID;

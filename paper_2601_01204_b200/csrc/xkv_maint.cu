@@ -43,20 +43,30 @@ constexpr int kBlocksPerSM = 2;
 constexpr uint32_t kBarSpin = 1u << 21;  // polls of a grid barrier before it gives up (about 0.1 s)
 
 // ---------------------------------------------------------------------------
-// Eq. 7-8, fixed-order fp32:  s = (max-min)/15 (1 if the range is 0),
-// inv = 1/s, z = rint(-min*inv) + 0, q = clamp(rint(x*inv) + z, 0, 15).
+// Eq. 7-8, fixed-order fp32:  s = (max-min)/(2^b - 1) (1 if the range is 0),
+// inv = 1/s, z = rint(-min*inv) + 0, q = clamp(rint(x*inv) + z, 0, 2^b - 1).  qmax = 2^b - 1.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ void quant_params(float mn, float mx, float& s, float& inv, float& z) {
+__device__ __forceinline__ void quant_params(float mn, float mx, float& s, float& inv, float& z, float qmax = 15.f) {
   const float r = __fsub_rn(mx, mn);
-  s = (r == 0.f) ? 1.f : __fdiv_rn(r, 15.f);
+  s = (r == 0.f) ? 1.f : __fdiv_rn(r, qmax);
   inv = __fdiv_rn(1.f, s);
   z = __fadd_rn(rintf(__fmul_rn(-mn, inv)), 0.f);
 }
 
-__device__ __forceinline__ uint32_t quant_code(float x, float inv, float z) {
+__device__ __forceinline__ uint32_t quant_code(float x, float inv, float z, float qmax = 15.f) {
   float q = __fadd_rn(rintf(__fmul_rn(x, inv)), z);
-  q = fminf(fmaxf(q, 0.f), 15.f);
+  q = fminf(fmaxf(q, 0.f), qmax);
   return (uint32_t)q;
+}
+
+// 8-bit storage: the codes of channels 4i..4i+3 form the word c0 | c2<<8 | c1<<16 | c3<<24, so that
+// the mask 0x00FF00FF yields the adjacent channels (0, 1) and, after a shift by 8, (2, 3).
+__device__ __forceinline__ uint32_t pack4_bytes(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3) {
+  return c0 | (c2 << 8) | (c1 << 16) | (c3 << 24);
+}
+__device__ __forceinline__ void unpack8_bytes(uint2 w, uint32_t (&c)[8]) {
+  c[0] = w.x & 0xFFu; c[2] = (w.x >> 8) & 0xFFu; c[1] = (w.x >> 16) & 0xFFu; c[3] = w.x >> 24;
+  c[4] = w.y & 0xFFu; c[6] = (w.y >> 8) & 0xFFu; c[5] = (w.y >> 16) & 0xFFu; c[7] = w.y >> 24;
 }
 
 // Bit position of channel j (0..7) inside the packed word:
@@ -299,17 +309,24 @@ __device__ __forceinline__ void phase_append(const MaintArgs& a) {
         mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
       }
+      constexpr float kQmax = (BITS == 8) ? 255.f : 15.f;
       float s, inv, z;
-      quant_params(mn, mx, s, inv, z);
+      quant_params(mn, mx, s, inv, z, kQmax);
       uint32_t c[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) c[j] = quant_code(x[j], inv, z);
-      const uint32_t word = pack8(c);
+      for (int j = 0; j < 8; ++j) c[j] = quant_code(x[j], inv, z, kQmax);
       if (valid) {
-        *reinterpret_cast<uint32_t*>(d0.v + slot * 32 + 4 * w) = word;
+        if (BITS == 8) {
+          const uint2 words = make_uint2(pack4_bytes(c[0], c[1], c[2], c[3]), pack4_bytes(c[4], c[5], c[6], c[7]));
+          *reinterpret_cast<uint2*>(d0.v + slot * 64 + 8 * w) = words;
+          if (two) *reinterpret_cast<uint2*>(d1.v + slot * 64 + 8 * w) = words;
+        } else {
+          const uint32_t word = pack8(c);
+          *reinterpret_cast<uint32_t*>(d0.v + slot * 32 + 4 * w) = word;
+          if (two) *reinterpret_cast<uint32_t*>(d1.v + slot * 32 + 4 * w) = word;
+        }
         if (w == 0) d0.vpar[slot] = make_float2(s, z);
         if (two) {
-          *reinterpret_cast<uint32_t*>(d1.v + slot * 32 + 4 * w) = word;
           if (w == 0) d1.vpar[slot] = make_float2(s, z);
         }
         if (!ONCE) __stcg(reinterpret_cast<uint4*>(a.kstage + ((size_t)h * a.max_n + tok) * 64 + 8 * w), kv);
@@ -434,8 +451,36 @@ __device__ __forceinline__ void kbar_run(const MaintArgs& a, Shared& sh, const B
     float acc[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    if (BITS == 8) {
+      // 8-bit codes: plain Eq. 10 per channel, parameters (s, z) [H][64] in shared memory
+      __syncthreads();
+      for (int e = tid; e < H * 64; e += kMT) sh.u.kbar.par[e] = __ldcg(&par[(size_t)(e >> 6) * par_stride + (e & 63)]);
+      __syncthreads();
+      for (int h0 = 0; h0 < H; h0 += 8) {
+        uint2 wide8[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          wide8[u] = make_uint2(0u, 0u);
+          if (valid && h0 + u < H) wide8[u] = __ldcg(reinterpret_cast<const uint2*>(b.k + ((size_t)(h0 + u) * cap + slot) * 64 + 8 * w));
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int h = h0 + u;
+          if (h < H) {
+            uint32_t c[8];
+            unpack8_bytes(wide8[u], c);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const float2 sz = sh.u.kbar.par[h * 64 + 8 * w + j];
+              const float x = __fmul_rn(sz.x, __fsub_rn((float)c[j], sz.y));
+              acc[j] = (h == 0) ? x : __fadd_rn(acc[j], x);
+            }
+          }
+        }
+      }
+    }
     constexpr int kHB = (BITS == 4) ? 16 : 4;     // heads whose words are in flight together
-    for (int h0 = 0; h0 < H; h0 += kHB) {
+    for (int h0 = 0; BITS != 8 && h0 < H; h0 += kHB) {
       uint32_t word[BITS == 4 ? kHB : 1];
       uint4 wide[BITS == 4 ? 1 : kHB];
 #pragma unroll
@@ -510,7 +555,9 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+template <int BITS>
 __device__ __forceinline__ void phase_quant_keys_once(const MaintArgs& a, Shared& sh) {
+  constexpr float kQmax = (BITS == 8) ? 255.f : 15.f;
   const BufSet& d0 = a.oth;
   const BufSet& d1 = a.cur;
   const bool two = a.first != 0;
@@ -569,11 +616,11 @@ __device__ __forceinline__ void phase_quant_keys_once(const MaintArgs& a, Shared
 #pragma unroll
       for (int r = 1; r < 4; ++r) { lo = fminf(lo, sh.u.kq.mn[hl][r][t]); hi = fmaxf(hi, sh.u.kq.mx[hl][r][t]); }
       float sc, inv, z;
-      quant_params(lo, hi, sc, inv, z);
+      quant_params(lo, hi, sc, inv, z, kQmax);
       sh.u.kq.iz[hl][t] = make_float2(inv, z);
       float zl, zh, cc;
       dequant_consts(sc, z, zl, zh, cc);
-      const float zo = (((t & 7) >> 1) & 1) ? zh : zl;
+      const float zo = (BITS == 4 && (((t & 7) >> 1) & 1)) ? zh : zl;      // 8-bit codes all carry the bias 1024
       // the neighbouring channel's constants: pairs (2p, 2p + 1) share a word
       const float sc1 = __shfl_xor_sync(0xffffffffu, sc, 1), zo1 = __shfl_xor_sync(0xffffffffu, zo, 1);
       const float cc1 = __shfl_xor_sync(0xffffffffu, cc, 1);
@@ -585,7 +632,7 @@ __device__ __forceinline__ void phase_quant_keys_once(const MaintArgs& a, Shared
           e[4] = pack_half2(zo, zo1);
           e[8] = pack_half2(cc, cc1);
         }
-        if (!(fabsf(sc) * (fabsf(z) + 15.f) <= 65504.f)) atomicCAS(a.status, 0, (int)XKV_E_RANGE);
+        if (!(fabsf(sc) * (fabsf(z) + kQmax) <= 65504.f)) atomicCAS(a.status, 0, (int)XKV_E_RANGE);
       }
     }
     __syncthreads();
@@ -598,11 +645,17 @@ __device__ __forceinline__ void phase_quant_keys_once(const MaintArgs& a, Shared
         if (!live[u]) continue;
         uint32_t c[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) c[j] = quant_code(x[u][j], iz[j].x, iz[j].y);
-        const uint32_t word = pack8(c);
+        for (int j = 0; j < 8; ++j) c[j] = quant_code(x[u][j], iz[j].x, iz[j].y, kQmax);
         const size_t dslot = (size_t)h * cap + a.dst_slot + gamma * 64 + tq + 16 * u;
-        *reinterpret_cast<uint32_t*>(d0.k + dslot * 32 + 4 * w) = word;
-        if (two) *reinterpret_cast<uint32_t*>(d1.k + dslot * 32 + 4 * w) = word;
+        if (BITS == 8) {
+          const uint2 words = make_uint2(pack4_bytes(c[0], c[1], c[2], c[3]), pack4_bytes(c[4], c[5], c[6], c[7]));
+          *reinterpret_cast<uint2*>(d0.k + dslot * 64 + 8 * w) = words;
+          if (two) *reinterpret_cast<uint2*>(d1.k + dslot * 64 + 8 * w) = words;
+        } else {
+          const uint32_t word = pack8(c);
+          *reinterpret_cast<uint32_t*>(d0.k + dslot * 32 + 4 * w) = word;
+          if (two) *reinterpret_cast<uint32_t*>(d1.k + dslot * 32 + 4 * w) = word;
+        }
       }
     }
     if (quad == 0 && tid < 64 && gamma * 64 + tid < n) {
@@ -614,19 +667,23 @@ __device__ __forceinline__ void phase_quant_keys_once(const MaintArgs& a, Shared
 
 // Quantise-once mode: head means (Eq. 4) of the frame just quantised, into the destination's
 // array: one run per arrival group, whose parameters sit in the group's table slot.
+template <int BITS>
 __device__ __forceinline__ void phase_kbar_new_once(const MaintArgs& a, Shared& sh) {
   const int n_groups = (a.n + 63) >> 6;
   const BufSet& d = a.oth;
   for (int gamma = blockIdx.x; gamma < n_groups; gamma += gridDim.x) {
     const int slot = __ldcg(&d.kslot[a.dst_slot + gamma * 64]);
-    kbar_run<4>(a, sh, d, a.ktab32 + (size_t)slot * a.H * 64, 64, a.dst_slot + gamma * 64,
-                a.dst_slot - a.rest_base + gamma * 64, min(64, a.n - gamma * 64));
+    kbar_run<BITS>(a, sh, d, a.ktab32 + (size_t)slot * a.H * 64, 64, a.dst_slot + gamma * 64,
+                   a.dst_slot - a.rest_base + gamma * 64, min(64, a.n - gamma * 64));
   }
 }
 
 // Quantise-once mode, PACK: the survivors' key and value code rows, value parameters, group
 // references, origins and head means move to their new places in the other buffer set.
+template <int BITS>
 __device__ __forceinline__ void phase_gather_once(const MaintArgs& a) {
+  constexpr int kRow = (BITS == 8) ? 64 : 32;       // bytes of a code row
+  constexpr int kRC = kRow / 16;                    // 16-byte chunks of a row
   const BufSet& src = a.cur;
   const BufSet& dst = a.oth;
   const int32_t* kept = a.identity ? nullptr : a.kept;
@@ -642,15 +699,15 @@ __device__ __forceinline__ void phase_gather_once(const MaintArgs& a) {
     return;
   }
   // four items per thread and pass: the kept indices, then the rows, then the stores
-  const long long items = (long long)a.H * a.kk * 4;                 // (head, survivor, 16-byte chunk of K | V codes)
+  const long long items = (long long)a.H * a.kk * (2 * kRC);         // (head, survivor, 16-byte chunk of K | V codes)
   for (long long g0 = first; g0 < items; g0 += 4 * stride) {
     int old[4]; size_t so[4], dd[4]; int chn[4]; bool ok[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const long long g = g0 + u * stride;
       ok[u] = g < items;
-      chn[u] = (int)(g & 3);
-      const long long r = ok[u] ? (g >> 2) : 0;
+      chn[u] = (int)(g % (2 * kRC));
+      const long long r = ok[u] ? (g / (2 * kRC)) : 0;
       const int i = (int)(r % a.kk), h = (int)(r / a.kk);
       old[u] = kept ? __ldcg(&kept[i]) : i;
       dd[u] = (size_t)h * a.cap + a.rest_base + i;
@@ -660,16 +717,16 @@ __device__ __forceinline__ void phase_gather_once(const MaintArgs& a) {
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const size_t s = so[u] + old[u];
-      const uint8_t* base = chn[u] < 2 ? src.k : src.v;
-      row[u] = ok[u] ? *reinterpret_cast<const uint4*>(base + s * 32 + 16 * (chn[u] & 1)) : make_uint4(0, 0, 0, 0);
-      vp[u] = (ok[u] && chn[u] == 2) ? src.vpar[s] : make_float2(0.f, 0.f);
+      const uint8_t* base = chn[u] < kRC ? src.k : src.v;
+      row[u] = ok[u] ? *reinterpret_cast<const uint4*>(base + s * kRow + 16 * (chn[u] % kRC)) : make_uint4(0, 0, 0, 0);
+      vp[u] = (ok[u] && chn[u] == kRC) ? src.vpar[s] : make_float2(0.f, 0.f);
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       if (!ok[u]) continue;
-      uint8_t* base = chn[u] < 2 ? dst.k : dst.v;
-      *reinterpret_cast<uint4*>(base + dd[u] * 32 + 16 * (chn[u] & 1)) = row[u];
-      if (chn[u] == 2) dst.vpar[dd[u]] = vp[u];
+      uint8_t* base = chn[u] < kRC ? dst.k : dst.v;
+      *reinterpret_cast<uint4*>(base + dd[u] * kRow + 16 * (chn[u] % kRC)) = row[u];
+      if (chn[u] == kRC) dst.vpar[dd[u]] = vp[u];
     }
   }
   const long long rows = (long long)a.kk * 16;                       // (survivor, 16-byte chunk of its head-mean row)
@@ -1201,7 +1258,7 @@ __global__ void __launch_bounds__(kMT, kBlocksPerSM) maint_kernel(const __grid_c
 
   if (ph & kPhAppend) {
     phase_append<BITS, ONCE>(a);
-    if (ONCE) phase_quant_keys_once(a, sh);
+    if (ONCE) phase_quant_keys_once<BITS>(a, sh);
     ran = true;
   }
   if (ph & kPhPool) { phase_pool(a, sh); ran = true; }
@@ -1209,7 +1266,7 @@ __global__ void __launch_bounds__(kMT, kBlocksPerSM) maint_kernel(const __grid_c
 
   if (ph & (kPhScore | kPhKbarNew)) {
     if (ran && !grid_barrier(a, epoch, sh)) return;
-    if (ONCE && (ph & kPhKbarNew)) phase_kbar_new_once(a, sh);
+    if (ONCE && (ph & kPhKbarNew)) phase_kbar_new_once<BITS>(a, sh);
     if (ph & kPhScore) phase_score(a, sh);
     ran = true;
   }
@@ -1222,7 +1279,7 @@ __global__ void __launch_bounds__(kMT, kBlocksPerSM) maint_kernel(const __grid_c
   }
   if (ph & kPhPack) {
     if (ran && !grid_barrier(a, epoch, sh)) return;
-    if (ONCE) phase_gather_once(a);
+    if (ONCE) phase_gather_once<BITS>(a);
     else if (BITS == 16 && a.kk > 0) phase_gather16(a);
   }
 }
@@ -1264,8 +1321,8 @@ static cudaError_t maint_grid(int* grid) {
     int sms = 0, per_sm = kBlocksPerSM;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    const void* fns[3] = {(const void*)maint_kernel<4, false>, (const void*)maint_kernel<16, false>,
-                          (const void*)maint_kernel<4, true>};
+    const void* fns[4] = {(const void*)maint_kernel<4, false>, (const void*)maint_kernel<16, false>,
+                          (const void*)maint_kernel<4, true>, (const void*)maint_kernel<8, true>};
     for (const void* fn : fns) {
       int nb = 0;
       e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, fn, kMT, 0);
@@ -1308,6 +1365,7 @@ cudaError_t launch_maint(xkv_cache* c, MaintArgs& a, int prof_cat, cudaStream_t 
   void* params[1] = {(void*)&a};
   a.push_pos = c->counters + 8;
   const void* fn = (c->p.kv_bits == 16) ? (const void*)maint_kernel<16, false>
+                   : (c->p.kv_bits == 8) ? (const void*)maint_kernel<8, true>
                    : c->p.key_mode == XKV_KEYS_ONCE ? (const void*)maint_kernel<4, true>
                                                     : (const void*)maint_kernel<4, false>;
   if (nb > 0) {

@@ -362,8 +362,9 @@ class Cache:
             out["k_val"] = (k[:, sl].astype(np.uint32) << 16).view(np.float32)
             out["v_val"] = (v[:, sl].astype(np.uint32) << 16).view(np.float32)
             return out
-        k = self.xkv_debug_export(BUF_K_CODES, H * cap * d // 2).reshape(H, cap, d // 2)
-        v = self.xkv_debug_export(BUF_V_CODES, H * cap * d // 2).reshape(H, cap, d // 2)
+        rb = d // 2 if self.p.kv_bits == 4 else d          # bytes of a code row
+        k = self.xkv_debug_export(BUF_K_CODES, H * cap * rb).reshape(H, cap, rb)
+        v = self.xkv_debug_export(BUF_V_CODES, H * cap * rb).reshape(H, cap, rb)
         kp = self.xkv_debug_export(BUF_K_PARAMS, H * (cap // 64) * 64 * 8).view(np.float32).reshape(H, cap // 64, d, 2)
         vp = self.xkv_debug_export(BUF_V_PARAMS, H * cap * 8).view(np.float32).reshape(H, cap, 2)
         out["k_packed"], out["v_packed"] = k[:, sl].copy(), v[:, sl].copy()

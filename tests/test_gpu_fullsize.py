@@ -71,18 +71,19 @@ def _stream(xkv, n, budget, frames, seed, attn_from, bits=4, layer=0, via_stream
             err = got.astype(np.float64) - ref
             assert np.abs(err).max() <= ATTN_MAXABS * np.abs(ref).max(), f"frame {t}"
             assert np.linalg.norm(err) <= ATTN_RELL2 * np.linalg.norm(ref), f"frame {t}"
-            # the same frame once more with its own K, V unquantised (Eq. 1 read literally)
-            cache.xkv_debug_rewind_attention()
-            cache.attn_packed_causal_tail(q, k, v, out)
-            Kt = np.concatenate([ora.keys_dequantized()[:, :ora.T - n], kf], axis=1)
-            Vt = np.concatenate([ora.values_dequantized()[:, :ora.T - n], vf], axis=1)
-            ref_t = xo.attention(qf[:, rows], Kt, Vt, scale)
-            got_t = bf16_tensor_to_f32(out)[:, rows]
-            err_t = got_t.astype(np.float64) - ref_t
-            assert np.abs(err_t).max() <= ATTN_MAXABS * np.abs(ref_t).max(), f"frame {t} (tail)"
-            assert np.linalg.norm(err_t) <= ATTN_RELL2 * np.linalg.norm(ref_t), f"frame {t} (tail)"
-            if bits == 4:   # and it is that reading, not the packed one
-                assert np.linalg.norm(err_t) < 0.5 * np.linalg.norm(got_t.astype(np.float64) - ref), f"frame {t}"
+            if bits != 8:       # (the unquantised tail is built for 4-bit and 16-bit caches)
+                # the same frame once more with its own K, V unquantised (Eq. 1 read literally)
+                cache.xkv_debug_rewind_attention()
+                cache.attn_packed_causal_tail(q, k, v, out)
+                Kt = np.concatenate([ora.keys_dequantized()[:, :ora.T - n], kf], axis=1)
+                Vt = np.concatenate([ora.values_dequantized()[:, :ora.T - n], vf], axis=1)
+                ref_t = xo.attention(qf[:, rows], Kt, Vt, scale)
+                got_t = bf16_tensor_to_f32(out)[:, rows]
+                err_t = got_t.astype(np.float64) - ref_t
+                assert np.abs(err_t).max() <= ATTN_MAXABS * np.abs(ref_t).max(), f"frame {t} (tail)"
+                assert np.linalg.norm(err_t) <= ATTN_RELL2 * np.linalg.norm(ref_t), f"frame {t} (tail)"
+                if bits == 4:   # and it is that reading, not the packed one
+                    assert np.linalg.norm(err_t) < 0.5 * np.linalg.norm(got_t.astype(np.float64) - ref), f"frame {t}"
         assert cache.xkv_poll_status() == 0
     return cache, evicting
 
@@ -103,6 +104,12 @@ def test_full_stack_layer_keys_quantised_once(xkv):
     cache, evicting = _stream(xkv, 1374, 16384, 15, seed=3, attn_from=12, via_stream_step=True, key_mode=1)
     info = cache.xkv_get_info()
     assert info.T == 16384 and evicting >= 3 and info.last_evicted == 1374
+
+
+def test_full_stack_layer_8bit_keys_quantised_once(xkv):
+    """The same layer with 8-bit codes (beyond the paper's INT4), quantise-once mode."""
+    cache, evicting = _stream(xkv, 1374, 16384, 14, seed=3, attn_from=12, via_stream_step=True, key_mode=1, bits=8)
+    assert cache.xkv_get_info().T == 16384 and evicting >= 2
 
 
 def test_full_stack_last_layer_through_stream_step(xkv):

@@ -535,3 +535,51 @@ def test_chunked_prefill_is_frame_causal(xkv, bits, key_mode):
         cache.attn_packed_frame_causal(q, [64, 32])              # sizes must add up to what was appended
     cache.attn_packed_frame_causal(q, [64, 64])
     assert cache.xkv_get_info().stage == 0
+
+
+# ------------------------------------------------------------------ 8-bit codes
+@pytest.mark.parametrize("impl", [0, 1])
+def test_tiny_stream_8bit_keys_quantised_once(xkv, impl):
+    """kv_bits = 8 (Eq. 7-8 with 256 levels; the paper evaluates INT4 only) through the quantise-once
+    path: codes (bytes in the order c0, c2, c1, c3 per word), parameters through the table, scores,
+    kept indices bit-exact; attention within the usual tolerance."""
+    p = xkv.Params(budget=1024, max_frame_tokens=261, kv_bits=8, key_mode=xkv.KEYS_ONCE)
+    cache, ora, worst = run_stream(xkv, p, 261, 9, seed=1, impl=impl)
+    assert cache.xkv_get_info().T == 1024
+    print("tiny 8-bit impl", impl, "worst (max-abs, rel-L2)", worst)
+    # 8-bit codes are only built for the quantise-once mode
+    import ctypes as C
+    h = C.c_void_p()
+    bad = xkv.Params(budget=1024, max_frame_tokens=261, kv_bits=8)
+    assert xkv.lib.xkv_create(C.byref(bad.c()), cache.workspace.data_ptr(), 1 << 40, 0, C.byref(h)) == xkv.XKV_E_UNSUPPORTED
+
+
+def test_8bit_ragged_frames_chunks_and_budget_changes(xkv):
+    """8-bit codes with ragged frame sizes and few heads, a capped attention grid, a chunk of frames
+    and a budget change."""
+    import torch
+    from xkv_testlib import compare_state, oracle_params, bf16_tensor_to_f32, check_attention
+    from oracle import xkv_oracle as xo
+    p = xkv.Params(n_heads=3, budget=500, max_frame_tokens=150, kv_bits=8, pool_g=7, n_special=2, key_mode=xkv.KEYS_ONCE)
+    run_stream(xkv, p, [129, 64, 150, 5, 77, 150, 33, 128, 150, 1, 150], 11, seed=5, max_blocks=9)
+    H, d = 4, 64
+    p = xkv.Params(n_heads=H, budget=700, max_frame_tokens=400, kv_bits=8, key_mode=xkv.KEYS_ONCE)
+    cache, ora = xkv.Cache(p), xo.OracleLayer(oracle_params(p))
+    t = 0
+    for ci, chunk in enumerate([[150, 200], [261], [100, 200, 37], [261], [261]]):
+        if ci == 3:
+            cache.xkv_set_budget(500); ora.set_budget(500)
+        fr = [synth.gen_frame(93, 0, t + j, H, n, d) for j, n in enumerate(chunk)]
+        t += len(chunk)
+        qf, kf, vf = ([synth.bf16_bits_to_f32(f[i]) for f in fr] for i in range(3))
+        q, k, v = (to_device_bf16(np.concatenate([f[i] for f in fr], axis=1)) for i in range(3))
+        out = cache.xkv_prefill_chunk(q, k, v, chunk)
+        refs = ora.step_chunk(qf, kf, vf)
+        compare_state(cache.export(), ora.export(), f"chunk {ci}")
+        got = bf16_tensor_to_f32(out).transpose(1, 0, 2)
+        r0 = 0
+        for f, n in enumerate(chunk):
+            check_attention(got[r0:r0 + n], refs[f], f"chunk {ci} frame {f}")
+            r0 += n
+        assert cache.xkv_poll_status() == 0
+    assert cache.xkv_get_info().T == ora.T and ora.last_scores is not None

@@ -132,6 +132,17 @@ def test_nibble_order_vectors_and_roundtrip():
     assert np.array_equal(xo.unpack_nibbles(p), q)
 
 
+def test_byte_order_of_8_bit_codes():
+    """4 channels per little-endian word c0 | c2<<8 | c1<<16 | c3<<24."""
+    codes = np.array([0x11, 0x22, 0x33, 0x44, 1, 2, 3, 4], dtype=np.uint8)
+    p = xo.pack_bytes8(codes)
+    assert p.view("<u4").tolist() == [0x11 | 0x33 << 8 | 0x22 << 16 | 0x44 << 24, 1 | 3 << 8 | 2 << 16 | 4 << 24]
+    w = int(p.view("<u4")[0])
+    assert (w & 0x00FF00FF) == (0x11 | 0x22 << 16) and ((w >> 8) & 0x00FF00FF) == (0x33 | 0x44 << 16)
+    q = _rng(33).integers(0, 256, size=(2, 5, 64)).astype(np.uint8)
+    assert np.array_equal(xo.unpack_bytes8(xo.pack_bytes8(q)), q)
+
+
 # ------------------------------------------------------------------- scores
 def test_pooled_query_shapes_and_partial_group():
     rng = _rng(4)

@@ -44,6 +44,7 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 constexpr int kThreads = 480;
+constexpr int kThreadsSplit = 768;      // 16 softmax warps, 4 producers, 4 for the MMA issuers and the copies
 constexpr int kQRows = 128;
 constexpr int kMaxGrid = 160;                 // CTAs the scratch is sized for (>= SM count of the part)
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -83,7 +84,10 @@ constexpr int kTabBytes = 768 + 2048;
 constexpr int kOffBar = kOffTab + 2 * kTabBytes;  // barriers, tmem base, abort flag
 constexpr int kBarBytes = 512;
 constexpr int kOffRaw = kOffBar + kBarBytes;      // raw stages (16-byte aligned)
-template <int BITS> constexpr int smem_bytes() { return kOffRaw + Cfg<BITS>::kNR * Cfg<BITS>::kRawStage + 1024; }
+constexpr int kXchgBytes = 4096;                  // split softmax: values exchanged between the two halves of a row
+template <int BITS, bool SPLIT = false> constexpr int smem_bytes() {
+  return kOffRaw + Cfg<BITS>::kNR * Cfg<BITS>::kRawStage + (SPLIT ? kXchgBytes : 0) + 1024;
+}
 
 // tensor memory columns (all 512)
 constexpr int kColS = 0;      // + 128 t : 128 fp32 columns per query tile
@@ -148,19 +152,37 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// The same with a time the hardware may keep the thread suspended before it answers "not yet"
+// (it answers at once when the phase completes).
+__device__ __forceinline__ bool mbar_try_suspend(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
 // Bounded wait.  On exhaustion the failure is recorded (device status word and a
 // per-CTA flag); once the flag is up every later wait of the CTA gives up at once.
 struct WaitCtx { int* status; volatile int* abort_flag; };
-// SLEEP_NS: back-off between polls.  Warps that wait long (operand producers, the copy thread)
-// poll rarely so that they do not take issue slots from the softmax warps.
+// The waiting thread is suspended inside the try (up to kSuspendNs at a time) instead of
+// polling with sleeps in between: polls are shared-memory instructions that compete with the
+// softmax warps' tensor-memory traffic and the producers' stores.  The bound is one of time.
+// SLEEP_NS is kept as a template argument for the call sites and is unused.
+constexpr uint32_t kSuspendNs = 2000;
+constexpr uint64_t kWaitLimitNs = 1000000000ull;      // one second, then XKV_E_TIMEOUT
 template <int SLEEP_NS = 32>
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc) {
   if (mbar_try(bar, parity)) return;          // the common case costs one instruction
   if (*wc.abort_flag) return;
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try(bar, parity)) return;
-    __nanosleep(SLEEP_NS);
-  }
+  const uint64_t t0 = global_ns();
+  do {
+    if (mbar_try_suspend(bar, parity, kSuspendNs)) return;
+  } while (global_ns() - t0 < kWaitLimitNs);
   *wc.abort_flag = 1;
   atomicExch(wc.status, (int)XKV_E_TIMEOUT);
 }
@@ -405,9 +427,9 @@ __device__ __forceinline__ void tma_load_1d(uint32_t dst, const void* src, uint3
 }
 // O[row][0..63] *= alpha for the 32 rows (TMEM lanes) of the calling warp; a real call, to keep its
 // registers out of the softmax loop.  Warp-collective.
-__device__ __noinline__ void rescale_rows(uint32_t col_o, float alpha) {
+__device__ __noinline__ void rescale_rows(uint32_t col_o, float alpha, int cols = 64) {
 #pragma unroll 1
-  for (int c0 = 0; c0 < 64; c0 += 32) {
+  for (int c0 = 0; c0 < cols; c0 += 32) {
     uint32_t ra[32];
     XKV_TMEM_LD32(col_o + c0, ra);
     tc_wait_ld();
@@ -425,9 +447,12 @@ __device__ __forceinline__ void producer_sync() { asm volatile("bar.sync 1, 128;
 // instantiation, so that the kernel without a tail carries none of its code).
 // ONCE: the keys' dequantisation constants are looked up per token (quantise-once mode) instead of
 // per 64-slot run.
-template <int BITS, bool TAIL = false, bool ONCE = false>
-__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
+template <int BITS, bool TAIL = false, bool ONCE = false, bool SPLIT = false>
+__global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_kernel(const Args a) {
   using C = Cfg<BITS>;
+  constexpr int kSW = SPLIT ? 16 : 8;        // softmax warps
+  constexpr uint32_t kRowThreads = SPLIT ? 256 : 128;   // threads that work on one query tile
+  constexpr int kOffX = kOffRaw + C::kNR * C::kRawStage;   // exchange area of the split softmax
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
@@ -457,12 +482,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
     for (int i = 0; i < kNV; ++i) { mbar_init(b_vfull + 8 * i, 128); mbar_init(b_vfree + 8 * i, 2); }
     for (int i = 0; i < C::kNR; ++i) { mbar_init(b_rfull + 8 * i, 1); mbar_init(b_rfree + 8 * i, 128); }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(b_qfull + 8 * t, 128); mbar_init(b_sfull + 8 * t, 1);
-      mbar_init(b_pfull + 8 * t, 128); mbar_init(b_pvdone + 8 * t, 1); mbar_init(b_sfree + 8 * t, 128);
+      mbar_init(b_qfull + 8 * t, kRowThreads); mbar_init(b_sfull + 8 * t, 1);
+      mbar_init(b_pfull + 8 * t, kRowThreads); mbar_init(b_pvdone + 8 * t, 1); mbar_init(b_sfree + 8 * t, kRowThreads);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 13) {
+  if (warp == kSW + 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32((const void*)tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -472,7 +497,200 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp < 8) {
+  if (SPLIT) {
+    // Registers move from the warps that need few to the softmax warps, which keep half a row of
+    // scores in registers.  The pool is what the CTA was launched with (per scheduler 6 warps x 80
+    // registers per lane = 480); afterwards 4 x 96 + 40 + 48 = 472 of them are in use.
+    if (warp < 16) asm volatile("setmaxnreg.inc.sync.aligned.u32 96;");
+    else if (warp < 20) asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    else asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+  }
+
+  if (SPLIT && warp < 16) {
+    // ============== softmax warps, two per 32 rows of a query tile ==============
+    // Warps w and w + 8 work on the same rows: each takes 64 of a key tile's 128 score columns, the
+    // matching 32 columns of P and 32 of the accumulator.  A thread reads its half row of scores
+    // into registers at once and releases the score columns, so that the next S = Q K~^T runs while
+    // the exponentials are computed.  What the row needs as a whole (its maximum, its sum) the two
+    // threads exchange through shared memory.
+    const int t = (warp >> 2) & 1;           // query tile of the pair
+    const int hf = warp >> 3;                // half of the key columns
+    const int r = (warp & 3) * 32 + (tid & 31);   // row of the tile = TMEM lane
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t colS = lane_addr + kColS + 128 * t + 64 * hf, colP = lane_addr + kColP + 64 * t + 32 * hf;
+    const uint32_t colO = lane_addr + kColO + 64 * t + 32 * hf;
+    const uint32_t sfull = b_sfull + 8 * t, pfull = b_pfull + 8 * t, pvdone = b_pvdone + 8 * t, sfree = b_sfree + 8 * t;
+    const int pad_tile = (a.t_first & 127) ? (a.t_first >> 7) : -1;
+    const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2);
+    const int pair_bar = 2 + (warp & 7);     // named barrier of the two warps with these rows
+    volatile float* xmine = reinterpret_cast<volatile float*>(sgen + kOffX) + ((t * 2 + hf) * 128 + r);
+    volatile float* xpeer = reinterpret_cast<volatile float*>(sgen + kOffX) + ((t * 2 + (hf ^ 1)) * 128 + r);
+    uint32_t xc = 0;
+    // One value per thread to the thread of the other half with the same row.  Two buffers in turn:
+    // a value is overwritten two exchanges later, after a barrier the reader has passed since.
+    auto exchange = [&](float v) -> float {
+      const uint32_t o = (xc++ & 1) * 512;
+      xmine[o] = v;
+      __syncwarp();
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+      return xpeer[o];
+    };
+    uint32_t cnt = 0;                        // steps this tile has been through (barrier phases)
+    int seg_idx = 0;
+    for (long long pos = step_lo; pos < step_hi; ++seg_idx) {
+      const int item = (int)(pos / a.n_tiles);
+      const int tile_lo = (int)(pos - (long long)item * a.n_tiles);
+      const int nt = (int)min((long long)(a.n_tiles - tile_lo), step_hi - pos);
+      pos += nt;
+      const int h = item / a.n_pairs, pair = item - h * a.n_pairs;
+      const int qt = 2 * pair + t;
+      if (qt >= a.q_tiles) continue;          // the pair has no second tile
+      // ---- Q tile: half of row r, bf16 -> operand type, into the swizzled K-major layout ----
+      const int row = qt * kQRows + r;
+      {
+        uint4 u[4];
+        if (row < a.n) {
+          const __nv_bfloat16* qp = a.q + (int64_t)h * a.hs + (int64_t)row * a.ts + 32 * hf;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) u[c] = *reinterpret_cast<const uint4*>(qp + 8 * c);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) u[c] = make_uint4(0, 0, 0, 0);
+        }
+        bool q_bad = false;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint4 o = u[c];
+          if (!kBf16) {
+            const uint32_t rr[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
+            uint32_t hh[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              hh[i] = pack_h2(__uint_as_float(rr[i] << 16), __uint_as_float(rr[i] & 0xFFFF0000u));
+              q_bad |= h2_not_finite(hh[i]);
+            }
+            o = make_uint4(hh[0], hh[1], hh[2], hh[3]);
+          }
+          *reinterpret_cast<uint4*>(sgen + kOffQ + t * 16384 + swz_off(r, 4 * hf + c)) = o;
+        }
+        if (q_bad) report_range(a.status);
+        fence_proxy_async();
+        mbar_arrive(b_qfull + 8 * t);
+      }
+      float m_ref = -INFINITY;   // reference maximum of the row (scaled, log2 units; the same in both halves)
+      uint64_t l2 = 0ull, l2b = 0ull;   // four partial sums of this half of the row (two packed fp32 pairs)
+      for (int jj = 0; jj < nt; ++jj, ++cnt) {
+        const int tile = tile_lo + jj;
+        int lim = 128;           // columns [lim, 128) are masked (pad slots after the first frame, the tail)
+        if (tile == pad_tile) lim = a.t_first & 127;
+        if (tile == a.n_tiles - 1) lim = min(lim, a.t_phys - tile * 128);
+        mbar_wait(sfull, cnt & 1, wc);
+        __syncwarp();            // the waits may leave the warp diverged; tcgen05.ld/st are warp-collective
+        tc_fence_after();
+        // ---- this half of the scores (64 columns) into registers; after that the score columns
+        // may take the next tile's scores ----
+        uint32_t ra[32], rb[32];
+        XKV_TMEM_LD32(colS, ra);
+        XKV_TMEM_LD32(colS + 32, rb);
+        tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(sfree);
+        if (lim < 128) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            if (64 * hf + i >= lim) ra[i] = 0xff800000u;           // -inf: exponential 0
+            if (64 * hf + 32 + i >= lim) rb[i] = 0xff800000u;
+          }
+        }
+        float mx1 = -INFINITY, mx2 = -INFINITY;      // two chains of 16, not one of 32
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          mx1 = max3(mx1, __uint_as_float(ra[i]), __uint_as_float(ra[i + 1]));
+          mx2 = max3(mx2, __uint_as_float(rb[i]), __uint_as_float(rb[i + 1]));
+        }
+        float mx = fmaxf(mx1, mx2);
+        mx = fmaxf(mx, exchange(mx)) * a.scale_log2;
+        // The reference maximum moves only when the row maximum grew by more than 2^kGrow over it;
+        // then the sums and (at the end of the step, when the registers are free) the accumulator
+        // are rescaled.  Every tile has a column that is not masked, so mx is finite.
+        float alpha = 1.f;
+        const bool grow = mx > m_ref + kGrow;
+        if (grow) {
+          alpha = exp2f(m_ref - mx);      // 0 on the first tile (m_ref = -inf)
+          m_ref = mx;
+          l2 = mul_f2(l2, pack_f2(alpha, alpha));
+          l2b = mul_f2(l2b, pack_f2(alpha, alpha));
+        }
+        const uint64_t nm2 = pack_f2(-m_ref, -m_ref);
+        // exponentials of 16 columns against the reference; P (16-bit pairs) -> TMEM
+        auto chunk16 = [&](const uint32_t* rr, int c) {
+          uint64_t x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            x[i] = fma_f2(pack_f2(__uint_as_float(rr[2 * i]), __uint_as_float(rr[2 * i + 1])), sc2, nm2);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[i] = pack_f2(fast_exp2(f2_lo(x[i])), fast_exp2(f2_hi(x[i])));
+          uint32_t pk[8];
+#pragma unroll
+          for (int i = 0; i < 8; i += 2) {
+            l2 = add_f2(l2, x[i]);
+            l2b = add_f2(l2b, x[i + 1]);
+            pk[i] = kBf16 ? pack_bf2(f2_lo(x[i]), f2_hi(x[i])) : pack_h2(f2_lo(x[i]), f2_hi(x[i]));
+            pk[i + 1] = kBf16 ? pack_bf2(f2_lo(x[i + 1]), f2_hi(x[i + 1])) : pack_h2(f2_lo(x[i + 1]), f2_hi(x[i + 1]));
+          }
+          if (c == 0 && jj > 0) {  // P of the previous step consumed, O quiescent (its PV completed)
+            mbar_wait(pvdone, (cnt - 1) & 1, wc);
+            __syncwarp();
+            tc_fence_after();
+          }
+          XKV_TMEM_ST8(colP + 8 * c, pk);
+        };
+        chunk16(ra, 0);
+        chunk16(ra + 16, 1);
+        chunk16(rb, 2);
+        chunk16(rb + 16, 3);
+        if (jj > 0 && __any_sync(0xffffffffu, grow)) rescale_rows(colO, alpha, 32);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(pfull);
+      }
+      // ---- epilogue of the segment: 32 channels of the row per thread ----
+      mbar_wait(pvdone, (cnt - 1) & 1, wc);
+      __syncwarp();
+      tc_fence_after();
+      const float l_half = (f2_lo(l2) + f2_hi(l2)) + (f2_lo(l2b) + f2_hi(l2b));
+      const float l_peer = exchange(l_half);
+      const float l = hf ? (l_peer + l_half) : (l_half + l_peer);     // the same sum in both halves
+      const bool whole = (tile_lo == 0 && nt == a.n_tiles);
+      uint32_t ro[32];
+      XKV_TMEM_LD32(colO, ro);
+      tc_wait_ld();
+      if (whole) {
+        const float inv_l = 1.f / l;
+        if (row < a.n) {
+          __nv_bfloat16* op = a.out + (int64_t)h * a.hs + (int64_t)row * a.ts + 32 * hf;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              o[i] = pack_bf2(__uint_as_float(ro[8 * c + 2 * i]) * inv_l, __uint_as_float(ro[8 * c + 2 * i + 1]) * inv_l);
+            *reinterpret_cast<uint4*>(op + 8 * c) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+        }
+      } else {
+        const size_t slot = (size_t)2 * blockIdx.x + (seg_idx == 0 ? 0 : 1);
+        const size_t prow = (slot * 2 + t) * 128 + r;
+        float4* dst = reinterpret_cast<float4*>(a.part_o + prow * 64 + 32 * hf);
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          dst[c] = make_float4(__uint_as_float(ro[4 * c]), __uint_as_float(ro[4 * c + 1]),
+                               __uint_as_float(ro[4 * c + 2]), __uint_as_float(ro[4 * c + 3]));
+        if (hf == 0) a.part_ml[prow] = make_float2(m_ref, l);
+      }
+      tc_fence_before();
+    }
+  } else if (!SPLIT && warp < 8) {
     // =========================== softmax warps ===============================
     const int t = warp >> 2;                 // query tile of the pair
     const int r = tid & 127;                 // row of the tile = TMEM lane
@@ -720,9 +938,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
       }
       tc_fence_before();
     }
-  } else if (warp < 12) {
+  } else if (warp < kSW + 4) {
     // =========================== operand producers ===========================
-    const int t = tid - 256;
+    const int t = tid - 32 * kSW;
     const int w = t & 7;          // 16-byte chunk = 8 channels
     const int kb = t >> 3;        // keys kb + 16 i
     const uint32_t row_off = (uint32_t)((kb >> 3) * 1024 + (kb & 7) * 128 + ((w ^ (kb & 7)) << 4));
@@ -920,11 +1138,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
         }
       }
     }
-  } else if (tid == 384 || tid == 448) {
+  } else if (tid == 32 * (kSW + 4) || tid == 32 * (kSW + 6)) {
     // =========================== MMA issuers ==================================
     // One thread per query tile.  Both release the K~/V~ stages (two arrivals each), also for an
     // item that has no second tile: then the second thread only follows the rings.
-    const int t = (tid == 448) ? 1 : 0;
+    const int t = (tid == 32 * (kSW + 6)) ? 1 : 0;
     const uint32_t idesc_qk = make_idesc(128, kBf16, false);
     const uint32_t idesc_pv = make_idesc(64, kBf16, true);
     const uint64_t dq = make_desc(sQ + t * 16384);
@@ -973,7 +1191,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
     // all MMAs must be done before the CTA may free tensor memory: the softmax warps have waited
     // for every PV (pvdone) before their epilogues, and every QK (sfull) before that.
     tc_fence_before();
-  } else if (tid == 416) {
+  } else if (tid == 32 * (kSW + 5)) {
     // =========================== TMA loader ===================================
     uint32_t g = 0;
     for (long long pos = step_lo; pos < step_hi;) {
@@ -1019,7 +1237,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const Args a) {
     }
   }
   __syncthreads();
-  if (warp == 13) {
+  if (warp == kSW + 5) {
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -1123,6 +1341,8 @@ static cudaError_t attn_device_setup(int* sm_count) {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_tc_kernel<4, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4, true>());
+    if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<16>());
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
@@ -1197,7 +1417,7 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
     else if (a.k_tail && once) attn_tc_kernel<4, true, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
     else if (a.k_tail) attn_tc_kernel<4, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
     else if (once) attn_tc_kernel<4, false, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
-    else attn_tc_kernel<4><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
+    else attn_tc_kernel<4, false, false, true><<<(int)grid, kThreadsSplit, smem_bytes<4, true>(), st>>>(a);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }

@@ -453,6 +453,8 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
   constexpr int kSW = SPLIT ? 16 : 8;        // softmax warps
   constexpr uint32_t kRowThreads = SPLIT ? 256 : 128;   // threads that work on one query tile
   constexpr int kOffX = kOffRaw + C::kNR * C::kRawStage;   // exchange area of the split softmax
+  constexpr int kRegProd = (ONCE || TAIL) ? 56 : 40;      // registers per thread after the reallocation:
+  constexpr int kRegMisc = (ONCE || TAIL) ? 40 : 48;      // producers; MMA issuers and copy thread
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
@@ -500,10 +502,11 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
   if (SPLIT) {
     // Registers move from the warps that need few to the softmax warps, which keep half a row of
     // scores in registers.  The pool is what the CTA was launched with (per scheduler 6 warps x 80
-    // registers per lane = 480); afterwards 4 x 96 + 40 + 48 = 472 of them are in use.
+    // registers per lane = 480); afterwards 4 x 96 + 40 + 48 (or 56 + 40 where the producers look up
+    // per-token constants) of them are in use: 472 or 480.
     if (warp < 16) asm volatile("setmaxnreg.inc.sync.aligned.u32 96;");
-    else if (warp < 20) asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
-    else asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+    else if (warp < 20) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegProd));
+    else asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegMisc));
   }
 
   if (SPLIT && warp < 16) {
@@ -991,33 +994,33 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
           for (int i = 0; i < 8; ++i) wd[i] = *reinterpret_cast<const uint32_t*>(raw + (kb + 16 * i) * 32 + 4 * w);
           if (ONCE) {
             // constants of each token's own key group, from the table in global memory (the tokens of
-            // a group mostly sit next to each other, so the lines are shared); four tokens at a time
-            int sl[8];
+            // a group mostly sit next to each other, so the lines are shared); two tokens at a time,
+            // the next two fetched while these are dequantised
+            const uint8_t* slp = raw + C::kRawK + C::kRawV + 4 * kb;      // group references of keys kb + 16 i
+            auto entry = [&](int i) {
+              const int sl = *reinterpret_cast<const int*>(slp + 64 * i);
+              return reinterpret_cast<const uint4*>(a.ktab16 + (((size_t)sl * a.n_heads + h) * 8 + w) * 12);
+            };
+            uint4 sv[2], zv[2], cv[2];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) sl[i] = *reinterpret_cast<const int*>(raw + C::kRawK + C::kRawV + 4 * (kb + 16 * i));
-            uint4 sv[4], zv[4], cv[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const uint4* e = reinterpret_cast<const uint4*>(a.ktab16 + (((size_t)sl[i] * a.n_heads + h) * 8 + w) * 12);
-              sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2);
-            }
+            for (int i = 0; i < 2; ++i) { const uint4* e = entry(i); sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2); }
             mbar_wait<256>(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
+            for (int q2 = 0; q2 < 4; ++q2) {
+              uint4 o[2];
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
+              for (int i = 0; i < 2; ++i) {
                 const uint32_t s2[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w}, zo[4] = {zv[i].x, zv[i].y, zv[i].z, zv[i].w};
                 const uint32_t c2[4] = {cv[i].x, cv[i].y, cv[i].z, cv[i].w};
-                const uint4 o = dequant_word_h(wd[4 * half + i], s2, zo, c2);
-                *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (4 * half + i) * 2048) = o;
+                o[i] = dequant_word_h(wd[2 * q2 + i], s2, zo, c2);
               }
-              if (half == 0) {
+              if (q2 < 3) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const uint4* e = reinterpret_cast<const uint4*>(a.ktab16 + (((size_t)sl[4 + i] * a.n_heads + h) * 8 + w) * 12);
-                  sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2);
-                }
+                for (int i = 0; i < 2; ++i) { const uint4* e = entry(2 * q2 + 2 + i); sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2); }
               }
+#pragma unroll
+              for (int i = 0; i < 2; ++i)
+                *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (2 * q2 + i) * 2048) = o[i];
             }
           } else {
           mbar_wait<256>(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
@@ -1073,32 +1076,31 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
           uint2 wd8[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) wd8[i] = *reinterpret_cast<const uint2*>(raw + (kb + 16 * i) * 64 + 8 * w);
-          int sl[8];
+          const uint8_t* slp = raw + C::kRawK + C::kRawV + 4 * kb;      // group references of keys kb + 16 i
+          auto entry = [&](int i) {
+            const int sl = *reinterpret_cast<const int*>(slp + 64 * i);
+            return reinterpret_cast<const uint4*>(a.ktab16 + (((size_t)sl * a.n_heads + h) * 8 + w) * 12);
+          };
+          uint4 sv[2], zv[2], cv[2];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) sl[i] = *reinterpret_cast<const int*>(raw + C::kRawK + C::kRawV + 4 * (kb + 16 * i));
-          uint4 sv[4], zv[4], cv[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint4* e = reinterpret_cast<const uint4*>(a.ktab16 + (((size_t)sl[i] * a.n_heads + h) * 8 + w) * 12);
-            sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2);
-          }
+          for (int i = 0; i < 2; ++i) { const uint4* e = entry(i); sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2); }
           mbar_wait<256>(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
+          for (int q2 = 0; q2 < 4; ++q2) {
+            uint4 o[2];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < 2; ++i) {
               const uint32_t s2[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w}, zo[4] = {zv[i].x, zv[i].y, zv[i].z, zv[i].w};
               const uint32_t c2[4] = {cv[i].x, cv[i].y, cv[i].z, cv[i].w};
-              const uint4 o = dequant_words8_h(wd8[4 * half + i], s2, zo, c2);
-              *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (4 * half + i) * 2048) = o;
+              o[i] = dequant_words8_h(wd8[2 * q2 + i], s2, zo, c2);
             }
-            if (half == 0) {
+            if (q2 < 3) {
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const uint4* e = reinterpret_cast<const uint4*>(a.ktab16 + (((size_t)sl[4 + i] * a.n_heads + h) * 8 + w) * 12);
-                sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2);
-              }
+              for (int i = 0; i < 2; ++i) { const uint4* e = entry(2 * q2 + 2 + i); sv[i] = __ldg(e); zv[i] = __ldg(e + 1); cv[i] = __ldg(e + 2); }
             }
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+              *reinterpret_cast<uint4*>(sgen + kOffK + kbuf * 16384 + row_off + (2 * q2 + i) * 2048) = o[i];
           }
           fence_proxy_async();
           mbar_arrive(b_kfull + 8 * kbuf);
@@ -1339,13 +1341,11 @@ static cudaError_t attn_device_setup(int* sm_count) {
     int sms = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
-    if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<4, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4, true>());
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<16>());
+    e = cudaFuncSetAttribute(attn_tc_kernel<16, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<16, true>());
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_tc_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
+    e = cudaFuncSetAttribute(attn_tc_kernel<4, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4, true>());
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<4, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
     if (e != cudaSuccess) return e;
@@ -1412,12 +1412,16 @@ static cudaError_t launch_attn_tc_on(xkv_cache* c, const void* q, void* out, int
   {
     LaunchScope ls(c, XKV_PROF_ATTN, st);
     const bool once = c->p.key_mode == XKV_KEYS_ONCE;
-    if (c->p.kv_bits == 16) attn_tc_kernel<16><<<(int)grid, kThreads, smem_bytes<16>(), st>>>(a);
+    // The 16-warp softmax where the producers have registers to spare for it; with per-token
+    // constants (keys quantised once, 8-bit codes) the producers need theirs and the 8-warp
+    // softmax measured faster.
+    const int T = kThreadsSplit;
+    if (c->p.kv_bits == 16) attn_tc_kernel<16, false, false, true><<<(int)grid, T, smem_bytes<16, true>(), st>>>(a);
     else if (c->p.kv_bits == 8) attn_tc_kernel<8, false, true><<<(int)grid, kThreads, smem_bytes<8>(), st>>>(a);
     else if (a.k_tail && once) attn_tc_kernel<4, true, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
-    else if (a.k_tail) attn_tc_kernel<4, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
+    else if (a.k_tail) attn_tc_kernel<4, true, false, true><<<(int)grid, T, smem_bytes<4, true>(), st>>>(a);
     else if (once) attn_tc_kernel<4, false, true><<<(int)grid, kThreads, smem_bytes<4>(), st>>>(a);
-    else attn_tc_kernel<4, false, false, true><<<(int)grid, kThreadsSplit, smem_bytes<4, true>(), st>>>(a);
+    else attn_tc_kernel<4, false, false, true><<<(int)grid, T, smem_bytes<4, true>(), st>>>(a);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }

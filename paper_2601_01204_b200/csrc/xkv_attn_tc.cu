@@ -152,6 +152,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+constexpr uint32_t kSuspendNs = 2000;
 // The same with a time the hardware may keep the thread suspended before it answers "not yet"
 // (it answers at once when the phase completes).
 __device__ __forceinline__ bool mbar_try_suspend(uint32_t bar, uint32_t parity, uint32_t ns) {
@@ -159,6 +160,23 @@ __device__ __forceinline__ bool mbar_try_suspend(uint32_t bar, uint32_t parity, 
   asm volatile(
       "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+  return ok != 0;
+}
+// Up to 64 suspended tries in a loop of three instructions (try, branch out, count and branch back).
+__device__ __forceinline__ bool mbar_try_many(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .pred q;\n\t.reg .u32 n;\n\t"
+      "mov.u32 n, 64;\n\t"
+      "XKV_TRY_%=:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "@p bra XKV_DONE_%=;\n\t"
+      "sub.u32 n, n, 1;\n\t"
+      "setp.ne.u32 q, n, 0;\n\t"
+      "@q bra XKV_TRY_%=;\n\t"
+      "XKV_DONE_%=:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
   return ok != 0;
 }
 __device__ __forceinline__ uint64_t global_ns() {
@@ -169,11 +187,11 @@ __device__ __forceinline__ uint64_t global_ns() {
 // Bounded wait.  On exhaustion the failure is recorded (device status word and a
 // per-CTA flag); once the flag is up every later wait of the CTA gives up at once.
 struct WaitCtx { int* status; volatile int* abort_flag; };
-// The waiting thread is suspended inside the try (up to kSuspendNs at a time) instead of
-// polling with sleeps in between: polls are shared-memory instructions that compete with the
-// softmax warps' tensor-memory traffic and the producers' stores.  The bound is one of time.
-// SLEEP_NS is kept as a template argument for the call sites and is unused.
-constexpr uint32_t kSuspendNs = 2000;
+// Threads on the critical chain (softmax warps, MMA issuers: SLEEP_NS below 128) retry at once, each
+// try suspended by the hardware for a short while: their wake-up latency is part of every step.
+// Threads that wait long and have slack (operand producers, the copy thread) sleep SLEEP_NS between
+// tries, so that their polls (shared-memory instructions) do not take issue slots and queue space
+// from the softmax warps.  The bound is one of time, looked at every 32 tries.
 constexpr uint64_t kWaitLimitNs = 1000000000ull;      // one second, then XKV_E_TIMEOUT
 template <int SLEEP_NS = 32>
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc) {
@@ -181,7 +199,15 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const W
   if (*wc.abort_flag) return;
   const uint64_t t0 = global_ns();
   do {
-    if (mbar_try_suspend(bar, parity, kSuspendNs)) return;
+    if (SLEEP_NS >= 128) {
+#pragma unroll 1
+      for (int it = 0; it < 32; ++it) {
+        if (mbar_try_suspend(bar, parity, kSuspendNs)) return;
+        __nanosleep(SLEEP_NS);
+      }
+    } else if (mbar_try_many(bar, parity)) {
+      return;
+    }
   } while (global_ns() - t0 < kWaitLimitNs);
   *wc.abort_flag = 1;
   atomicExch(wc.status, (int)XKV_E_TIMEOUT);

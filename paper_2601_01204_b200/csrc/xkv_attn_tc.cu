@@ -93,6 +93,9 @@ template <int BITS, bool SPLIT = false> constexpr int smem_bytes() {
 constexpr int kColS = 0;      // + 128 t : 128 fp32 columns per query tile
 constexpr int kColP = 256;    // + 64 t  : 64 columns of packed 16-bit pairs
 constexpr int kColO = 384;    // + 64 t  : 64 fp32 columns
+// 16-warp form: one score buffer for both tiles, two P buffers per tile
+constexpr int kColS1 = 0;     // 128 fp32 columns
+constexpr int kColP2 = 128;   // + 128 t + 64 b
 constexpr int kTmemCols = 512;
 
 // one partial slot: two query tiles x 128 rows x (64 accumulators + max + sum)
@@ -492,6 +495,7 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
   const uint32_t b_rfull = b_vfree + 8 * kNV, b_rfree = b_rfull + 8 * C::kNR;
   const uint32_t b_qfull = b_rfree + 8 * C::kNR;      // [2]
   const uint32_t b_sfull = b_qfull + 16, b_pfull = b_sfull + 16, b_pvdone = b_pfull + 16, b_sfree = b_pvdone + 16;
+  const uint32_t b_pvdone2 = b_sfree + 16;             // [2 tiles][2 P buffers], 16-warp form
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sgen + kOffBar + kBarBytes - 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sgen + kOffBar + kBarBytes - 12);
   const WaitCtx wc{a.status, abort_flag};
@@ -512,6 +516,7 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
     for (int t = 0; t < 2; ++t) {
       mbar_init(b_qfull + 8 * t, kRowThreads); mbar_init(b_sfull + 8 * t, 1);
       mbar_init(b_pfull + 8 * t, kRowThreads); mbar_init(b_pvdone + 8 * t, 1); mbar_init(b_sfree + 8 * t, kRowThreads);
+      mbar_init(b_pvdone2 + 16 * t, 1); mbar_init(b_pvdone2 + 16 * t + 8, 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -546,9 +551,11 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
     const int hf = warp >> 3;                // half of the key columns
     const int r = (warp & 3) * 32 + (tid & 31);   // row of the tile = TMEM lane
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t colS = lane_addr + kColS + 128 * t + 64 * hf, colP = lane_addr + kColP + 64 * t + 32 * hf;
+    // tensor memory of this form: one score buffer that the two tiles use in turn (a tile holds it
+    // only from its MMAs to its loads), two P buffers per tile, one accumulator per tile
+    const uint32_t colS = lane_addr + kColS1 + 64 * hf, colP0 = lane_addr + kColP2 + 128 * t + 32 * hf;
     const uint32_t colO = lane_addr + kColO + 64 * t + 32 * hf;
-    const uint32_t sfull = b_sfull + 8 * t, pfull = b_pfull + 8 * t, pvdone = b_pvdone + 8 * t, sfree = b_sfree + 8 * t;
+    const uint32_t sfull = b_sfull + 8 * t, pfull = b_pfull + 8 * t, pvdone2 = b_pvdone2 + 16 * t;
     const int pad_tile = (a.t_first & 127) ? (a.t_first >> 7) : -1;
     const uint64_t sc2 = pack_f2(a.scale_log2, a.scale_log2);
     const int pair_bar = 2 + (warp & 7);     // named barrier of the two warps with these rows
@@ -565,6 +572,7 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
       return xpeer[o];
     };
     uint32_t cnt = 0;                        // steps this tile has been through (barrier phases)
+    uint32_t g_seg = 0;                      // uses of the score buffer (both tiles) before this segment
     int seg_idx = 0;
     for (long long pos = step_lo; pos < step_hi; ++seg_idx) {
       const int item = (int)(pos / a.n_tiles);
@@ -573,6 +581,9 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
       pos += nt;
       const int h = item / a.n_pairs, pair = item - h * a.n_pairs;
       const int qt = 2 * pair + t;
+      const uint32_t per_step = (2 * pair + 1 < a.q_tiles) ? 2u : 1u;   // tiles that use the score buffer
+      const uint32_t use0 = g_seg + (uint32_t)t;     // this tile's uses: use0 + jj * per_step
+      g_seg += (uint32_t)nt * per_step;
       if (qt >= a.q_tiles) continue;          // the pair has no second tile
       // ---- Q tile: half of row r, bf16 -> operand type, into the swizzled K-major layout ----
       const int row = qt * kQRows + r;
@@ -623,7 +634,7 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
         XKV_TMEM_LD32(colS + 32, rb);
         tc_wait_ld();
         tc_fence_before();
-        mbar_arrive(sfree);
+        mbar_arrive(b_sfree + 8 * ((use0 + (uint32_t)jj * per_step) & 1));    // uses alternate between two barriers
         if (lim < 128) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
@@ -651,6 +662,7 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
           l2b = mul_f2(l2b, pack_f2(alpha, alpha));
         }
         const uint64_t nm2 = pack_f2(-m_ref, -m_ref);
+        const uint32_t colP = colP0 + 64 * (cnt & 1);
         // exponentials of 16 columns against the reference; P (16-bit pairs) -> TMEM
         auto chunk16 = [&](const uint32_t* rr, int c) {
           uint64_t x[8];
@@ -667,8 +679,8 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
             pk[i] = kBf16 ? pack_bf2(f2_lo(x[i]), f2_hi(x[i])) : pack_h2(f2_lo(x[i]), f2_hi(x[i]));
             pk[i + 1] = kBf16 ? pack_bf2(f2_lo(x[i + 1]), f2_hi(x[i + 1])) : pack_h2(f2_lo(x[i + 1]), f2_hi(x[i + 1]));
           }
-          if (c == 0 && jj > 0) {  // P of the previous step consumed, O quiescent (its PV completed)
-            mbar_wait(pvdone, (cnt - 1) & 1, wc);
+          if (c == 0 && cnt >= 2) {  // this P buffer's previous contents (two steps ago) consumed
+            mbar_wait(pvdone2 + 8 * (cnt & 1), ((cnt >> 1) - 1) & 1, wc);
             __syncwarp();
             tc_fence_after();
           }
@@ -678,13 +690,19 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
         chunk16(ra + 16, 1);
         chunk16(rb, 2);
         chunk16(rb + 16, 3);
-        if (jj > 0 && __any_sync(0xffffffffu, grow)) rescale_rows(colO, alpha, 32);
+        if (jj > 0 && __any_sync(0xffffffffu, grow)) {
+          // the accumulator is quiescent once the previous step's PV has completed
+          mbar_wait(pvdone2 + 8 * ((cnt - 1) & 1), ((cnt - 1) >> 1) & 1, wc);
+          __syncwarp();
+          tc_fence_after();
+          rescale_rows(colO, alpha, 32);
+        }
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(pfull);
       }
       // ---- epilogue of the segment: 32 channels of the row per thread ----
-      mbar_wait(pvdone, (cnt - 1) & 1, wc);
+      mbar_wait(pvdone2 + 8 * ((cnt - 1) & 1), ((cnt - 1) >> 1) & 1, wc);    // the last PV (they complete in order)
       __syncwarp();
       tc_fence_after();
       const float l_half = (f2_lo(l2) + f2_hi(l2)) + (f2_lo(l2b) + f2_hi(l2b));
@@ -1166,7 +1184,74 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
         }
       }
     }
-  } else if (tid == 32 * (kSW + 4) || tid == 32 * (kSW + 6)) {
+  } else if (SPLIT && (tid == 32 * (kSW + 4) || tid == 32 * (kSW + 6))) {
+    // =========================== MMA issuers, 16-warp form ====================
+    // One thread per query tile, products in program order (S of step j, then P V~ of step j - 1).
+    // The two tiles share one score buffer: its uses are numbered in the order tile 0, tile 1,
+    // tile 0, ... (tile 0 alone where the item has no second tile), and use G is issued once the
+    // softmax warps have loaded use G - 1.  Even and odd uses are released on two barriers: the
+    // barrier of use G - 1 cannot complete again before use G + 1 has been issued, and a thread
+    // waits for uses that are at most two apart, so a parity wait is never two phases off.
+    const int t = (tid == 32 * (kSW + 6)) ? 1 : 0;
+    const uint32_t idesc_qk = make_idesc(128, kBf16, false);
+    const uint32_t idesc_pv = make_idesc(64, kBf16, true);
+    const uint64_t dq = make_desc(sQ + t * 16384);
+    const uint32_t d_s = tmem + kColS1, d_p0 = tmem + kColP2 + 128 * t, d_o = tmem + kColO + 64 * t;
+    uint32_t g = 0, cq = 0, cp = 0, segq = 0;
+    uint32_t g_seg = 0;              // score-buffer uses before this segment
+    for (long long pos = step_lo; pos < step_hi;) {
+      const int item = (int)(pos / a.n_tiles);
+      const int tile_lo = (int)(pos - (long long)item * a.n_tiles);
+      const int nt = (int)min((long long)(a.n_tiles - tile_lo), step_hi - pos);
+      pos += nt;
+      const int pair = item % a.n_pairs;
+      const bool active = 2 * pair + t < a.q_tiles;
+      const uint32_t per_step = (2 * pair + 1 < a.q_tiles) ? 2u : 1u;     // tiles that use the score buffer
+      auto issue_pv = [&](uint32_t gv, bool first_of_segment) {
+        mbar_wait(b_vfull + 8 * (gv % kNV), (gv / kNV) & 1, wc);
+        if (active) {
+          mbar_wait(b_pfull + 8 * t, cp & 1, wc);               // P_t of that step written
+          tc_fence_after();
+          const uint64_t dv = make_desc(sV + (gv % kNV) * 16384);
+          const uint32_t d_p = d_p0 + 64 * (cp & 1);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)   // 16 keys per step: 2 swizzle atoms = 2048 B of V~, 8 columns of P
+            mma_ts(d_o, d_p + 8 * ks, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv,
+                   (!first_of_segment || ks > 0) ? 1u : 0u);
+          tc_commit(b_pvdone2 + 16 * t + 8 * (cp & 1));
+          ++cp;
+        }
+        tc_commit(b_vfree + 8 * (gv % kNV));
+      };
+      for (int jj = 0; jj < nt; ++jj, ++g) {
+        mbar_wait(b_kfull + 8 * (g % kNK), (g / kNK) & 1, wc);
+        if (active) {
+          const uint32_t use = g_seg + (uint32_t)jj * per_step + (uint32_t)t;
+          if (use > 0) mbar_wait(b_sfree + 8 * ((use - 1) & 1), ((use - 1) >> 1) & 1, wc);   // use - 1 is in registers
+          if (jj == 0) mbar_wait(b_qfull + 8 * t, segq & 1, wc);
+          tc_fence_after();
+          const uint64_t dk = make_desc(sK + (g % kNK) * 16384);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)   // 16 channels per step: 32 B inside the swizzle span
+            mma_ss(d_s, dq + (uint64_t)(ks * 2), dk + (uint64_t)(ks * 2), idesc_qk, ks > 0 ? 1u : 0u);
+          tc_commit(b_sfull + 8 * t);
+          ++cq;
+        } else {
+          // An item without a second tile: this thread follows the other tile's uses of the score
+          // buffer one by one.  A parity wait is only sound while the waiter is at most one
+          // completion ahead of the barrier, so no use may be skipped.
+          const uint32_t use = g_seg + (uint32_t)jj;
+          if (use > 0) mbar_wait(b_sfree + 8 * ((use - 1) & 1), ((use - 1) >> 1) & 1, wc);
+        }
+        tc_commit(b_kfree + 8 * (g % kNK));
+        if (jj > 0) issue_pv(g - 1, jj == 1);
+      }
+      issue_pv(g - 1, nt == 1);           // the last PV of the segment
+      g_seg += (uint32_t)nt * per_step;
+      if (active) ++segq;
+    }
+    tc_fence_before();
+  } else if (!SPLIT && (tid == 32 * (kSW + 4) || tid == 32 * (kSW + 6))) {
     // =========================== MMA issuers ==================================
     // One thread per query tile.  Both release the K~/V~ stages (two arrivals each), also for an
     // item that has no second tile: then the second thread only follows the rings.

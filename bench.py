@@ -29,7 +29,7 @@ METRIC = "stream frames/s (24-layer compressed-KV attention)"
 UNIT = "frames/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture
 # summarised under profiles/ (None until a capture of the current kernel exists).
-ATTN_DRAM_TRAFFIC_BYTES = 23.5e6
+ATTN_DRAM_TRAFFIC_BYTES = 23.3e6
 
 
 def _peaks() -> dict:

@@ -8,29 +8,33 @@
 // not cover an item completely leaves partial results (accumulator, running max
 // and sum) in a scratch slot; a second kernel merges them.
 //
-// One CTA, 15 warps:
-//   warps 0-3   softmax of query tile 0: thread r owns query row r = TMEM lane r.
-//               Reads S from tensor memory, online max/sum, writes P (16-bit) back
-//               to tensor memory, rescales O only when the running maximum grew by
-//               more than 2^14, epilogue.
-//   warps 4-7   the same for query tile 1.  The two groups alternate naturally:
-//               while one computes exponentials the tensor pipe produces the
-//               other's scores.
-//   warps 8-11  operand producers: packed 4-bit codes (raw, as copied by TMA) ->
-//               fp16 K~ (per channel and 64-slot group) and V~ (per token) in the
-//               128-byte-swizzled layouts the MMA descriptors expect.  One
-//               dequantised tile serves both query tiles.
-//   warps 12,14 one thread each issues the MMAs of query tile 0 resp. 1:
+// One CTA.  The roles are the same in both forms of the kernel; the softmax comes in two:
+//   softmax, 8 warps (SPLIT = false, 15 warps in all): warps 0-3 query tile 0, warps 4-7 query
+//               tile 1; thread r owns query row r = TMEM lane r.  Reads S from tensor memory
+//               chunk by chunk, online max/sum in one pass, writes P (16-bit) back to tensor
+//               memory, rescales O only when the running maximum grew by more than 2^14.
+//               Tensor memory: S 2 x 128 columns, P 2 x 64, O 2 x 64.
+//   softmax, 16 warps (SPLIT = true, 24 warps in all): warps w and w + 8 share the rows of a
+//               lane quarter, each takes 64 of the 128 key columns; a thread loads its half row
+//               of scores into registers at once and releases the score columns, the maximum
+//               is taken from the registers.  Registers move to these warps with setmaxnreg.
+//               Tensor memory: ONE score buffer of 128 columns that the two tiles use in turn,
+//               P 2 x 2 x 64 (two buffers per tile), O 2 x 64.
+//   4 warps     operand producers: packed codes (raw, as copied by TMA) -> fp16 K~ (per channel
+//               and key group) and V~ (per token) in the 128-byte-swizzled layouts the MMA
+//               descriptors expect.  One dequantised tile serves both query tiles.
+//   2 threads   (in warps of their own) issue the MMAs of query tile 0 resp. 1:
 //               S_t = Q_t K~^T (M128 N128 K64) and O_t += P_t V~ (M128 N64 K128,
-//               A = P from tensor memory).  A single issuing thread for both tiles
-//               was the bottleneck of the CTA.
-//   warp 13     one thread issues the bulk copies of the raw tiles, several steps
-//               ahead; the warp owns the tensor-memory allocation (all 512 columns).
+//               A = P from tensor memory).  A thread gets one tcgen05.mma through about every
+//               125 cycles whatever its shape; a single issuing thread for both tiles was the
+//               bottleneck of the CTA.
+//   1 thread    issues the bulk copies of the raw tiles, several steps ahead; its warp owns the
+//               tensor-memory allocation (all 512 columns).
 // 4-bit caches multiply in fp16 (the dequantised keys are not bf16-representable:
 // rounding them to bf16 alone costs ~1e-2 relative L2 with outlier channels);
 // 16-bit caches hold bf16 and multiply in bf16.  Accumulation is fp32.
 //
-// Every mbarrier wait is bounded: when the bound is hit the thread records
+// Every mbarrier wait is bounded (by time: one second): when the bound is hit the thread records
 // XKV_E_TIMEOUT in the cache's status word and carries on without waiting, so the
 // kernel always terminates, drains its copies and frees its tensor memory.
 #include <mutex>

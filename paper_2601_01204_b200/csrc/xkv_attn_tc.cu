@@ -1012,6 +1012,32 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
         const uint32_t vbuf = g % kNV, vu = g / kNV;
         const uint8_t* raw = sgen + kOffRaw + rs * C::kRawStage;
         mbar_wait<256>(b_rfull + 8 * rs, ru & 1, wc);
+        if (TAIL && BITS == 4 && (tile_lo + jj) * 128 >= a.tail_lo && (tile_lo + jj) * 128 + 127 < a.t_phys) {
+          // ---- a tile that lies in the unquantised frame as a whole: K~ and V~ are the caller's
+          // bf16 rows converted to fp16, the packed codes of the stage are not looked at ----
+          bool bad = false;
+#pragma unroll
+          for (int kv = 0; kv < 2; ++kv) {
+            const __nv_bfloat16* src = (kv ? a.v_tail : a.k_tail) + tail_off + (int64_t)(slot0 - a.tail_lo) * a.tail_ts;
+            uint4 u[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) u[i] = *reinterpret_cast<const uint4*>(src + (int64_t)(16 * i) * a.tail_ts);
+            if (kv == 0) mbar_wait<256>(b_kfree + 8 * kbuf, (ku & 1) ^ 1, wc);
+            else mbar_wait<256>(b_vfree + 8 * vbuf, (vu & 1) ^ 1, wc);
+            uint8_t* dst = sgen + (kv ? kOffV + vbuf * 16384 : kOffK + kbuf * 16384) + row_off;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const uint4 hv = bf16x8_to_h8(u[i]);
+              bad |= h2_not_finite(hv.x) || h2_not_finite(hv.y) || h2_not_finite(hv.z) || h2_not_finite(hv.w);
+              *reinterpret_cast<uint4*>(dst + i * 2048) = hv;
+            }
+            fence_proxy_async();
+            mbar_arrive(kv ? b_vfull + 8 * vbuf : b_kfull + 8 * kbuf);
+          }
+          if (bad) report_range(a.status);
+          mbar_arrive(b_rfree + 8 * rs);
+          continue;
+        }
         if (BITS == 4) {
           // ---- fp16 parameter tables of this tile (one (group, channel) and one key per thread) ----
           uint8_t* tab = sgen + kOffTab + (g & 1) * kTabBytes;

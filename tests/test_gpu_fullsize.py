@@ -226,3 +226,42 @@ def test_ablation_budget_32768_int4(xkv):
     every item of the attention is cut into three or four pieces), first evicting frame 24."""
     cache, evicting = _stream(xkv, 1374, 32768, 26, seed=5, attn_from=24)
     assert cache.xkv_get_info().T == 32768 and evicting >= 2
+
+
+@pytest.mark.parametrize("variant", ["int4", "int4-tail", "bf16", "int4-once", "int8-once", "int4-20-blocks"])
+def test_attention_repeated_launches_are_bit_identical(xkv, variant):
+    """The attention kernel passes tensor-memory buffers between its warps through barriers (one score
+    buffer serves both query tiles in turn, P has two buffers per tile).  A protocol error there is a
+    race: it shows as launches on the same inputs that differ.  Full-size layer (1374 tokens, budget
+    16384, cache full and evicting), 12 launches per variant, outputs compared bit for bit."""
+    import torch
+    H, n, d = 16, 1374, 64
+    bits = 16 if variant == "bf16" else (8 if variant == "int8-once" else 4)
+    once = variant.endswith("once")
+    p = xkv.Params(n_heads=H, budget=16384, max_frame_tokens=n, kv_bits=bits, key_mode=xkv.KEYS_ONCE if once else 0)
+    cache = xkv.Cache(p)
+    if variant == "int4-20-blocks":
+        cache.xkv_debug_limit_attention_blocks(20)
+    q = torch.empty(H, n, d, dtype=torch.bfloat16, device="cuda")
+    k, v, out = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    for t in range(14):
+        for x, w in ((q, 0), (k, 1), (v, 2)):
+            xkv.xkv_synth_fill(x, 5, 0, t, w)
+        cache.step(q, k, v, out)
+    first = None
+    for rep in range(12):
+        cache.xkv_debug_rewind_attention()
+        out.zero_()
+        if variant == "int4-tail":
+            cache.attn_packed_causal_tail(q, k, v, out)
+        else:
+            cache.attn_packed_causal(q, out)
+        torch.cuda.synchronize()
+        assert cache.xkv_poll_status() == 0
+        bits_out = out.view(torch.int16).clone()
+        if first is None:
+            first = bits_out
+            assert bool(torch.isfinite(out.float()).all())
+        else:
+            assert torch.equal(first, bits_out), f"{variant}: launch {rep} differs from launch 0"
+    cache.close()

@@ -1227,7 +1227,7 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
     const uint32_t idesc_pv = make_idesc(64, kBf16, true);
     const uint64_t dq = make_desc(sQ + t * 16384);
     const uint32_t d_s = tmem + kColS1, d_p0 = tmem + kColP2 + 128 * t, d_o = tmem + kColO + 64 * t;
-    uint32_t g = 0, cq = 0, cp = 0, segq = 0;
+    uint32_t g = 0, cp = 0, segq = 0;
     uint32_t g_seg = 0;              // score-buffer uses before this segment
     for (long long pos = step_lo; pos < step_hi;) {
       const int item = (int)(pos / a.n_tiles);
@@ -1265,7 +1265,6 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
           for (int ks = 0; ks < 4; ++ks)   // 16 channels per step: 32 B inside the swizzle span
             mma_ss(d_s, dq + (uint64_t)(ks * 2), dk + (uint64_t)(ks * 2), idesc_qk, ks > 0 ? 1u : 0u);
           tc_commit(b_sfull + 8 * t);
-          ++cq;
         } else {
           // An item without a second tile: this thread follows the other tile's uses of the score
           // buffer one by one.  A parity wait is only sound while the waiter is at most one

@@ -34,7 +34,7 @@
 // rounding them to bf16 alone costs ~1e-2 relative L2 with outlier channels);
 // 16-bit caches hold bf16 and multiply in bf16.  Accumulation is fp32.
 //
-// Every mbarrier wait is bounded (by time: one second): when the bound is hit the thread records
+// Every mbarrier wait is bounded (one second of running time): when the bound is hit the thread records
 // XKV_E_TIMEOUT in the cache's status word and carries on without waiting, so the
 // kernel always terminates, drains its copies and frees its tensor memory.
 #include <mutex>
@@ -198,13 +198,17 @@ struct WaitCtx { int* status; volatile int* abort_flag; };
 // try suspended by the hardware for a short while: their wake-up latency is part of every step.
 // Threads that wait long and have slack (operand producers, the copy thread) sleep SLEEP_NS between
 // tries, so that their polls (shared-memory instructions) do not take issue slots and queue space
-// from the softmax warps.  The bound is one of time, looked at every 32 tries.
-constexpr uint64_t kWaitLimitNs = 1000000000ull;      // one second, then XKV_E_TIMEOUT
+// from the softmax warps.  The wait gives up after one second AND kWaitMinRounds rounds of tries
+// (32 or 64 each): the rounds only count while the thread runs, so that a kernel that was
+// descheduled for a while (a GPU shared between processes) does not time out on the clock alone.
+constexpr uint64_t kWaitLimitNs = 1000000000ull;      // one second ...
+constexpr uint32_t kWaitMinRounds = 1u << 12;         // ... and this many rounds, then XKV_E_TIMEOUT
 template <int SLEEP_NS = 32>
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc) {
   if (mbar_try(bar, parity)) return;          // the common case costs one instruction
   if (*wc.abort_flag) return;
   const uint64_t t0 = global_ns();
+  uint32_t rounds = 0;
   do {
     if (SLEEP_NS >= 128) {
 #pragma unroll 1
@@ -215,7 +219,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const W
     } else if (mbar_try_many(bar, parity)) {
       return;
     }
-  } while (global_ns() - t0 < kWaitLimitNs);
+  } while (++rounds < kWaitMinRounds || global_ns() - t0 < kWaitLimitNs);
   *wc.abort_flag = 1;
   atomicExch(wc.status, (int)XKV_E_TIMEOUT);
 }

@@ -48,6 +48,10 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 constexpr int kThreads = 480;
+// 16-warp form: registers per thread after the reallocation (softmax warps kSplitRegsSoftmax)
+constexpr int kSplitRegsSoftmax = 96;
+__host__ __device__ constexpr int split_regs_producers(bool once, bool tail) { return (once || tail) ? 56 : 40; }
+__host__ __device__ constexpr int split_regs_misc(bool once, bool tail) { return (once || tail) ? 40 : 48; }   // MMA issuers, copy thread
 constexpr int kThreadsSplit = 768;      // 16 softmax warps, 4 producers, 4 for the MMA issuers and the copies
 constexpr int kQRows = 128;
 constexpr int kMaxGrid = 160;                 // CTAs the scratch is sized for (>= SM count of the part)
@@ -490,8 +494,7 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
   constexpr int kSW = SPLIT ? 16 : 8;        // softmax warps
   constexpr uint32_t kRowThreads = SPLIT ? 256 : 128;   // threads that work on one query tile
   constexpr int kOffX = kOffRaw + C::kNR * C::kRawStage;   // exchange area of the split softmax
-  constexpr int kRegProd = (ONCE || TAIL) ? 56 : 40;      // registers per thread after the reallocation:
-  constexpr int kRegMisc = (ONCE || TAIL) ? 40 : 48;      // producers; MMA issuers and copy thread
+  constexpr int kRegProd = split_regs_producers(ONCE, TAIL), kRegMisc = split_regs_misc(ONCE, TAIL);
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
@@ -543,7 +546,7 @@ __global__ void __launch_bounds__(SPLIT ? kThreadsSplit : kThreads, 1) attn_tc_k
     // scores in registers.  The pool is what the CTA was launched with (per scheduler 6 warps x 80
     // registers per lane = 480); afterwards 4 x 96 + 40 + 48 (or 56 + 40 where the producers look up
     // per-token constants) of them are in use: 472 or 480.
-    if (warp < 16) asm volatile("setmaxnreg.inc.sync.aligned.u32 96;");
+    if (warp < 16) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSplitRegsSoftmax));
     else if (warp < 20) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegProd));
     else asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegMisc));
   }
@@ -1475,6 +1478,19 @@ struct TailArgs { const void* k; const void* v; int64_t ts, hs; };
 static std::mutex g_setup_mutex;
 static int g_sm_count[kMaxDevices] = {0};       // 0: not set up yet
 
+// The 16-warp form moves registers between its warps with setmaxnreg; the pool they move in is
+// what the CTA was launched with.  If a compiler ever gave the kernel fewer registers at launch
+// than the reallocation needs, setmaxnreg.inc would wait for ever: refuse to run instead.
+template <typename K>
+static cudaError_t check_register_pool(K kernel, bool once, bool tail) {
+  cudaFuncAttributes fa;
+  const cudaError_t e = cudaFuncGetAttributes(&fa, kernel);
+  if (e != cudaSuccess) return e;
+  const int warps_per_scheduler = kThreadsSplit / 32 / 4;
+  return (fa.numRegs * warps_per_scheduler >= 4 * kSplitRegsSoftmax + split_regs_producers(once, tail) + split_regs_misc(once, tail)) ? cudaSuccess
+                                                                                    : cudaErrorLaunchOutOfResources;
+}
+
 static cudaError_t attn_device_setup(int* sm_count) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
@@ -1496,6 +1512,12 @@ static cudaError_t attn_device_setup(int* sm_count) {
     e = cudaFuncSetAttribute(attn_tc_kernel<4, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<4>());
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_tc_kernel<8, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<8>());
+    if (e != cudaSuccess) return e;
+    e = check_register_pool(attn_tc_kernel<4, false, false, true>, false, false);
+    if (e != cudaSuccess) return e;
+    e = check_register_pool(attn_tc_kernel<16, false, false, true>, false, false);
+    if (e != cudaSuccess) return e;
+    e = check_register_pool(attn_tc_kernel<4, true, false, true>, false, true);
     if (e != cudaSuccess) return e;
     g_sm_count[dev] = sms;
   }
